@@ -1,0 +1,143 @@
+/*
+ * bwla.h - C ABI of the BWLA W1AX linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer (assembled from the paper's weight format Eq. 1-4, the Orthogonal-Kronecker
+ * Transformation of Sec. 3.1, the PSP residual of Sec. 3.2 and the per-token activation
+ * quantisation of Sec. 4.1), per token x_t in R^K:
+ *
+ *   Y_t   = P1^T * reshape(x_t, n1 x n2) * P2               (OKT applied online, K = n1*n2)
+ *   s_t   = max|Y_t| / qmax,  q_t = clamp(rne(Y_t / s_t))    (symmetric INT-b, qmax = 2^(b-1) - 1)
+ *   acc   = sum_k sign(W')[n][k] * q_t[k]                    (1-bit weights, exact int32)
+ *   out   = bf16( alpha[n] * s_t * acc + U[n,:] . (V x_t) [+ mu[n] * s_t * sum_k q_t[k]] )
+ *
+ * General rules for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller.  The library never allocates,
+ *     frees or keeps them.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - Calls are asynchronous on `stream`; nothing synchronises the host except bwla_check_status.
+ *   - Matrices are row-major.  bf16 data is passed as void* to 16-bit elements.
+ *   - Return value: BWLA_OK or a negative error code.  Invalid arguments never launch anything.
+ *   - There is no CPU fallback: on a machine without an sm_100 device the compute entry points
+ *     return BWLA_ERR_UNSUPPORTED.
+ *   - Packed sign format: uint32 words, row-major [N][K/32]; weight k of output row n is bit
+ *     (k & 31) of word (k >> 5); bit 1 means +1, bit 0 means -1.  Sign(w) = +1 iff w > 0 (Eq. 3),
+ *     so 0, -0.0 and NaN pack as -1.
+ */
+#ifndef BWLA_H_
+#define BWLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    BWLA_OK = 0,
+    BWLA_ERR_INVALID_ARG = -1,     /* NULL pointer, bad dimension, K != n1*n2, K % 32 != 0, bits not in {4,6,8}, ... */
+    BWLA_ERR_UNSUPPORTED = -2,     /* no sm_100 device is current */
+    BWLA_ERR_WORKSPACE = -3,       /* workspace NULL, misaligned (256 B) or smaller than bwla_workspace_bytes */
+    BWLA_ERR_CUDA = -4,            /* a CUDA call failed; see bwla_last_cuda_error */
+    BWLA_ERR_DEVICE_TIMEOUT = -5   /* a bounded device-side wait ran out (only from bwla_check_status) */
+};
+
+/* Kernel families the layer can run its contraction on (see bwla_force_path). */
+enum {
+    BWLA_PATH_AUTO = 0,       /* per-shape choice */
+    BWLA_PATH_SIMPLE = 1,     /* one-thread-per-output CUDA kernel: slow, used as an on-device cross-check */
+    BWLA_PATH_BITPLANE = 2,   /* activation bit-planes x packed weight bits, AND-popcount tensor-core MMA */
+    BWLA_PATH_I8 = 3          /* weights expanded to +-1 int8 in shared memory, tcgen05 kind::i8 into TMEM */
+};
+
+#define BWLA_DTYPE_F32 0
+#define BWLA_DTYPE_BF16 1
+
+/*
+ * Binarise already rotated/centred weights: packed[n][k>>5] bit (k&31) = (W'[n][k] > 0).   (Eq. 2-3)
+ *   w      device, [N][ldw] fp32 (dtype 0) or bf16 (dtype 1), ldw >= K elements
+ *   packed device, uint32 [N][K/32], written in full
+ *   K must be a positive multiple of 32; N >= 0 (N == 0 is a no-op).
+ */
+int bwla_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw,
+                    uint32_t* packed, void* stream);
+
+/*
+ * Online OKT + per-token symmetric quantisation.   (Sec. 3.1 Kronecker evaluation; Sec. 4.1 per-token)
+ *   x_bf16 device, bf16 [M][ldx], ldx >= K
+ *   P1     device, fp32 [n1][n1];  P2 device, fp32 [n2][n2];  n1*n2 == K
+ *   bits   4, 6 or 8;  qmax = 2^(bits-1) - 1; the most negative code is never produced
+ *   codes  device, int8 [M][K];  scales device, fp32 [M]   (both written in full)
+ * Arithmetic: fp32 accumulation; s_t = amax / qmax; q = rne(Y * (qmax / amax)); an all-zero row
+ * gives s_t = 1 and zero codes.  M == 0 is a no-op.  K must be a multiple of 32, K <= 65536 and
+ * 8*K bytes of shared memory must fit one block (K <= 25600 elements).
+ */
+int bwla_rotate_quant_act(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                          const float* P1, int n1, const float* P2, int n2, int bits,
+                          int8_t* codes, float* scales, void* stream);
+
+/*
+ * Bytes of scratch bwla_w1ax_linear / bwla_w1a_gemm_codes need for this problem (a multiple of 256).
+ * Returns 0 for invalid dimensions.
+ */
+size_t bwla_workspace_bytes(int64_t M, int64_t K, int64_t N, int r, int bits);
+
+/*
+ * The whole layer (formula at the top of this file).
+ *   packed device uint32 [N][K/32];  alpha device fp32 [N];  mu device fp32 [N] or NULL   (Eq. 4)
+ *   U_bf16 device bf16 [N][r], V_bf16 device bf16 [r][K]; both may be NULL iff r == 0      (Sec. 3.2, M = A B)
+ *   out_bf16 device bf16 [M][ldo], ldo >= N
+ *   workspace device, 256-byte aligned, >= bwla_workspace_bytes(M,K,N,r,bits); contents are scratch.
+ *     Its first word is a status word that bounded device-side waits set; read it with bwla_check_status.
+ *   Two calls that share a workspace must be ordered on one stream.
+ */
+int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                     const float* P1, int n1, const float* P2, int n2, int bits,
+                     const uint32_t* packed, const float* alpha, const float* mu,
+                     const void* U_bf16, const void* V_bf16, int r,
+                     void* out_bf16, int64_t N, int64_t ldo,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Contraction + epilogue from given codes (the part of the layer after the quantiser), so that
+ * integer accumulators can be compared for identical codes.
+ *   codes device int8 [M][K]; scales device fp32 [M]
+ *   x_bf16 (with ldx) is only read for the low-rank branch and may be NULL iff r == 0
+ *   out_bf16 may be NULL when only accumulators are wanted
+ *   acc_debug device int32 [M][N] or NULL: receives sum_k sign[n][k] * codes[t][k]
+ */
+int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int64_t K, int bits,
+                        const uint32_t* packed, const float* alpha, const float* mu,
+                        const void* x_bf16, int64_t ldx,
+                        const void* U_bf16, const void* V_bf16, int r,
+                        void* out_bf16, int64_t N, int64_t ldo, int32_t* acc_debug,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronise `stream`, read the workspace status word and clear it.
+ * Returns BWLA_OK, BWLA_ERR_DEVICE_TIMEOUT (a device-side wait gave up; outputs of that call are
+ * invalid but the context stays usable) or BWLA_ERR_CUDA.
+ */
+int bwla_check_status(void* workspace, void* stream);
+
+/* Force every later call in this process onto one kernel family (benchmarking the non-chosen path,
+ * cross-checks).  Returns BWLA_ERR_INVALID_ARG for an unknown value.  Not thread-safe against
+ * concurrent compute calls. */
+int bwla_force_path(int path);
+
+/* The family BWLA_PATH_AUTO resolves to for this problem (no launch). */
+int bwla_chosen_path(int64_t M, int64_t K, int64_t N, int r, int bits);
+
+/* Number of kernels the most recent bwla_w1ax_linear / bwla_w1a_gemm_codes / bwla_rotate_quant_act /
+ * bwla_pack_signs call on this thread launched. */
+int bwla_last_launch_count(void);
+
+/* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
+int bwla_last_cuda_error(void);
+
+/* Static, human-readable name of a status code. */
+const char* bwla_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BWLA_H_ */

@@ -1,0 +1,226 @@
+"""Thin Python binding of the C ABI in ``include/bwla.h``.
+
+Argument marshalling only: each function here checks tensor types, takes ``data_ptr()`` and the current CUDA
+stream from PyTorch and calls the entry point of the same name in ``libbwla.so``.  Every step of the layer
+runs in the library's CUDA kernels.  There is no fallback: if the shared object is missing the import fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbwla.so")
+
+BWLA_OK = 0
+BWLA_ERR_INVALID_ARG = -1
+BWLA_ERR_UNSUPPORTED = -2
+BWLA_ERR_WORKSPACE = -3
+BWLA_ERR_CUDA = -4
+BWLA_ERR_DEVICE_TIMEOUT = -5
+
+BWLA_PATH_AUTO = 0
+BWLA_PATH_SIMPLE = 1
+BWLA_PATH_BITPLANE = 2
+BWLA_PATH_I8 = 3
+
+EXPORTS = [
+    "bwla_pack_signs", "bwla_rotate_quant_act", "bwla_workspace_bytes", "bwla_w1ax_linear", "bwla_w1a_gemm_codes",
+    "bwla_check_status", "bwla_force_path", "bwla_chosen_path", "bwla_last_launch_count", "bwla_last_cuda_error",
+    "bwla_status_string",
+]
+
+
+class BwlaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {bwla_status_string(status)} (cuda error {bwla_last_cuda_error()})")
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2605_00422_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    lib = C.CDLL(LIB_PATH)
+    i64, vp, ci, sz = C.c_int64, C.c_void_p, C.c_int, C.c_size_t
+    lib.bwla_pack_signs.argtypes = [vp, ci, i64, i64, i64, vp, vp]
+    lib.bwla_rotate_quant_act.argtypes = [vp, i64, i64, i64, vp, ci, vp, ci, ci, vp, vp, vp]
+    lib.bwla_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
+    lib.bwla_workspace_bytes.restype = sz
+    lib.bwla_w1ax_linear.argtypes = [vp, i64, i64, i64, vp, ci, vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, i64, i64,
+                                     vp, sz, vp]
+    lib.bwla_w1a_gemm_codes.argtypes = [vp, vp, i64, i64, ci, vp, vp, vp, vp, i64, vp, vp, ci, vp, i64, i64, vp,
+                                        vp, sz, vp]
+    lib.bwla_check_status.argtypes = [vp, vp]
+    lib.bwla_force_path.argtypes = [ci]
+    lib.bwla_chosen_path.argtypes = [i64, i64, i64, ci, ci]
+    lib.bwla_status_string.argtypes = [ci]
+    lib.bwla_status_string.restype = C.c_char_p
+    for name in ("bwla_pack_signs", "bwla_rotate_quant_act", "bwla_w1ax_linear", "bwla_w1a_gemm_codes",
+                 "bwla_check_status", "bwla_force_path", "bwla_chosen_path", "bwla_last_launch_count",
+                 "bwla_last_cuda_error"):
+        getattr(lib, name).restype = ci
+    return lib
+
+
+_lib = _load()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _need(t: torch.Tensor, dtype, name: str, ndim: Optional[int] = None):
+    if not t.is_cuda or t.dtype != dtype or (ndim is not None and t.dim() != ndim):
+        raise TypeError(f"{name}: expected a CUDA tensor of {dtype}" + (f" with {ndim} dims" if ndim else ""))
+    if t.stride(-1) != 1 and t.numel() > 0:
+        raise TypeError(f"{name}: innermost dimension must be contiguous")
+
+
+def _check(status: int, where: str):
+    if status != BWLA_OK:
+        raise BwlaError(status, where)
+
+
+def bwla_status_string(status: int) -> str:
+    return _lib.bwla_status_string(status).decode()
+
+
+def bwla_last_cuda_error() -> int:
+    return int(_lib.bwla_last_cuda_error())
+
+
+def bwla_last_launch_count() -> int:
+    return int(_lib.bwla_last_launch_count())
+
+
+def bwla_force_path(path: int) -> None:
+    _check(_lib.bwla_force_path(path), "bwla_force_path")
+
+
+def bwla_chosen_path(M: int, K: int, N: int, r: int, bits: int) -> int:
+    return int(_lib.bwla_chosen_path(M, K, N, r, bits))
+
+
+def bwla_workspace_bytes(M: int, K: int, N: int, r: int, bits: int) -> int:
+    return int(_lib.bwla_workspace_bytes(M, K, N, r, bits))
+
+
+def new_workspace(M: int, K: int, N: int, r: int, bits: int, device="cuda") -> torch.Tensor:
+    """Scratch buffer for bwla_w1ax_linear / bwla_w1a_gemm_codes (device memory from PyTorch, zero-filled)."""
+    n = bwla_workspace_bytes(M, K, N, r, bits)
+    if n == 0:
+        raise ValueError("invalid dimensions")
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def bwla_pack_signs(w: torch.Tensor, packed: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """w: fp32 or bf16 [N][K] (row stride >= K) -> uint32 words stored as int32 [N][K/32]."""
+    if w.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("w must be fp32 or bf16")
+    _need(w, w.dtype, "w", 2)
+    N, K = w.shape
+    if packed is None:
+        packed = torch.empty((N, K // 32), dtype=torch.int32, device=w.device)
+    _need(packed, torch.int32, "packed", 2)
+    st = _lib.bwla_pack_signs(_ptr(w), 0 if w.dtype == torch.float32 else 1, N, K, w.stride(0) if N > 0 else K,
+                              _ptr(packed), _stream())
+    _check(st, "bwla_pack_signs")
+    return packed
+
+
+def bwla_rotate_quant_act(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, bits: int,
+                          codes: Optional[torch.Tensor] = None, scales: Optional[torch.Tensor] = None):
+    """x: bf16 [M][K]; P1 fp32 [n1][n1]; P2 fp32 [n2][n2] -> (codes int8 [M][K], scales fp32 [M])."""
+    _need(x, torch.bfloat16, "x", 2)
+    _need(P1, torch.float32, "P1", 2)
+    _need(P2, torch.float32, "P2", 2)
+    M, K = x.shape
+    if codes is None:
+        codes = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    if scales is None:
+        scales = torch.empty((M,), dtype=torch.float32, device=x.device)
+    st = _lib.bwla_rotate_quant_act(_ptr(x), M, K, x.stride(0) if M > 0 else K, _ptr(P1.contiguous()), P1.shape[0],
+                                    _ptr(P2.contiguous()), P2.shape[0], bits, _ptr(codes), _ptr(scales), _stream())
+    _check(st, "bwla_rotate_quant_act")
+    return codes, scales
+
+
+def bwla_w1ax_linear(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, bits: int, packed: torch.Tensor,
+                     alpha: torch.Tensor, U: Optional[torch.Tensor] = None, V: Optional[torch.Tensor] = None,
+                     mu: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                     workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The whole layer: bf16 x [M][K] -> bf16 out [M][N]."""
+    _need(x, torch.bfloat16, "x", 2)
+    _need(packed, torch.int32, "packed", 2)
+    _need(alpha, torch.float32, "alpha", 1)
+    M, K = x.shape
+    N = packed.shape[0]
+    r = 0
+    if U is not None:
+        _need(U, torch.bfloat16, "U", 2)
+        _need(V, torch.bfloat16, "V", 2)
+        r = U.shape[1]
+        if not (U.is_contiguous() and V.is_contiguous()) or tuple(V.shape) != (r, K) or U.shape[0] != N:
+            raise TypeError("U must be contiguous [N][r] and V contiguous [r][K]")
+    if mu is not None:
+        _need(mu, torch.float32, "mu", 1)
+    if not (packed.is_contiguous() and P1.is_contiguous() and P2.is_contiguous()):
+        raise TypeError("packed, P1 and P2 must be contiguous")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    _need(out, torch.bfloat16, "out", 2)
+    if workspace is None:
+        workspace = new_workspace(M, K, N, r, bits, x.device)
+    st = _lib.bwla_w1ax_linear(_ptr(x), M, K, x.stride(0) if M > 0 else K, _ptr(P1), P1.shape[0], _ptr(P2),
+                               P2.shape[0], bits, _ptr(packed), _ptr(alpha), _ptr(mu), _ptr(U), _ptr(V), r,
+                               _ptr(out), N, out.stride(0) if M > 0 else N, _ptr(workspace), workspace.numel(),
+                               _stream())
+    _check(st, "bwla_w1ax_linear")
+    return out
+
+
+def bwla_w1a_gemm_codes(codes: torch.Tensor, scales: torch.Tensor, bits: int, packed: torch.Tensor,
+                        alpha: torch.Tensor, x: Optional[torch.Tensor] = None, U: Optional[torch.Tensor] = None,
+                        V: Optional[torch.Tensor] = None, mu: Optional[torch.Tensor] = None,
+                        out: Optional[torch.Tensor] = None, acc: Optional[torch.Tensor] = None,
+                        want_out: bool = True, want_acc: bool = False, workspace: Optional[torch.Tensor] = None):
+    """Contraction + epilogue from given int8 codes [M][K]; returns (out bf16 or None, acc int32 or None)."""
+    _need(codes, torch.int8, "codes", 2)
+    _need(scales, torch.float32, "scales", 1)
+    _need(packed, torch.int32, "packed", 2)
+    _need(alpha, torch.float32, "alpha", 1)
+    M, K = codes.shape
+    N = packed.shape[0]
+    r = 0
+    if U is not None:
+        _need(U, torch.bfloat16, "U", 2)
+        _need(V, torch.bfloat16, "V", 2)
+        _need(x, torch.bfloat16, "x", 2)
+        r = U.shape[1]
+    if not codes.is_contiguous() or not packed.is_contiguous():
+        raise TypeError("codes and packed must be contiguous")
+    if out is None and want_out:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=codes.device)
+    if acc is None and want_acc:
+        acc = torch.empty((M, N), dtype=torch.int32, device=codes.device)
+    if workspace is None:
+        workspace = new_workspace(M, K, N, r, bits, codes.device)
+    st = _lib.bwla_w1a_gemm_codes(_ptr(codes), _ptr(scales), M, K, bits, _ptr(packed), _ptr(alpha), _ptr(mu),
+                                  _ptr(x), x.stride(0) if (x is not None and M > 0) else K, _ptr(U), _ptr(V), r,
+                                  _ptr(out), N, out.stride(0) if (out is not None and M > 0) else N, _ptr(acc),
+                                  _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "bwla_w1a_gemm_codes")
+    return out, acc
+
+
+def bwla_check_status(workspace: torch.Tensor) -> int:
+    """Synchronises the current stream and returns the status a bounded device-side wait may have left."""
+    return int(_lib.bwla_check_status(_ptr(workspace), _stream()))

@@ -1,0 +1,195 @@
+// extern "C" boundary: argument validation, workspace carving and per-shape dispatch.  No compute happens here.
+#include "bwla_common.cuh"
+
+namespace bwla {
+
+thread_local int g_last_cuda_error = 0;
+thread_local int g_launch_count = 0;
+static int g_forced_path = BWLA_PATH_AUTO;
+
+static bool valid_bits(int bits) { return bits == 4 || bits == 6 || bits == 8; }
+
+// The compute entry points need an sm_100 device to be current.
+static int check_device() {
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; cudaGetLastError(); return BWLA_ERR_UNSUPPORTED; }
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; cudaGetLastError(); return BWLA_ERR_UNSUPPORTED; }
+    return major == 10 ? BWLA_OK : BWLA_ERR_UNSUPPORTED;
+}
+
+static bool valid_rotation_dims(int64_t K, int n1, int n2) {
+    return K > 0 && K % 32 == 0 && K <= 25600 && n1 > 0 && n2 > 0 && (int64_t)n1 * n2 == K;
+}
+
+static int resolve_path(int64_t M, int64_t K, int64_t N, int r, int bits) {
+    (void)M; (void)K; (void)N; (void)r; (void)bits;
+    if (g_forced_path != BWLA_PATH_AUTO) return g_forced_path;
+    return BWLA_PATH_SIMPLE;
+}
+
+static int run_contraction(int path, GemmArgs& g, const int8_t* codes_natural, cudaStream_t stream) {
+    (void)path;
+    g.codes = codes_natural;
+    return launch_gemm_simple(g, stream);
+}
+
+}  // namespace bwla
+
+using namespace bwla;
+
+extern "C" {
+
+int bwla_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw, uint32_t* packed, void* stream) {
+    g_launch_count = 0;
+    if (N < 0 || K <= 0 || K % 32 != 0 || ldw < K || (dtype != BWLA_DTYPE_F32 && dtype != BWLA_DTYPE_BF16))
+        return BWLA_ERR_INVALID_ARG;
+    if (N == 0) return BWLA_OK;
+    if (!w || !packed) return BWLA_ERR_INVALID_ARG;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+    return launch_pack_signs(w, dtype, N, K, ldw, packed, (cudaStream_t)stream);
+}
+
+int bwla_rotate_quant_act(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1,
+                          const float* P2, int n2, int bits, int8_t* codes, float* scales, void* stream) {
+    g_launch_count = 0;
+    if (M < 0 || !valid_rotation_dims(K, n1, n2) || ldx < K || !valid_bits(bits)) return BWLA_ERR_INVALID_ARG;
+    if (M == 0) return BWLA_OK;
+    if (!x_bf16 || !P1 || !P2 || !codes || !scales) return BWLA_ERR_INVALID_ARG;
+    if (((uintptr_t)codes & 15) || ((uintptr_t)P1 & 15) || ((uintptr_t)P2 & 15)) return BWLA_ERR_INVALID_ARG;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+    return launch_rotate_quant(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, 0, scales, nullptr, nullptr,
+                               nullptr, (cudaStream_t)stream);
+}
+
+size_t bwla_workspace_bytes(int64_t M, int64_t K, int64_t N, int r, int bits) {
+    if (M < 0 || K <= 0 || K % 32 != 0 || N < 0 || r < 0 || !valid_bits(bits)) return 0;
+    return workspace_layout(M, K, N, r, bits).total;
+}
+
+static int validate_gemm_tail(int64_t M, int64_t K, int bits, const uint32_t* packed, const float* alpha,
+                              const void* U, const void* V, int r, int64_t N, int64_t ldo, const void* workspace,
+                              size_t workspace_bytes) {
+    if (M < 0 || N < 0 || K <= 0 || K % 32 != 0 || r < 0 || r > 256 || !valid_bits(bits)) return BWLA_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return BWLA_OK;
+    if (!packed || !alpha || ldo < N) return BWLA_ERR_INVALID_ARG;
+    if (r > 0 && (!U || !V)) return BWLA_ERR_INVALID_ARG;
+    if (((uintptr_t)packed & 15)) return BWLA_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < workspace_layout(M, K, N, r, bits).total)
+        return BWLA_ERR_WORKSPACE;
+    return BWLA_OK;
+}
+
+int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2,
+                     int n2, int bits, const uint32_t* packed, const float* alpha, const float* mu, const void* U_bf16,
+                     const void* V_bf16, int r, void* out_bf16, int64_t N, int64_t ldo, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    g_launch_count = 0;
+    if (!valid_rotation_dims(K, n1, n2) || ldx < K) return BWLA_ERR_INVALID_ARG;
+    int st = validate_gemm_tail(M, K, bits, packed, alpha, U_bf16, V_bf16, r, N, ldo, workspace, workspace_bytes);
+    if (st != BWLA_OK) return st;
+    if (M == 0 || N == 0) return BWLA_OK;
+    if (!x_bf16 || !P1 || !P2 || !out_bf16) return BWLA_ERR_INVALID_ARG;
+    if (((uintptr_t)P1 & 15) || ((uintptr_t)P2 & 15)) return BWLA_ERR_INVALID_ARG;
+    st = check_device();
+    if (st != BWLA_OK) return st;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const Workspace ws = workspace_layout(M, K, N, r, bits);
+    char* base = (char*)workspace;
+    float* scales = (float*)(base + ws.scales);
+    int32_t* qsum = (int32_t*)(base + ws.qsum);
+    float* T = (float*)(base + ws.T);
+    int8_t* codes = (int8_t*)(base + ws.codes);
+    const int path = resolve_path(M, K, N, r, bits);
+
+    st = launch_rotate_quant(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, 0, scales, qsum, nullptr,
+                             (uint32_t*)(base + ws.status), s);
+    if (st != BWLA_OK) return st;
+    if (r > 0) {
+        st = launch_lowrank_T(x_bf16, M, K, ldx, V_bf16, r, T, s);
+        if (st != BWLA_OK) return st;
+    }
+    GemmArgs g{};
+    g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
+    g.mu = mu; g.T = r > 0 ? T : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = nullptr;
+    g.status = (uint32_t*)(base + ws.status);
+    return run_contraction(path, g, codes, s);
+}
+
+int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int64_t K, int bits,
+                        const uint32_t* packed, const float* alpha, const float* mu, const void* x_bf16, int64_t ldx,
+                        const void* U_bf16, const void* V_bf16, int r, void* out_bf16, int64_t N, int64_t ldo,
+                        int32_t* acc_debug, void* workspace, size_t workspace_bytes, void* stream) {
+    g_launch_count = 0;
+    int st = validate_gemm_tail(M, K, bits, packed, alpha, U_bf16, V_bf16, r, N, ldo, workspace, workspace_bytes);
+    if (st != BWLA_OK) return st;
+    if (M == 0 || N == 0) return BWLA_OK;
+    if (!codes || !scales || (!out_bf16 && !acc_debug)) return BWLA_ERR_INVALID_ARG;
+    if (((uintptr_t)codes & 15)) return BWLA_ERR_INVALID_ARG;
+    if (r > 0 && (!x_bf16 || ldx < K)) return BWLA_ERR_INVALID_ARG;
+    st = check_device();
+    if (st != BWLA_OK) return st;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const Workspace ws = workspace_layout(M, K, N, r, bits);
+    char* base = (char*)workspace;
+    int32_t* qsum = (int32_t*)(base + ws.qsum);
+    float* T = (float*)(base + ws.T);
+    const int path = resolve_path(M, K, N, r, bits);
+
+    st = launch_prepare_codes(codes, M, K, nullptr, qsum, (uint32_t*)(base + ws.status), s);
+    if (st != BWLA_OK) return st;
+    if (r > 0) {
+        st = launch_lowrank_T(x_bf16, M, K, ldx, V_bf16, r, T, s);
+        if (st != BWLA_OK) return st;
+    }
+    GemmArgs g{};
+    g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
+    g.mu = mu; g.T = r > 0 ? T : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = acc_debug;
+    g.status = (uint32_t*)(base + ws.status);
+    return run_contraction(path, g, codes, s);
+}
+
+int bwla_check_status(void* workspace, void* stream) {
+    if (!workspace) return BWLA_ERR_INVALID_ARG;
+    uint32_t host[4] = {0, 0, 0, 0};
+    cudaStream_t s = (cudaStream_t)stream;
+    BWLA_CUDA_TRY(cudaMemcpyAsync(host, workspace, sizeof(host), cudaMemcpyDeviceToHost, s));
+    BWLA_CUDA_TRY(cudaStreamSynchronize(s));
+    if (host[0] != 0) {
+        BWLA_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBytes, s));
+        BWLA_CUDA_TRY(cudaStreamSynchronize(s));
+        return BWLA_ERR_DEVICE_TIMEOUT;
+    }
+    return BWLA_OK;
+}
+
+int bwla_force_path(int path) {
+    if (path < BWLA_PATH_AUTO || path > BWLA_PATH_I8) return BWLA_ERR_INVALID_ARG;
+    g_forced_path = path;
+    return BWLA_OK;
+}
+
+int bwla_chosen_path(int64_t M, int64_t K, int64_t N, int r, int bits) { return resolve_path(M, K, N, r, bits); }
+
+int bwla_last_launch_count(void) { return g_launch_count; }
+
+int bwla_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* bwla_status_string(int status) {
+    switch (status) {
+        case BWLA_OK: return "BWLA_OK";
+        case BWLA_ERR_INVALID_ARG: return "BWLA_ERR_INVALID_ARG";
+        case BWLA_ERR_UNSUPPORTED: return "BWLA_ERR_UNSUPPORTED";
+        case BWLA_ERR_WORKSPACE: return "BWLA_ERR_WORKSPACE";
+        case BWLA_ERR_CUDA: return "BWLA_ERR_CUDA";
+        case BWLA_ERR_DEVICE_TIMEOUT: return "BWLA_ERR_DEVICE_TIMEOUT";
+        default: return "BWLA_ERR_UNKNOWN";
+    }
+}
+
+}  // extern "C"

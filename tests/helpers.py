@@ -1,0 +1,92 @@
+"""Shared pieces of the GPU parity tests: host<->device marshalling and the comparison rules.
+
+Tolerances (all stated here, used by every parity test):
+  * packed sign words, int32 accumulators for identical codes: bit-exact.
+  * quantised codes: bit-exact against the fp64 oracle except where the oracle's pre-rounding value lies within
+    1e-6 * qmax (1e-6 of the token's full scale, in code units) of a rounding boundary; such mismatches must be
+    exactly +-1 and are counted.
+  * per-token scale: within 2 fp32 ulp of amax / qmax.
+  * bf16 output: relative L2 error <= 2e-3; every element within 1 bf16 ulp of the correctly rounded oracle value
+    or within 1e-2 * rms(y) + 2^-8 * |y| of the fp64 oracle value (a correctly rounded bf16 is already up to
+    2^-9 * |y| away, so the absolute bound alone cannot hold for elements several rms large).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2605_00422_b200 import inputs as gen
+
+
+def bf16_to_dev(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def bf16_to_host(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def words_to_dev(packed: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(packed).view(np.int32)).cuda()
+
+
+def words_to_host(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().cpu().numpy().view(np.uint32)
+
+
+def f32_to_dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+
+
+class DeviceLayer:
+    """One layer's static tensors on the device plus the host copies the oracle needs."""
+
+    def __init__(self, lay: gen.LayerTensors, bwla):
+        self.lay = lay
+        self.P1 = f32_to_dev(lay.P1)
+        self.P2 = f32_to_dev(lay.P2)
+        self.alpha = f32_to_dev(lay.alpha)
+        self.U = bf16_to_dev(lay.U) if lay.U is not None else None
+        self.V = bf16_to_dev(lay.V) if lay.V is not None else None
+        self.mu = f32_to_dev(lay.mu) if lay.mu is not None else None
+        if lay.packed is not None:
+            self.packed_host = lay.packed
+            self.packed = words_to_dev(lay.packed)
+        else:
+            self.packed = bwla.bwla_pack_signs(f32_to_dev(lay.W))
+            self.packed_host = words_to_host(self.packed)
+
+
+def check_codes(gpu_codes: np.ndarray, gpu_scales: np.ndarray, Y: np.ndarray, bits: int) -> dict:
+    """The benchmark spec rule for the integer codes; returns counts for the report."""
+    ref = oracle.quantize(Y, bits, "f64")
+    diff = gpu_codes.astype(np.int32) - ref["codes"].astype(np.int32)
+    bad = diff != 0
+    window = oracle.near_tie_window(bits)
+    flagged = ref["dist"] <= window
+    unflagged = bad & ~flagged
+    assert np.all(np.abs(diff[bad]) == 1), "a code differs from the oracle by more than one step"
+    assert not unflagged.any(), (
+        f"{int(unflagged.sum())} code mismatches outside the near-tie window; "
+        f"worst distance to a boundary {ref['dist'][unflagged].max():.3e} (window {window:.1e})")
+    ulp = np.spacing(ref["scales"].astype(np.float32))
+    assert np.all(np.abs(gpu_scales.astype(np.float64) - ref["scales"].astype(np.float64)) <= 2 * ulp)
+    return {"near_ties": int(flagged.sum()), "mismatches": int(bad.sum()), "elements": int(bad.size)}
+
+
+def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray) -> dict:
+    got = gen.f32_from_bf16_bits(gpu_bits).astype(np.float64)
+    err = got - y_ref
+    rel_l2 = float(np.linalg.norm(err) / max(np.linalg.norm(y_ref), 1e-300))
+    rms = float(np.sqrt(np.mean(y_ref ** 2)))
+    assert rel_l2 <= 2e-3, f"relative L2 error {rel_l2:.3e} > 2e-3"
+    bound = 1e-2 * rms + 2.0 ** -8 * np.abs(y_ref)
+    assert np.all(np.abs(err) <= bound), f"max |err| {np.abs(err).max():.3e} exceeds 1e-2*rms + 2^-8*|y|"
+    # distance to the correctly rounded value, in bf16 steps of the reference
+    ref_bits = oracle.bf16_round(y_ref)
+    ref_val = gen.f32_from_bf16_bits(ref_bits).astype(np.float64)
+    step = np.maximum(np.abs(ref_val), 2.0 ** -126) * 2.0 ** -7
+    ulps = np.abs(got - ref_val) / step
+    return {"rel_l2": rel_l2, "max_abs_over_rms": float(np.abs(err).max() / max(rms, 1e-300)),
+            "max_bf16_steps": float(ulps.max()), "exact_bf16": float(np.mean(gpu_bits == ref_bits))}

@@ -1,0 +1,189 @@
+"""Parity of the CUDA path (called through the C ABI) with the CPU oracle, element by element.
+
+The tolerances are stated in tests/helpers.py.  All inputs are seeded and synthetic.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_00422_b200 import inputs as gen
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bwla():
+    from paper_2605_00422_b200 import bwla as b
+    b.bwla_force_path(b.BWLA_PATH_AUTO)
+    return b
+
+
+# ------------------------------------------------------------------------------------------------
+# pack_signs
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N,K", [(1, 32), (5, 96), (130, 1024), (33, 11008)])
+def test_pack_signs_bit_exact(bwla, N, K):
+    rng = np.random.default_rng(N * 7 + K)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    W[0, :3] = [0.0, -0.0, np.nan]
+    got = H.words_to_host(bwla.bwla_pack_signs(torch.from_numpy(W).cuda()))
+    assert np.array_equal(got, oracle.pack_signs(W))
+    Wb = gen.bf16_bits_from_f32(W)
+    got_b = H.words_to_host(bwla.bwla_pack_signs(H.bf16_to_dev(Wb)))
+    assert np.array_equal(got_b, oracle.pack_signs_bf16(Wb))
+
+
+def test_pack_signs_strided_and_empty(bwla):
+    W = torch.randn(7, 128, device="cuda")
+    view = W[:, :64]
+    got = H.words_to_host(bwla.bwla_pack_signs(view))
+    assert np.array_equal(got, oracle.pack_signs(view.cpu().numpy()))
+    assert bwla.bwla_pack_signs(torch.empty(0, 64, device="cuda")).shape == (0, 2)
+
+
+# ------------------------------------------------------------------------------------------------
+# rotate + quantise
+# ------------------------------------------------------------------------------------------------
+ROT_CASES = [
+    # (n1, n2, M, bits)
+    (32, 32, 16, 6),      # config 0
+    (8, 12, 3, 6),        # n2 multiple of 4, tiny
+    (4, 8, 5, 4),         # K = 32, a single word
+    (32, 3, 2, 8),        # n2 not a multiple of 4: scalar contraction
+    (64, 80, 9, 6),       # Qwen3 hidden 5120
+    (86, 128, 4, 6),      # LLaMA down_proj, n1 not a multiple of 4
+    (64, 128, 4, 8),
+    (160, 160, 3, 4),     # largest K (25600)
+]
+
+
+@pytest.mark.parametrize("n1,n2,M,bits", ROT_CASES)
+def test_rotate_quant_codes_and_scales(bwla, n1, n2, M, bits):
+    K = n1 * n2
+    shape = gen.small_shape(K, 32, n1, n2, 0, shape_id=n1 * 1000 + n2)
+    lay = gen.make_layer(0, shape, bits)
+    xb = gen.make_activations(0, shape, M)
+    codes, scales = bwla.bwla_rotate_quant_act(H.bf16_to_dev(xb), H.f32_to_dev(lay.P1), H.f32_to_dev(lay.P2), bits)
+    Y = oracle.rotate(xb, lay.P1, lay.P2)
+    rep = H.check_codes(codes.cpu().numpy(), scales.cpu().numpy(), Y, bits)
+    assert rep["mismatches"] <= max(4, rep["elements"] // 10000)
+
+
+def test_rotate_quant_heavy_tails_all_bit_widths(bwla):
+    # config 3 recipe: Student-t nu = 2.5, 1 % of channels x100
+    shape = gen.CONFIG_SHAPES[3][0]
+    lay = gen.make_layer(3, shape, 6)
+    xb = gen.make_activations(3, shape, 4)
+    Y = oracle.rotate(xb, lay.P1, lay.P2)
+    xd, P1, P2 = H.bf16_to_dev(xb), H.f32_to_dev(lay.P1), H.f32_to_dev(lay.P2)
+    for bits in (4, 6, 8):
+        codes, scales = bwla.bwla_rotate_quant_act(xd, P1, P2, bits)
+        H.check_codes(codes.cpu().numpy(), scales.cpu().numpy(), Y, bits)
+
+
+def test_rotate_quant_degenerate_rows_and_strided_input(bwla):
+    n1, n2, bits = 8, 8, 6
+    x = np.zeros((4, 64), np.float32)
+    x[1, 5] = 3.0                                  # a single non-zero entry
+    x[2, :] = 1.0                                  # constant row
+    x[3, :] = np.linspace(-1, 1, 64)
+    xb = gen.bf16_bits_from_f32(x)
+    eye = torch.eye(8, device="cuda")
+    wide = torch.zeros(4, 128, dtype=torch.bfloat16, device="cuda")
+    wide[:, :64] = H.bf16_to_dev(xb)
+    codes, scales = bwla.bwla_rotate_quant_act(wide[:, :64], eye, eye, bits)
+    Y = oracle.rotate(xb, np.eye(8, dtype=np.float32), np.eye(8, dtype=np.float32))
+    H.check_codes(codes.cpu().numpy(), scales.cpu().numpy(), Y, bits)
+    assert scales[0].item() == 1.0 and int(codes[0].abs().max()) == 0
+    c0, s0 = bwla.bwla_rotate_quant_act(torch.empty(0, 64, dtype=torch.bfloat16, device="cuda"), eye, eye, bits)
+    assert c0.shape == (0, 64) and s0.shape == (0,)
+
+
+# ------------------------------------------------------------------------------------------------
+# whole layer and the contraction from given codes
+# ------------------------------------------------------------------------------------------------
+def _run_layer_case(bwla, cfg, shape, M, bits, with_mu=False, direct_words=False, path=None):
+    lay = gen.make_layer(cfg, shape, bits, direct_words=direct_words, with_mu=with_mu)
+    xb = gen.make_activations(cfg, shape, M)
+    dl = H.DeviceLayer(lay, bwla)
+    xd = H.bf16_to_dev(xb)
+    if path is not None:
+        bwla.bwla_force_path(path)
+    try:
+        ws = bwla.new_workspace(M, shape.K, shape.N, shape.r, bits)
+        out = bwla.bwla_w1ax_linear(xd, dl.P1, dl.P2, bits, dl.packed, dl.alpha, dl.U, dl.V, dl.mu, workspace=ws)
+        assert bwla.bwla_check_status(ws) == 0
+        ref = oracle.linear(xb, lay.P1, lay.P2, bits, dl.packed_host, lay.alpha, lay.U, lay.V, lay.mu)
+        rep = H.check_output(H.bf16_to_host(out), ref["y"])
+        # identical codes in -> identical integer accumulators out
+        codes = torch.from_numpy(ref["codes"]).cuda()
+        scales = torch.from_numpy(ref["scales"]).cuda()
+        out2, acc = bwla.bwla_w1a_gemm_codes(codes, scales, bits, dl.packed, dl.alpha, xd, dl.U, dl.V, dl.mu,
+                                             want_acc=True, workspace=ws)
+        assert bwla.bwla_check_status(ws) == 0
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), ref["acc"])
+        rep2 = H.check_output(H.bf16_to_host(out2), ref["y"])
+        assert rep2["max_bf16_steps"] <= 1.0 + 1e-9
+    finally:
+        bwla.bwla_force_path(bwla.BWLA_PATH_AUTO)
+    return rep
+
+
+def test_config0_single_w1a6_linear(bwla):
+    rep = _run_layer_case(bwla, 0, gen.CONFIG_SHAPES[0][0], 16, 6)
+    assert rep["rel_l2"] <= 2e-3
+
+
+@pytest.mark.parametrize("K,N,n1,n2,r,M,bits", [
+    (96, 40, 8, 12, 4, 3, 6),        # ragged everything
+    (32, 1, 4, 8, 0, 1, 8),          # one word, one row, one token, no low-rank branch
+    (256, 130, 16, 16, 8, 17, 4),    # N and M straddle tile edges
+    (1024, 300, 32, 32, 16, 70, 6),
+    (2048, 129, 32, 64, 0, 9, 8),
+])
+def test_small_and_ragged_shapes(bwla, K, N, n1, n2, r, M, bits):
+    _run_layer_case(bwla, 0, gen.small_shape(K, N, n1, n2, r, shape_id=K + N), M, bits)
+
+
+def test_mu_shift_is_applied(bwla):
+    _run_layer_case(bwla, 0, gen.small_shape(512, 96, 16, 32, 8, shape_id=5), 6, 6, with_mu=True)
+
+
+@pytest.mark.parametrize("idx,M", [(0, 16), (1, 1), (3, 16)])
+def test_llama7b_shapes(bwla, idx, M):
+    _run_layer_case(bwla, 1, gen.CONFIG_SHAPES[1][idx], M, 6)
+
+
+@pytest.mark.parametrize("idx,M", [(0, 8), (1, 64), (3, 8), (6, 8)])
+def test_qwen32b_shapes(bwla, idx, M):
+    _run_layer_case(bwla, 2, gen.CONFIG_SHAPES[2][idx], M, 6, direct_words=True)
+
+
+@pytest.mark.parametrize("bits", [4, 6, 8])
+def test_bit_width_sweep_down_proj(bwla, bits):
+    _run_layer_case(bwla, 3, gen.CONFIG_SHAPES[3][0], 1, bits, direct_words=True)
+
+
+def test_empty_batch_and_argument_errors(bwla):
+    shape = gen.small_shape(64, 16, 8, 8, 0)
+    lay = gen.make_layer(0, shape, 6)
+    dl = H.DeviceLayer(lay, bwla)
+    x0 = torch.empty(0, 64, dtype=torch.bfloat16, device="cuda")
+    ws = bwla.new_workspace(1, 64, 16, 0, 6)
+    assert bwla.bwla_w1ax_linear(x0, dl.P1, dl.P2, 6, dl.packed, dl.alpha, workspace=ws).shape == (0, 16)
+    x = H.bf16_to_dev(gen.make_activations(0, shape, 2))
+    with pytest.raises(bwla.BwlaError) as e:
+        bwla.bwla_w1ax_linear(x, dl.P1, dl.P2, 5, dl.packed, dl.alpha, workspace=ws)     # bits not in {4,6,8}
+    assert e.value.status == bwla.BWLA_ERR_INVALID_ARG
+    with pytest.raises(bwla.BwlaError) as e:
+        bwla.bwla_w1ax_linear(x, dl.P1, dl.P2[:4, :4].contiguous(), 6, dl.packed, dl.alpha, workspace=ws)  # K != n1*n2
+    assert e.value.status == bwla.BWLA_ERR_INVALID_ARG
+    with pytest.raises(bwla.BwlaError) as e:
+        bwla.bwla_w1ax_linear(x, dl.P1, dl.P2, 6, dl.packed, dl.alpha, workspace=ws[:256])  # workspace too small
+    assert e.value.status == bwla.BWLA_ERR_WORKSPACE
+    # the context is still healthy
+    out = bwla.bwla_w1ax_linear(x, dl.P1, dl.P2, 6, dl.packed, dl.alpha, workspace=bwla.new_workspace(2, 64, 16, 0, 6))
+    torch.cuda.synchronize()
+    assert out.shape == (2, 16)
