@@ -5,8 +5,9 @@ Tolerances (all stated here, used by every parity test):
   * quantised codes: bit-exact against the fp64 oracle except where the oracle's pre-rounding value lies within
     1e-6 * qmax (1e-6 of the token's full scale, in code units) of a rounding boundary; such mismatches must be
     exactly +-1 and are counted.
-  * per-token scale: within 2 fp32 ulp of amax / qmax.
-  * bf16 output: relative L2 error <= 2e-3; every element within 1 bf16 ulp of the correctly rounded oracle value
+  * per-token scale: within 2e-6 relative of amax / qmax (amax comes out of two fp32 contractions of up to
+    n1 + n2 = 320 terms; sqrt(320) * 2^-24 ~ 1e-6 of the row's scale).
+  * bf16 output: relative L2 error <= 2e-3 (asserted for outputs of >= 1024 elements); every element within 1 bf16 ulp of the correctly rounded oracle value
     or within 1e-2 * rms(y) + 2^-8 * |y| of the fp64 oracle value (a correctly rounded bf16 is already up to
     2^-9 * |y| away, so the absolute bound alone cannot hold for elements several rms large).
 """
@@ -70,9 +71,12 @@ def check_codes(gpu_codes: np.ndarray, gpu_scales: np.ndarray, Y: np.ndarray, bi
     assert not unflagged.any(), (
         f"{int(unflagged.sum())} code mismatches outside the near-tie window; "
         f"worst distance to a boundary {ref['dist'][unflagged].max():.3e} (window {window:.1e})")
-    ulp = np.spacing(ref["scales"].astype(np.float32))
-    assert np.all(np.abs(gpu_scales.astype(np.float64) - ref["scales"].astype(np.float64)) <= 2 * ulp)
-    return {"near_ties": int(flagged.sum()), "mismatches": int(bad.sum()), "elements": int(bad.size)}
+    exact_scale = np.abs(Y).max(axis=1) / float((1 << (bits - 1)) - 1)
+    exact_scale[exact_scale == 0] = 1.0
+    scale_err = np.abs(gpu_scales.astype(np.float64) - exact_scale) / exact_scale
+    assert scale_err.max() <= 2e-6, f"scale off by {scale_err.max():.2e} relative"
+    return {"near_ties": int(flagged.sum()), "mismatches": int(bad.sum()), "elements": int(bad.size),
+            "scale_rel_err": float(scale_err.max())}
 
 
 def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray) -> dict:
@@ -80,7 +84,10 @@ def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray) -> dict:
     err = got - y_ref
     rel_l2 = float(np.linalg.norm(err) / max(np.linalg.norm(y_ref), 1e-300))
     rms = float(np.sqrt(np.mean(y_ref ** 2)))
-    assert rel_l2 <= 2e-3, f"relative L2 error {rel_l2:.3e} > 2e-3"
+    # the L2 figure is a statistic of the output rounding (a single correctly rounded bf16 can be 2^-8 away),
+    # so it is only asserted where there are enough elements for it to mean something
+    if y_ref.size >= 1024:
+        assert rel_l2 <= 2e-3, f"relative L2 error {rel_l2:.3e} > 2e-3"
     bound = 1e-2 * rms + 2.0 ** -8 * np.abs(y_ref)
     assert np.all(np.abs(err) <= bound), f"max |err| {np.abs(err).max():.3e} exceeds 1e-2*rms + 2^-8*|y|"
     # distance to the correctly rounded value, in bf16 steps of the reference
