@@ -23,15 +23,19 @@ static bool valid_rotation_dims(int64_t K, int n1, int n2) {
     return K > 0 && K % 32 == 0 && K <= 25600 && n1 > 0 && n2 > 0 && (int64_t)n1 * n2 == K;
 }
 
+// Which kernel family runs the contraction.  A forced family that cannot take the shape falls back to the simple one.
 static int resolve_path(int64_t M, int64_t K, int64_t N, int r, int bits) {
-    (void)M; (void)K; (void)N; (void)r; (void)bits;
-    if (g_forced_path != BWLA_PATH_AUTO) return g_forced_path;
-    return BWLA_PATH_SIMPLE;
+    (void)r; (void)bits;
+    int path = g_forced_path;
+    if (path == BWLA_PATH_AUTO) path = BWLA_PATH_I8;
+    if (path == BWLA_PATH_BITPLANE) path = BWLA_PATH_SIMPLE;   // not built yet
+    if (path == BWLA_PATH_I8 && !umma_supports(M, K, N)) path = BWLA_PATH_SIMPLE;
+    return path;
 }
 
-static int run_contraction(int path, GemmArgs& g, const int8_t* codes_natural, cudaStream_t stream) {
-    (void)path;
-    g.codes = codes_natural;
+static int run_contraction(int path, GemmArgs& g, const int8_t* codes, int32_t* raw, cudaStream_t stream) {
+    if (path == BWLA_PATH_I8) return launch_gemm_umma(g, codes, g.acc_debug ? g.acc_debug : raw, stream);
+    g.codes = codes;
     return launch_gemm_simple(g, stream);
 }
 
@@ -106,8 +110,8 @@ int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, cons
     int8_t* codes = (int8_t*)(base + ws.codes);
     const int path = resolve_path(M, K, N, r, bits);
 
-    st = launch_rotate_quant(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, 0, scales, qsum, nullptr,
-                             (uint32_t*)(base + ws.status), s);
+    st = launch_rotate_quant(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum,
+                             nullptr, (uint32_t*)(base + ws.status), s);
     if (st != BWLA_OK) return st;
     if (r > 0) {
         st = launch_lowrank_T(x_bf16, M, K, ldx, V_bf16, r, T, s);
@@ -117,7 +121,7 @@ int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, cons
     g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
     g.mu = mu; g.T = r > 0 ? T : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = nullptr;
     g.status = (uint32_t*)(base + ws.status);
-    return run_contraction(path, g, codes, s);
+    return run_contraction(path, g, codes, (int32_t*)(base + ws.acc), s);
 }
 
 int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int64_t K, int bits,
@@ -141,7 +145,8 @@ int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int
     float* T = (float*)(base + ws.T);
     const int path = resolve_path(M, K, N, r, bits);
 
-    st = launch_prepare_codes(codes, M, K, nullptr, qsum, (uint32_t*)(base + ws.status), s);
+    int8_t* inter = (path == BWLA_PATH_I8) ? (int8_t*)(base + ws.codes) : nullptr;
+    st = launch_prepare_codes(codes, M, K, inter, qsum, (uint32_t*)(base + ws.status), s);
     if (st != BWLA_OK) return st;
     if (r > 0) {
         st = launch_lowrank_T(x_bf16, M, K, ldx, V_bf16, r, T, s);
@@ -151,7 +156,7 @@ int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int
     g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
     g.mu = mu; g.T = r > 0 ? T : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = acc_debug;
     g.status = (uint32_t*)(base + ws.status);
-    return run_contraction(path, g, codes, s);
+    return run_contraction(path, g, inter ? inter : codes, (int32_t*)(base + ws.acc), s);
 }
 
 int bwla_check_status(void* workspace, void* stream) {

@@ -56,7 +56,7 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     w.T = off;      off += align_up((size_t)M * (size_t)(r > 0 ? r : 1) * 4, 256);
     w.codes = off;  off += align_up((size_t)M * (size_t)K, 256);
     w.planes = off; off += (M <= kBitplaneMaxTokens) ? align_up((size_t)M * 8 * (size_t)(K / 32) * 4, 256) : 0;
-    w.acc = off;    off += (M <= kSplitKMaxTokens) ? align_up((size_t)M * (size_t)N * 4, 256) : 0;
+    w.acc = off;    off += align_up((size_t)M * (size_t)N * 4, 256);
     (void)bits;
     w.total = off;
     return w;
@@ -102,5 +102,9 @@ struct GemmArgs {
 };
 
 int launch_gemm_simple(const GemmArgs& a, cudaStream_t stream);
+
+// tcgen05 path.  codes_interleaved: int8 [M][K] in the interleaved order; raw: int32 [M][N] scratch.
+bool umma_supports(int64_t M, int64_t K, int64_t N);
+int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, int32_t* raw, cudaStream_t stream);
 
 }  // namespace bwla
