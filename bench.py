@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the BWLA W1A6 linear hot path on the Qwen3-32B-shaped linear stack.
+
+A step is one pass over all 7 linears of all layers (rotate + quantise + binary contraction + low-rank + bf16
+epilogue for every linear), back to back on one stream, replayed from a CUDA graph.  Inputs are seeded and
+synthetic (no checkpoints or datasets exist here); all layers' weights stay resident in HBM (about 5 GB, far
+larger than L2, so every step streams them from DRAM again).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is the decode figure (algorithmic HBM bytes of the whole stack per second
+at --decode-m tokens); `prefill` holds the INT8 TOPS figure at --prefill-m tokens; `roofline` is for the dominant
+kernel (the tcgen05 contraction) timed with CUDA events around each of its launches.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_00422_b200 import inputs as gen  # noqa: E402
+
+METRIC = "W1A6 linear: decode HBM GB/s & prefill INT8 TOPS vs B200 roofline, Qwen3-32B"
+BITS = 6
+
+
+# ----------------------------------------------------------------------------------------------
+# workload arithmetic
+# ----------------------------------------------------------------------------------------------
+def call_bytes(sh: gen.LinearShape, M: int) -> int:
+    """Algorithmic HBM bytes of one whole linear call: sign bits, low-rank factors, alpha, Kronecker factors,
+    activations in, outputs out."""
+    return (sh.N * sh.K // 8 + 2 * sh.r * (sh.N + sh.K) + 4 * sh.N + 4 * (sh.n1 ** 2 + sh.n2 ** 2)
+            + 2 * M * sh.K + 2 * M * sh.N)
+
+
+def contraction_kernel_bytes(sh: gen.LinearShape, M: int) -> int:
+    """Algorithmic bytes of one launch of the contraction kernel: sign bits + int8 codes + int32 accumulators."""
+    return sh.N * sh.K // 8 + M * sh.K + 4 * M * sh.N
+
+
+def call_ops(sh: gen.LinearShape, M: int) -> int:
+    return 2 * M * sh.K * sh.N
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid = uuid
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, mx = [], set(), None
+        try:
+            for ln in open(self.path):
+                p = [v.strip() for v in ln.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0]))
+                    mx = float(p[1])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample
+# ----------------------------------------------------------------------------------------------
+def host_layer(layer: int):
+    """Host tensors of one layer's 7 linears (numpy recipe of the parity tests)."""
+    out = []
+    for sh in gen.CONFIG_SHAPES[4]:
+        lay = gen.make_layer(4, sh, BITS, layer=layer, direct_words=True)
+        out.append((sh, lay))
+    return out
+
+
+def oracle_pass(layer_tensors, xs):
+    import oracle
+    for sh, lay in layer_tensors:
+        oracle.linear(xs[sh.K], lay.P1, lay.P2, BITS, lay.packed, lay.alpha, lay.U, lay.V)
+
+
+def run_reference(args):
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    M = args.decode_m
+    lt = host_layer(0)
+    xs = {}
+    for sh, _ in lt:
+        if sh.K not in xs:
+            xs[sh.K] = gen.make_activations(4, sh, M)
+    nbytes = sum(call_bytes(sh, M) for sh, _ in lt)
+    for _ in range(max(1, min(args.warmup, 1))):
+        oracle_pass(lt, xs)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(lt, xs)
+    dt = time.perf_counter() - t0
+    val = nbytes * args.steps / dt / 1e9
+    sample = f"one layer (7 linears) of the stack at M={M} per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64/int64", "data": "synthetic",
+        "config": {"workload": f"qwen3-32b linear stack, decode M={M}, bounded sample: {sample}", "bits": BITS},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------
+class Linear:
+    __slots__ = ("shape", "P1", "P2", "packed", "alpha", "U", "V")
+
+
+def build_stack(layers: int, device, torch):
+    """Per-layer seeded weights generated on the device (same distributions as the host recipe of the tests)."""
+    stack = []
+    for layer in range(layers):
+        row = []
+        for sh in gen.CONFIG_SHAPES[4]:
+            g = torch.Generator(device=device)
+            g.manual_seed(gen.ROOT_SEED * 1000003 + layer * 101 + sh.shape_id)
+            lin = Linear()
+            lin.shape = sh
+            lin.P1 = torch.from_numpy(gen.orthogonal_f32(sh.n1, gen._rng(4, layer, sh.shape_id, gen.T_P1))).to(device)
+            lin.P2 = torch.from_numpy(gen.orthogonal_f32(sh.n2, gen._rng(4, layer, sh.shape_id, gen.T_P2))).to(device)
+            lin.packed = torch.randint(-2 ** 31, 2 ** 31, (sh.N, sh.K // 32), dtype=torch.int64, device=device,
+                                       generator=g).to(torch.int32)
+            lin.alpha = torch.exp(-4.0 + 0.3 * torch.randn(sh.N, device=device, generator=g))
+            lin.U = (0.01 * torch.randn(sh.N, sh.r, device=device, generator=g)).to(torch.bfloat16)
+            lin.V = (0.01 * torch.randn(sh.r, sh.K, device=device, generator=g)).to(torch.bfloat16)
+            row.append(lin)
+        stack.append(row)
+    return stack
+
+
+def student_t_activations(M: int, K: int, device, torch, seed: int):
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    z = torch.randn(M, K, device=device, generator=g)
+    chi = (torch.randn(3, M, K, device=device, generator=g) ** 2).sum(0)
+    x = z / torch.sqrt(chi / 3.0)
+    ch = torch.randperm(K, device=device, generator=g)[:8]
+    x[:, ch] *= 50.0
+    return x.to(torch.bfloat16)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2605_00422_b200 import bwla
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    peaks = measured_peaks()
+    shapes = gen.CONFIG_SHAPES[4]
+    stack = build_stack(args.layers, device, torch)
+    Ks = sorted({sh.K for sh in shapes})
+    Ns = sorted({sh.N for sh in shapes})
+
+    def make_io(M):
+        xs = {K: student_t_activations(M, K, device, torch, 7000 + K + M) for K in Ks}
+        outs = {N: torch.empty(M, N, dtype=torch.bfloat16, device=device) for N in Ns}
+        ws_bytes = max(bwla.bwla_workspace_bytes(M, sh.K, sh.N, sh.r, BITS) for sh in shapes)
+        ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
+        return xs, outs, ws
+
+    def step(xs, outs, ws, layers=None):
+        n = 0
+        for row in (stack if layers is None else stack[:layers]):
+            for lin in row:
+                bwla.bwla_w1ax_linear(xs[lin.shape.K], lin.P1, lin.P2, BITS, lin.packed, lin.alpha, lin.U, lin.V,
+                                      out=outs[lin.shape.N], workspace=ws)
+                n += bwla.bwla_last_launch_count()
+        return n
+
+    def capture(xs, outs, ws, layers=None):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step(xs, outs, ws, 1)        # sets per-kernel attributes before capture
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            launches = step(xs, outs, ws, layers)
+        return g, launches
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    def kernel_profile(xs, outs, ws, passes=1, layers=None):
+        bwla.bwla_profile_enable(True)
+        for _ in range(passes):
+            step(xs, outs, ws, layers)
+        prof = bwla.bwla_profile_collect()
+        bwla.bwla_profile_enable(False)
+        return {k: (ms / passes, n // passes) for k, (ms, n) in prof.items() if n}
+
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid).replace("GPU-", "")
+    sampler = ClockSampler(uuid)
+
+    # ------------------------------ decode ------------------------------
+    M = args.decode_m
+    xs, outs, ws = make_io(M)
+    graph, launches_per_step = capture(xs, outs, ws)
+    sampler.start()
+    ms = timed(graph.replay, args.steps, max(args.warmup, 3))
+    clocks = sampler.stop()
+    status = bwla.bwla_check_status(ws)
+    step_bytes = args.layers * sum(call_bytes(sh, M) for sh in shapes)
+    value = world * step_bytes * args.steps / (ms * 1e-3) / 1e9
+
+    # end to end: activations arrive from pinned host memory and the last layer's outputs go back, every step
+    h_xs = {K: xs[K].cpu().pin_memory() for K in Ks}
+    h_outs = {N: torch.empty(M, N, dtype=torch.bfloat16).pin_memory() for N in Ns}
+
+    def e2e_step():
+        for K in Ks:
+            xs[K].copy_(h_xs[K], non_blocking=True)
+        graph.replay()
+        for N in Ns:
+            h_outs[N].copy_(outs[N], non_blocking=True)
+
+    e2e_ms = timed(e2e_step, args.steps, 3)
+    h2d = sum(h_xs[K].numel() * 2 for K in Ks)
+    d2h = sum(h_outs[N].numel() * 2 for N in Ns)
+    e2e_value = world * step_bytes * args.steps / (e2e_ms * 1e-3) / 1e9
+
+    prof = kernel_profile(xs, outs, ws)
+    k_ms, k_n = prof.get("contraction", (0.0, 0))
+    k_bytes = args.layers * sum(contraction_kernel_bytes(sh, M) for sh in shapes)
+    achieved = k_bytes / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
+    roofline = {"bound": "hbm", "kernel": "umma_w1a_kernel (tcgen05 kind::i8 contraction), decode stack",
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": None,
+                "launches_per_step": k_n, "avg_launch_us": (k_ms / k_n * 1e3) if k_n else None,
+                "algorithmic_bytes_per_step": k_bytes}
+    del graph
+
+    # ------------------------------ prefill ------------------------------
+    prefill = None
+    if args.prefill_m > 0:
+        Mp = args.prefill_m
+        xs_p, outs_p, ws_p = make_io(Mp)
+        Lp = min(args.prefill_layers or args.layers, args.layers)
+        graph_p, _ = capture(xs_p, outs_p, ws_p, Lp)
+        steps_p = max(2, args.steps // 5)
+        sampler_p = ClockSampler(uuid)
+        sampler_p.start()
+        ms_p = timed(graph_p.replay, steps_p, 3)
+        clocks_p = sampler_p.stop()
+        ops = Lp * sum(call_ops(sh, Mp) for sh in shapes)
+        tops = world * ops * steps_p / (ms_p * 1e-3) / 1e12
+        prof_p = kernel_profile(xs_p, outs_p, ws_p, layers=Lp)
+        kp_ms, kp_n = prof_p.get("contraction", (0.0, 0))
+        k_tops = ops / (kp_ms * 1e-3) / 1e12 if kp_ms > 0 else None
+        i8_peak = 2.0 * peaks["bf16_tflops_sustained"]   # int8 dense = 2 x bf16 (nominal ratio) of the measured bf16 rate
+        prefill = {"metric": "prefill INT8 TOPS (2*M*K*N of the contraction / whole-step time)", "value": tops,
+                   "unit": "TOPS", "M": Mp, "layers": Lp, "steps": steps_p, "ms_per_step": ms_p / steps_p, "clocks": clocks_p,
+                   "roofline": {"bound": "tensor", "kernel": "umma_w1a_kernel, prefill stack", "achieved": k_tops,
+                                "peak": i8_peak, "peak_source": peaks["source"] + " bf16 sustained x 2 (int8:bf16 nominal ratio)",
+                                "unit": "TOP/s", "frac": (k_tops / i8_peak) if k_tops else None, "traffic": None,
+                                "launches_per_step": kp_n},
+                   "kernel_ms_per_step": {k: round(v[0], 4) for k, v in prof_p.items()},
+                   "status": bwla.bwla_check_status(ws_p)}
+        del graph_p
+
+    # ------------------------------ CPU baseline (rank 0, N = 1) ------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        lt = host_layer(0)
+        hx = {}
+        for sh, _ in lt:
+            if sh.K not in hx:
+                hx[sh.K] = gen.make_activations(4, sh, M)
+        t0 = time.perf_counter()
+        reps = 0
+        while reps < 1 or (time.perf_counter() - t0 < 10.0 and reps < 50):
+            oracle_pass(lt, hx)
+            reps += 1
+        dt = time.perf_counter() - t0
+        cpu = {"value": reps * sum(call_bytes(sh, M) for sh, _ in lt) / dt / 1e9, "unit": "GB/s",
+               "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"{reps} pass(es) over one layer (7 linears) at M={M}; {dt:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 x int1 -> int32 (fp32 rotation, bf16 out)", "data": "synthetic",
+            "config": {"workload": f"qwen3-32b linear stack (config 4): {args.layers} layers x 7 W1A6 linears, decode M={M}, "
+                                   f"rank 64, all weights resident ({step_bytes / 1e9:.2f} GB algorithmic bytes per step)",
+                       "bits": BITS, "l2": "inputs larger than L2 (weights of all layers are streamed every step)",
+                       "launch": "one CUDA graph per step, one stream", "parallelism": "replicas only"},
+            "clocks": clocks, "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                                      "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
+            "kernel_ms_per_step": {k: round(v[0], 4) for k, v in prof.items()},
+            "cpu_baseline": cpu, "prefill": prefill, "device_status": status,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=gen.QWEN3_32B_LAYERS)
+    ap.add_argument("--decode-m", type=int, default=16)
+    ap.add_argument("--prefill-m", type=int, default=2048)
+    ap.add_argument("--prefill-layers", type=int, default=0, help="layers in the prefill step (0 = all)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

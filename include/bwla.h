@@ -131,6 +131,16 @@ int bwla_chosen_path(int64_t M, int64_t K, int64_t N, int r, int bits);
  * bwla_pack_signs call on this thread launched. */
 int bwla_last_launch_count(void);
 
+/*
+ * Per-kernel timing for benchmarks.  While enabled (per calling thread), every kernel the library launches is
+ * bracketed by CUDA events recorded on the launching stream.  bwla_profile_collect waits for them, adds the
+ * elapsed milliseconds and launch counts per kernel kind into two caller arrays of 8 entries
+ * (0 rotate+quantise, 1 low-rank V x, 2 contraction, 3 accumulator epilogue, 4 code preparation, 5 pack_signs)
+ * and forgets the events.  Host arrays.  Do not enable during stream capture.
+ */
+int bwla_profile_enable(int on);
+int bwla_profile_collect(float* ms_by_kind, int* launches_by_kind);
+
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int bwla_last_cuda_error(void);
 

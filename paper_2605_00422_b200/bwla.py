@@ -30,7 +30,7 @@ BWLA_PATH_I8 = 3
 EXPORTS = [
     "bwla_pack_signs", "bwla_rotate_quant_act", "bwla_workspace_bytes", "bwla_w1ax_linear", "bwla_w1a_gemm_codes",
     "bwla_check_status", "bwla_force_path", "bwla_chosen_path", "bwla_last_launch_count", "bwla_last_cuda_error",
-    "bwla_status_string",
+    "bwla_status_string", "bwla_profile_enable", "bwla_profile_collect",
 ]
 
 
@@ -57,11 +57,13 @@ def _load() -> C.CDLL:
     lib.bwla_check_status.argtypes = [vp, vp]
     lib.bwla_force_path.argtypes = [ci]
     lib.bwla_chosen_path.argtypes = [i64, i64, i64, ci, ci]
+    lib.bwla_profile_enable.argtypes = [ci]
+    lib.bwla_profile_collect.argtypes = [vp, vp]
     lib.bwla_status_string.argtypes = [ci]
     lib.bwla_status_string.restype = C.c_char_p
     for name in ("bwla_pack_signs", "bwla_rotate_quant_act", "bwla_w1ax_linear", "bwla_w1a_gemm_codes",
                  "bwla_check_status", "bwla_force_path", "bwla_chosen_path", "bwla_last_launch_count",
-                 "bwla_last_cuda_error"):
+                 "bwla_last_cuda_error", "bwla_profile_enable", "bwla_profile_collect"):
         getattr(lib, name).restype = ci
     return lib
 
@@ -224,3 +226,18 @@ def bwla_w1a_gemm_codes(codes: torch.Tensor, scales: torch.Tensor, bits: int, pa
 def bwla_check_status(workspace: torch.Tensor) -> int:
     """Synchronises the current stream and returns the status a bounded device-side wait may have left."""
     return int(_lib.bwla_check_status(_ptr(workspace), _stream()))
+
+
+PROFILE_KINDS = ("rotate_quant", "lowrank_vx", "contraction", "acc_epilogue", "prepare_codes", "pack_signs")
+
+
+def bwla_profile_enable(on: bool) -> None:
+    _check(_lib.bwla_profile_enable(1 if on else 0), "bwla_profile_enable")
+
+
+def bwla_profile_collect() -> dict:
+    """Waits for the recorded events; returns {kind: (total_ms, launches)}."""
+    ms = (C.c_float * 8)()
+    n = (C.c_int * 8)()
+    _check(_lib.bwla_profile_collect(ms, n), "bwla_profile_collect")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(PROFILE_KINDS)}

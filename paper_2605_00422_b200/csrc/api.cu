@@ -1,4 +1,6 @@
 // extern "C" boundary: argument validation, workspace carving and per-shape dispatch.  No compute happens here.
+#include <vector>
+
 #include "bwla_common.cuh"
 
 namespace bwla {
@@ -6,6 +8,24 @@ namespace bwla {
 thread_local int g_last_cuda_error = 0;
 thread_local int g_launch_count = 0;
 static int g_forced_path = BWLA_PATH_AUTO;
+
+// ---- optional kernel timing -------------------------------------------------------------------
+struct ProfPair { cudaEvent_t a, b; int kind; };
+static thread_local bool g_prof_on = false;
+static thread_local std::vector<ProfPair>* g_prof = nullptr;
+
+void prof_begin(int kind, cudaStream_t stream) {
+    if (!g_prof_on) return;
+    if (!g_prof) g_prof = new std::vector<ProfPair>();
+    ProfPair p{nullptr, nullptr, kind};
+    if (cudaEventCreate(&p.a) != cudaSuccess || cudaEventCreate(&p.b) != cudaSuccess) return;
+    cudaEventRecord(p.a, stream);
+    g_prof->push_back(p);
+}
+void prof_end(int kind, cudaStream_t stream) {
+    if (!g_prof_on || !g_prof || g_prof->empty() || g_prof->back().kind != kind) return;
+    cudaEventRecord(g_prof->back().b, stream);
+}
 
 static bool valid_bits(int bits) { return bits == 4 || bits == 6 || bits == 8; }
 
@@ -182,6 +202,29 @@ int bwla_force_path(int path) {
 int bwla_chosen_path(int64_t M, int64_t K, int64_t N, int r, int bits) { return resolve_path(M, K, N, r, bits); }
 
 int bwla_last_launch_count(void) { return g_launch_count; }
+
+int bwla_profile_enable(int on) {
+    g_prof_on = on != 0;
+    return BWLA_OK;
+}
+
+int bwla_profile_collect(float* ms_by_kind, int* launches_by_kind) {
+    if (!ms_by_kind || !launches_by_kind) return BWLA_ERR_INVALID_ARG;
+    for (int i = 0; i < kProfKinds; ++i) { ms_by_kind[i] = 0.f; launches_by_kind[i] = 0; }
+    if (!g_prof) return BWLA_OK;
+    int st = BWLA_OK;
+    for (auto& p : *g_prof) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(p.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, p.a, p.b);
+        if (e == cudaSuccess && p.kind >= 0 && p.kind < kProfKinds) { ms_by_kind[p.kind] += ms; launches_by_kind[p.kind] += 1; }
+        else if (e != cudaSuccess) st = cuda_fail(e);
+        cudaEventDestroy(p.a);
+        cudaEventDestroy(p.b);
+    }
+    g_prof->clear();
+    return st;
+}
 
 int bwla_last_cuda_error(void) { return g_last_cuda_error; }
 

@@ -37,6 +37,20 @@ inline int after_launch() {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // ---------------------------------------------------------------------------------------------
+// optional per-kernel timing (bwla_profile_enable / bwla_profile_collect): CUDA events recorded on the launching
+// stream right around each kernel launch, summed per kernel kind.  Off by default; not usable under stream capture.
+// ---------------------------------------------------------------------------------------------
+enum ProfKind { kProfRotateQuant = 0, kProfLowrankT = 1, kProfContraction = 2, kProfFinalize = 3, kProfPrepare = 4,
+                kProfPack = 5, kProfKinds = 8 };
+void prof_begin(int kind, cudaStream_t stream);
+void prof_end(int kind, cudaStream_t stream);
+struct ProfScope {
+    int kind; cudaStream_t stream;
+    ProfScope(int k, cudaStream_t s) : kind(k), stream(s) { prof_begin(kind, stream); }
+    ~ProfScope() { prof_end(kind, stream); }
+};
+
+// ---------------------------------------------------------------------------------------------
 // workspace layout (byte offsets into the caller's scratch buffer; every section 256-byte aligned)
 // ---------------------------------------------------------------------------------------------
 constexpr int kStatusBytes = 256;        // word 0: status; words 1..: where a bounded wait gave up

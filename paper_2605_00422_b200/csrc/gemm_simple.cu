@@ -51,6 +51,7 @@ int launch_lowrank_T(const void* x, int64_t M, int64_t K, int64_t ldx, const voi
                      cudaStream_t stream) {
     if (M == 0 || r == 0) return BWLA_OK;
     dim3 grid((unsigned)r, (unsigned)((M + kTokTile - 1) / kTokTile));
+    ProfScope prof(kProfLowrankT, stream);
     lowrank_T_kernel<<<grid, 256, 0, stream>>>((const __nv_bfloat16*)x, M, (int)K, ldx, (const __nv_bfloat16*)V, r, T);
     return after_launch();
 }
@@ -108,6 +109,7 @@ __global__ void __launch_bounds__(128) gemm_simple_kernel(GemmArgs a) {
 int launch_gemm_simple(const GemmArgs& a, cudaStream_t stream) {
     if (a.M == 0 || a.N == 0) return BWLA_OK;
     dim3 grid((unsigned)((a.N + 3) / 4), (unsigned)((a.M + kTokTile - 1) / kTokTile));
+    ProfScope prof(kProfContraction, stream);
     gemm_simple_kernel<<<grid, 128, 0, stream>>>(a);
     return after_launch();
 }

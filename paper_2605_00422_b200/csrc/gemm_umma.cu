@@ -307,6 +307,7 @@ static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const Umm
         BWLA_CUDA_TRY(cudaFuncSetAttribute(umma_w1a_kernel<N_TOK, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total));
         configured = dev;
     }
+    ProfScope prof(kProfContraction, s);
     umma_w1a_kernel<N_TOK, WS><<<grid, kThreads, L::total, s>>>(wm, bm, p);
     return after_launch();
 }
@@ -350,6 +351,7 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, int32_t
     }
     if (st != BWLA_OK) return st;
     const int64_t total = (int64_t)M * N;
+    ProfScope prof(kProfFinalize, stream);
     finalize_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(a, raw);
     return after_launch();
 }

@@ -37,6 +37,7 @@ int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ld
     const int warps_per_block = 8;
     int64_t blocks = (total + warps_per_block - 1) / warps_per_block;
     if (blocks > 148 * 16) blocks = 148 * 16;
+    ProfScope prof(kProfPack, stream);
     if (dtype == BWLA_DTYPE_F32)
         pack_signs_kernel<float><<<(unsigned)blocks, 256, 0, stream>>>((const float*)w, N, words, ldw, packed);
     else

@@ -241,6 +241,7 @@ int launch_rotate_quant(const void* x, int64_t M, int64_t K, int64_t ldx, const 
     }
     const int threads = (K >= 8192) ? 512 : 256;
     const unsigned grid = (unsigned)(M < 148 * 64 ? M : 148 * 64);
+    ProfScope prof(kProfRotateQuant, stream);
     rotate_quant_kernel<<<grid, threads, smem, stream>>>((const __nv_bfloat16*)x, M, (int)K, ldx, P1, n1, P2, n2, bits,
                                                          codes, codes_layout, scales, qsum, planes, status);
     return after_launch();
@@ -294,6 +295,7 @@ __global__ void __launch_bounds__(256) prepare_codes_kernel(const int8_t* __rest
 int launch_prepare_codes(const int8_t* codes, int64_t M, int64_t K, int8_t* codes_interleaved, int32_t* qsum,
                          uint32_t* status, cudaStream_t stream) {
     if (M == 0) return BWLA_OK;
+    ProfScope prof(kProfPrepare, stream);
     prepare_codes_kernel<<<(unsigned)M, 256, 0, stream>>>(codes, M, (int)K, codes_interleaved, qsum, status);
     return after_launch();
 }
