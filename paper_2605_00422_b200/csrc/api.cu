@@ -12,13 +12,20 @@ static int g_forced_path = BWLA_PATH_AUTO;
 // ---- optional kernel timing -------------------------------------------------------------------
 struct ProfPair { cudaEvent_t a, b; int kind; };
 static thread_local bool g_prof_on = false;
-static thread_local std::vector<ProfPair>* g_prof = nullptr;
+static thread_local std::vector<ProfPair>* g_prof = nullptr;       // pairs recorded since the last collect
+static thread_local std::vector<ProfPair>* g_prof_pool = nullptr;  // idle pairs, reused so that recording stays cheap
 
 void prof_begin(int kind, cudaStream_t stream) {
     if (!g_prof_on) return;
-    if (!g_prof) g_prof = new std::vector<ProfPair>();
+    if (!g_prof) { g_prof = new std::vector<ProfPair>(); g_prof_pool = new std::vector<ProfPair>(); }
     ProfPair p{nullptr, nullptr, kind};
-    if (cudaEventCreate(&p.a) != cudaSuccess || cudaEventCreate(&p.b) != cudaSuccess) return;
+    if (!g_prof_pool->empty()) {
+        p = g_prof_pool->back();
+        p.kind = kind;
+        g_prof_pool->pop_back();
+    } else if (cudaEventCreate(&p.a) != cudaSuccess || cudaEventCreate(&p.b) != cudaSuccess) {
+        return;
+    }
     cudaEventRecord(p.a, stream);
     g_prof->push_back(p);
 }
@@ -219,8 +226,7 @@ int bwla_profile_collect(float* ms_by_kind, int* launches_by_kind) {
         if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, p.a, p.b);
         if (e == cudaSuccess && p.kind >= 0 && p.kind < kProfKinds) { ms_by_kind[p.kind] += ms; launches_by_kind[p.kind] += 1; }
         else if (e != cudaSuccess) st = cuda_fail(e);
-        cudaEventDestroy(p.a);
-        cudaEventDestroy(p.b);
+        g_prof_pool->push_back(p);
     }
     g_prof->clear();
     return st;

@@ -31,9 +31,7 @@ using namespace ptx;
 constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
 constexpr int kBlockK = 128;             // K per code stage / per tensor-memory A stage
-constexpr int kAbStages = 4;
-constexpr int kTmemCols = 256;
-constexpr int kTmemAcol = 128;           // A stages live in columns [128, 256); D in [0, N_TOK)
+constexpr int kTmemCols = 256;           // per CTA, so that two CTAs share an SM's 512 columns
 constexpr int kThreads = 224;            // warp 0: weight TMA, 1: MMA, 2: code TMA, 3..6: expand + epilogue
 constexpr uint32_t kWaitLimit = 1u << 20;   // polls per wait before giving up (tens of milliseconds)
 
@@ -45,12 +43,22 @@ struct UmmaParams {
     uint32_t* status;
 };
 
-template <int N_TOK, int WS>
-struct UmmaSmem {
+// Shared-memory and tensor-memory budget of one CTA.
+//   weights: WS stages of 128 rows x 128 bytes (one K-unit of 1024 weights per row);
+//   codes:   BS stages of 16 KB = SUBS k-blocks of (N_TOK rows x 128 bytes), so that small token tiles still move
+//            16 KB per barrier round trip;
+//   tensor memory: D in columns [0, DCOLS), then AS stages of 32 columns (one k-block of expanded weights each).
+template <int N_TOK, int WS, int BS>
+struct UmmaCfg {
     static constexpr int w_bytes = kRowsPerCta * 128;
-    static constexpr int b_bytes = N_TOK * 128;
-    static constexpr int bars_off = WS * w_bytes + kAbStages * b_bytes;
-    static constexpr int total = bars_off + 256 + 1024;   // + barriers + slack for 1024-byte alignment
+    static constexpr int sub_bytes = N_TOK * 128;
+    static constexpr int SUBS = (128 / N_TOK) < 1 ? 1 : ((128 / N_TOK) > 8 ? 8 : (128 / N_TOK));
+    static constexpr int b_bytes = SUBS * sub_bytes;
+    static constexpr int DCOLS = N_TOK <= 64 ? 64 : 128;
+    static constexpr int AS = (kTmemCols - DCOLS) / 32;
+    static constexpr int bars_off = WS * w_bytes + BS * b_bytes;
+    static constexpr int n_bars = 2 * WS + 2 * BS + 2 * AS + 1;
+    static constexpr int total = bars_off + n_bars * 8 + 64 + 1024;   // + slack for 1024-byte alignment
 };
 
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
@@ -71,21 +79,24 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
     return false;
 }
 
-template <int N_TOK, int WS>
+template <int N_TOK, int WS, int BS>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map, UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
-    using L = UmmaSmem<N_TOK, WS>;
+    using L = UmmaCfg<N_TOK, WS, BS>;
+    constexpr int AS = L::AS;
+    constexpr int SUBS = L::SUBS;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* wbuf = smem;
     uint8_t* bbuf = smem + WS * L::w_bytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::bars_off);
     uint64_t* w_full = bars;                 // [WS]
     uint64_t* w_empty = bars + WS;           // [WS]
-    uint64_t* b_full = bars + 2 * WS;        // [kAbStages]
-    uint64_t* a_full = b_full + kAbStages;   // [kAbStages]
-    uint64_t* ab_empty = a_full + kAbStages; // [kAbStages]
-    uint64_t* d_full = ab_empty + kAbStages; // [1]
+    uint64_t* b_full = bars + 2 * WS;        // [BS]
+    uint64_t* b_empty = b_full + BS;         // [BS]
+    uint64_t* a_full = b_empty + BS;         // [AS]
+    uint64_t* a_empty = a_full + AS;         // [AS]
+    uint64_t* d_full = a_empty + AS;         // [1]
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
@@ -100,7 +111,8 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         // a CTA of this launch that already gave up makes the rest of the grid skip its work
         abort_flag_s = (p.status && *reinterpret_cast<volatile uint32_t*>(p.status) != 0) ? 1 : 0;
         for (int i = 0; i < WS; ++i) { mbar_init(&w_full[i], 1); mbar_init(&w_empty[i], 4); }
-        for (int i = 0; i < kAbStages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&a_full[i], 4); mbar_init(&ab_empty[i], 1); }
+        for (int i = 0; i < BS; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < AS; ++i) { mbar_init(&a_full[i], 4); mbar_init(&a_empty[i], 1); }
         mbar_init(d_full, 1);
         fence_barrier_init();
         fence_proxy_async();
@@ -133,14 +145,17 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         // ---------------- activation codes: L2/HBM -> shared memory ----------------
         if (elect_one()) {
             tma_prefetch_desc(&b_map);
-            int ab = 0; uint32_t abph = 0;
-            for (int u = unit_begin; u < unit_end && !*abort_flag; ++u) {
+            int bs = 0; uint32_t bph = 0;
+            bool ok = true;
+            for (int u = unit_begin; u < unit_end && ok && !*abort_flag; ++u) {
                 const int ns = sub_count(u);
-                for (int s = 0; s < ns; ++s) {
-                    if (!wait_or_abort(&ab_empty[ab], abph ^ 1, abort_flag)) { give_up(p.status, abort_flag, 0x20); break; }
-                    mbar_expect_tx(&b_full[ab], L::b_bytes);
-                    tma_load_2d(bbuf + ab * L::b_bytes, &b_map, (u * 8 + s) * kBlockK, t0, &b_full[ab]);
-                    if (++ab == kAbStages) { ab = 0; abph ^= 1; }
+                for (int s0 = 0; s0 < ns; s0 += SUBS) {
+                    const int cnt = min(SUBS, ns - s0);
+                    if (!wait_or_abort(&b_empty[bs], bph ^ 1, abort_flag)) { give_up(p.status, abort_flag, 0x20); ok = false; break; }
+                    mbar_expect_tx(&b_full[bs], cnt * L::sub_bytes);
+                    for (int s = 0; s < cnt; ++s)
+                        tma_load_2d(bbuf + bs * L::b_bytes + s * L::sub_bytes, &b_map, (u * 8 + s0 + s) * kBlockK, t0, &b_full[bs]);
+                    if (++bs == BS) { bs = 0; bph ^= 1; }
                 }
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);
@@ -150,23 +165,28 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         if (elect_one()) {
             // instruction descriptor: D = s32, A = s8 (tensor memory, K-major), B = s8 (shared, K-major), M = 128
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
-            int ab = 0; uint32_t abph = 0; uint32_t first = 1;
+            int as = 0; uint32_t aph = 0; int bs = 0; uint32_t bph = 0; uint32_t first = 1;
             bool ok = true;
             for (int u = unit_begin; u < unit_end && ok; ++u) {
                 const int ns = sub_count(u);
                 for (int s = 0; s < ns; ++s) {
-                    if (!wait_or_abort(&b_full[ab], abph, abort_flag)) { give_up(p.status, abort_flag, 0x30); ok = false; break; }
-                    if (!wait_or_abort(&a_full[ab], abph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
+                    const int sb = s % SUBS;
+                    if (sb == 0 && !wait_or_abort(&b_full[bs], bph, abort_flag)) { give_up(p.status, abort_flag, 0x30); ok = false; break; }
+                    if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
                     tc_fence_after();
-                    const uint32_t b_addr = smem_u32(bbuf + ab * L::b_bytes);
-                    const uint32_t a_addr = tmem_base + kTmemAcol + 32 * ab;
+                    const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
+                    const uint32_t a_addr = tmem_base + L::DCOLS + 32 * as;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         mma_i8_ts(tmem_base, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, first ? 0u : 1u);
                         first = 0;
                     }
-                    tc_commit(&ab_empty[ab]);
-                    if (++ab == kAbStages) { ab = 0; abph ^= 1; }
+                    tc_commit(&a_empty[as]);
+                    if (++as == AS) { as = 0; aph ^= 1; }
+                    if (sb == SUBS - 1 || s == ns - 1) {
+                        tc_commit(&b_empty[bs]);
+                        if (++bs == BS) { bs = 0; bph ^= 1; }
+                    }
                 }
             }
             tc_commit(d_full);
@@ -176,7 +196,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         const int q = warp & 3;                       // tensor-memory lane quarter this warp may touch
         const int row = q * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        int ws = 0; uint32_t wph = 0; int ab = 0; uint32_t abph = 0;
+        int ws = 0; uint32_t wph = 0; int as = 0; uint32_t aph = 0;
         bool ok = true;
         for (int u = unit_begin; u < unit_end && ok; ++u) {
             if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&w_full[ws], wph, abort_flag))) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
@@ -190,14 +210,14 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[8 * i + j] = (w[i] << (7 - j)) & 0x80808080u;
-                if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&ab_empty[ab], abph ^ 1, abort_flag))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
+                if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&a_empty[as], aph ^ 1, abort_flag))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
                 tc_fence_after();
-                tmem_st_32x32(tmem_base + lane_addr + kTmemAcol + 32 * ab, v);
+                tmem_st_32x32(tmem_base + lane_addr + L::DCOLS + 32 * as, v);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[ab]);
-                if (++ab == kAbStages) { ab = 0; abph ^= 1; }
+                if (lane == 0) mbar_arrive(&a_full[as]);
+                if (++as == AS) { as = 0; aph ^= 1; }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&w_empty[ws]);
@@ -297,18 +317,20 @@ static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* bas
     return BWLA_OK;
 }
 
-template <int N_TOK, int WS>
+template <int N_TOK, int WS, int BS>
 static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const UmmaParams& p, dim3 grid, cudaStream_t s) {
-    using L = UmmaSmem<N_TOK, WS>;
+    using L = UmmaCfg<N_TOK, WS, BS>;
+    constexpr int AS = L::AS;
+    constexpr int SUBS = L::SUBS;
     static thread_local int configured = -1;
     int dev = 0;
     BWLA_CUDA_TRY(cudaGetDevice(&dev));
     if (configured != dev) {
-        BWLA_CUDA_TRY(cudaFuncSetAttribute(umma_w1a_kernel<N_TOK, WS>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total));
+        BWLA_CUDA_TRY(cudaFuncSetAttribute(umma_w1a_kernel<N_TOK, WS, BS>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total));
         configured = dev;
     }
     ProfScope prof(kProfContraction, s);
-    umma_w1a_kernel<N_TOK, WS><<<grid, kThreads, L::total, s>>>(wm, bm, p);
+    umma_w1a_kernel<N_TOK, WS, BS><<<grid, kThreads, L::total, s>>>(wm, bm, p);
     return after_launch();
 }
 
@@ -344,10 +366,10 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, int32_t
     if (split > 1) BWLA_CUDA_TRY(cudaMemsetAsync(raw, 0, (size_t)M * N * 4, stream));
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     switch (n_tok) {
-        case 16: st = launch_umma_t<16, 5>(wm, bm, p, grid, stream); break;
-        case 32: st = launch_umma_t<32, 5>(wm, bm, p, grid, stream); break;
-        case 64: st = launch_umma_t<64, 4>(wm, bm, p, grid, stream); break;
-        default: st = launch_umma_t<128, 2>(wm, bm, p, grid, stream); break;
+        case 16: st = launch_umma_t<16, 3, 3>(wm, bm, p, grid, stream); break;
+        case 32: st = launch_umma_t<32, 3, 3>(wm, bm, p, grid, stream); break;
+        case 64: st = launch_umma_t<64, 3, 3>(wm, bm, p, grid, stream); break;
+        default: st = launch_umma_t<128, 2, 4>(wm, bm, p, grid, stream); break;
     }
     if (st != BWLA_OK) return st;
     const int64_t total = (int64_t)M * N;
