@@ -52,16 +52,16 @@ static bool valid_rotation_dims(int64_t K, int n1, int n2) {
 
 // Which kernel family runs the contraction.  A forced family that cannot take the shape falls back to the simple one.
 static int resolve_path(int64_t M, int64_t K, int64_t N, int r, int bits) {
-    (void)r; (void)bits;
+    (void)bits;
     int path = g_forced_path;
     if (path == BWLA_PATH_AUTO) path = BWLA_PATH_I8;
     if (path == BWLA_PATH_BITPLANE) path = BWLA_PATH_SIMPLE;   // not built yet
-    if (path == BWLA_PATH_I8 && !umma_supports(M, K, N)) path = BWLA_PATH_SIMPLE;
+    if (path == BWLA_PATH_I8 && !umma_supports(M, K, N, r)) path = BWLA_PATH_SIMPLE;
     return path;
 }
 
-static int run_contraction(int path, GemmArgs& g, const int8_t* codes, int32_t* raw, cudaStream_t stream) {
-    if (path == BWLA_PATH_I8) return launch_gemm_umma(g, codes, g.acc_debug ? g.acc_debug : raw, stream);
+static int run_contraction(int path, GemmArgs& g, const int8_t* codes, cudaStream_t stream) {
+    if (path == BWLA_PATH_I8) return launch_gemm_umma(g, codes, stream);
     g.codes = codes;
     return launch_gemm_simple(g, stream);
 }
@@ -92,8 +92,8 @@ int bwla_rotate_quant_act(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
     if (((uintptr_t)codes & 15) || ((uintptr_t)P1 & 15) || ((uintptr_t)P2 & 15)) return BWLA_ERR_INVALID_ARG;
     int st = check_device();
     if (st != BWLA_OK) return st;
-    return launch_rotate_quant(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, 0, scales, nullptr, nullptr,
-                               nullptr, (cudaStream_t)stream);
+    return launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, 0, scales, nullptr, nullptr, 0, nullptr,
+                           (cudaStream_t)stream);
 }
 
 size_t bwla_workspace_bytes(int64_t M, int64_t K, int64_t N, int r, int bits) {
@@ -133,22 +133,18 @@ int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, cons
     char* base = (char*)workspace;
     float* scales = (float*)(base + ws.scales);
     int32_t* qsum = (int32_t*)(base + ws.qsum);
-    float* T = (float*)(base + ws.T);
+    void* Thl = base + ws.T;
     int8_t* codes = (int8_t*)(base + ws.codes);
     const int path = resolve_path(M, K, N, r, bits);
 
-    st = launch_rotate_quant(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum,
-                             nullptr, (uint32_t*)(base + ws.status), s);
+    st = launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum,
+                         V_bf16, r, Thl, s);
     if (st != BWLA_OK) return st;
-    if (r > 0) {
-        st = launch_lowrank_T(x_bf16, M, K, ldx, V_bf16, r, T, s);
-        if (st != BWLA_OK) return st;
-    }
     GemmArgs g{};
     g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
-    g.mu = mu; g.T = r > 0 ? T : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = nullptr;
+    g.mu = mu; g.Thl = r > 0 ? Thl : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = nullptr;
     g.status = (uint32_t*)(base + ws.status);
-    return run_contraction(path, g, codes, (int32_t*)(base + ws.acc), s);
+    return run_contraction(path, g, codes, s);
 }
 
 int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int64_t K, int bits,
@@ -169,21 +165,21 @@ int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int
     const Workspace ws = workspace_layout(M, K, N, r, bits);
     char* base = (char*)workspace;
     int32_t* qsum = (int32_t*)(base + ws.qsum);
-    float* T = (float*)(base + ws.T);
+    void* Thl = base + ws.T;
     const int path = resolve_path(M, K, N, r, bits);
 
     int8_t* inter = (path == BWLA_PATH_I8) ? (int8_t*)(base + ws.codes) : nullptr;
-    st = launch_prepare_codes(codes, M, K, inter, qsum, (uint32_t*)(base + ws.status), s);
+    st = launch_prepare_codes(codes, M, K, inter, qsum, s);
     if (st != BWLA_OK) return st;
     if (r > 0) {
-        st = launch_lowrank_T(x_bf16, M, K, ldx, V_bf16, r, T, s);
+        st = launch_prologue(x_bf16, M, K, ldx, nullptr, 0, nullptr, 0, bits, nullptr, 0, nullptr, nullptr, V_bf16, r, Thl, s);
         if (st != BWLA_OK) return st;
     }
     GemmArgs g{};
     g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
-    g.mu = mu; g.T = r > 0 ? T : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = acc_debug;
+    g.mu = mu; g.Thl = r > 0 ? Thl : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = acc_debug;
     g.status = (uint32_t*)(base + ws.status);
-    return run_contraction(path, g, inter ? inter : codes, (int32_t*)(base + ws.acc), s);
+    return run_contraction(path, g, inter ? inter : codes, s);
 }
 
 int bwla_check_status(void* workspace, void* stream) {

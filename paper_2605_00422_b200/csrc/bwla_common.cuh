@@ -54,11 +54,12 @@ struct ProfScope {
 // workspace layout (byte offsets into the caller's scratch buffer; every section 256-byte aligned)
 // ---------------------------------------------------------------------------------------------
 constexpr int kStatusBytes = 256;        // word 0: status; words 1..: where a bounded wait gave up
-constexpr int kBitplaneMaxTokens = 1;    // the bit-plane path keeps M*bits + 1 <= 8 MMA columns
-constexpr int kSplitKMaxTokens = 64;     // int32 partial sums in scratch are kept for M up to this
+constexpr int kLowrankPad = 64;          // T is kept as bf16 [3][M][64] (T = hi + mid + lo), zero beyond r <= 64
+
+__host__ __device__ inline int lowrank_cols(int r) { return r > kLowrankPad ? (r + 1) / 2 * 2 : kLowrankPad; }
 
 struct Workspace {
-    size_t status, scales, qsum, T, codes, planes, acc, total;
+    size_t status, scales, qsum, T, codes, total;
 };
 
 inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bits) {
@@ -67,11 +68,10 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     w.status = off; off += kStatusBytes;
     w.scales = off; off += align_up((size_t)M * 4, 256);
     w.qsum = off;   off += align_up((size_t)M * 4, 256);
-    w.T = off;      off += align_up((size_t)M * (size_t)(r > 0 ? r : 1) * 4, 256);
+    const size_t lr_cols = (size_t)lowrank_cols(r);
+    w.T = off;      off += align_up((size_t)M * lr_cols * 6, 256);     // bf16 [3][M][cols]
     w.codes = off;  off += align_up((size_t)M * (size_t)K, 256);
-    w.planes = off; off += (M <= kBitplaneMaxTokens) ? align_up((size_t)M * 8 * (size_t)(K / 32) * 4, 256) : 0;
-    w.acc = off;    off += align_up((size_t)M * (size_t)N * 4, 256);
-    (void)bits;
+    (void)N; (void)bits;
     w.total = off;
     return w;
 }
@@ -82,20 +82,17 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
 int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw, uint32_t* packed,
                       cudaStream_t stream);
 
-// Fused rotate + absmax + quantise.  codes_layout: 0 = natural k order, 1 = interleaved order used by the
-// tensor-core contraction (inside each group of 32, position 4*j + i holds k = j + 8*i).
-// qsum (int32 [M]) and planes (uint32 [M][bits+... ]) may be NULL.
-int launch_rotate_quant(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1,
-                        const float* P2, int n2, int bits, int8_t* codes, int codes_layout, float* scales,
-                        int32_t* qsum, uint32_t* planes, uint32_t* status, cudaStream_t stream);
-
-// T[t][j] = sum_k V[j][k] * x[t][k], fp32 accumulate.
-int launch_lowrank_T(const void* x, int64_t M, int64_t K, int64_t ldx, const void* V, int r, float* T,
-                     cudaStream_t stream);
+// One launch: fused rotate + absmax + quantise (skipped when codes == NULL) and T = V x (skipped when r == 0 or
+// Thl == NULL).  codes_layout: 0 = natural k order, 1 = interleaved order used by the tensor-core contraction (inside
+// each group of 32, position 4*j + i holds k = j + 8*i).  qsum (int32 [M]) may be NULL.
+// Thl: bf16 [3][M][cols], cols = lowrank_cols(r): T as the sum of three bf16 terms (exact for an fp32 T).
+int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2, int n2,
+                    int bits, int8_t* codes, int codes_layout, float* scales, int32_t* qsum, const void* V, int r,
+                    void* Thl, cudaStream_t stream);
 
 // qsum[t] = sum_k codes[t][k]; optionally rewrites natural-order codes into the interleaved order.
 int launch_prepare_codes(const int8_t* codes, int64_t M, int64_t K, int8_t* codes_interleaved, int32_t* qsum,
-                         uint32_t* status, cudaStream_t stream);
+                         cudaStream_t stream);
 
 struct GemmArgs {
     const int8_t* codes;      // [M][K]; natural order for the simple path
@@ -106,7 +103,7 @@ struct GemmArgs {
     const uint32_t* packed;   // [N][K/32]
     const float* alpha;       // [N]
     const float* mu;          // [N] or NULL
-    const float* T;           // [M][r] fp32 or NULL
+    const void* Thl;          // bf16 [3][M][lowrank_cols(r)] or NULL
     const void* U;            // bf16 [N][r] or NULL
     int r;
     void* out;                // bf16 [M][ldo] or NULL
@@ -117,8 +114,8 @@ struct GemmArgs {
 
 int launch_gemm_simple(const GemmArgs& a, cudaStream_t stream);
 
-// tcgen05 path.  codes_interleaved: int8 [M][K] in the interleaved order; raw: int32 [M][N] scratch.
-bool umma_supports(int64_t M, int64_t K, int64_t N);
-int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, int32_t* raw, cudaStream_t stream);
+// tcgen05 path with the fused epilogue.  codes_interleaved: int8 [M][K] in the interleaved order.
+bool umma_supports(int64_t M, int64_t K, int64_t N, int r);
+int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream);
 
 }  // namespace bwla

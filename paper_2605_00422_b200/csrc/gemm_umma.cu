@@ -1,24 +1,32 @@
-// Binary-weight contraction on tcgen05 tensor cores (kind::i8, accumulators in tensor memory).
+// Binary-weight contraction on tcgen05 tensor cores with the whole epilogue fused in.
 //
-//   D[n][t] = sum_k byte(n,k) * q[t][k],  byte(n,k) = -128 if the sign bit of weight (n,k) is set, else 0
+//   D[n][t]  = sum_k byte(n,k) * q[t][k],  byte(n,k) = -128 if the sign bit of weight (n,k) is set, else 0
 //   acc[t][n] = sum_k sign(n,k) * q[t][k] = -D/64 - sum_k q[t][k]            (sign = 2*bit - 1, exact in int32)
+//   D2[n][t] = sum_j U[n][j] * T[t][j]                                        (PSP low-rank term, Sec. 3.2)
+//   out[t][n] = bf16(alpha[n] * s_t * acc + D2 [+ mu[n] * s_t * sum_k q[t][k]])   (Eq. 4 on the accumulator)
 //
-// One CTA owns 128 output rows x up to 128 tokens x a slice of K:
-//   * a TMA warp streams packed sign words (128 rows x 128 bytes = 1024 weights per row, 128B-swizzled);
-//   * a second TMA warp streams the activation codes (tokens x 128 bytes per stage, the canonical K-major
-//     128B-swizzled UMMA layout);
-//   * four expander warps (one per tensor-memory lane quarter, thread = output row) turn each 32-bit word into eight
-//     registers of four int8 with one shift and one mask per register ((w << (7-j)) & 0x80808080) and write them
-//     with tcgen05.st into tensor memory, where they are the A operand -- expanded weights never touch shared memory;
-//   * one thread issues tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32) with A from tensor memory and B from
-//     shared memory, accumulating int32 in tensor memory;
-//   * the expander warps read the accumulator back (tcgen05.ld) and add it to the int32 result with red.global
-//     (split-K) or plain stores.
+// One CTA owns 128 output rows x up to 128 tokens x a slice of K; the CTAs that share a tile and split K form a
+// thread-block cluster and add their partial sums through distributed shared memory, so nothing but the bf16
+// result is written to global memory.  Inside a CTA:
+//   * warp 0 streams packed sign words by TMA (128 rows x 128 bytes = 1024 weights per row, 128B-swizzled); these
+//     loads do not depend on the activations and start before the preceding kernel of the stream has finished
+//     (programmatic dependent launch);
+//   * warp 2 waits for the preceding kernel, then streams the activation codes (tokens x 128 bytes per k-block, the
+//     canonical K-major 128B-swizzled UMMA layout) and the three bf16 terms of T;
+//   * warps 3..6 (one per tensor-memory lane quarter, thread = output row) stage the U tile in shared memory, then
+//     turn each 32-bit sign word into eight registers of four int8 with one shift and one mask per register
+//     ((w << (7-j)) & 0x80808080) and write them with tcgen05.st into tensor memory, where they are the A operand:
+//     expanded weights never touch shared memory;
+//   * one thread of warp 1 issues tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor memory, B from
+//     shared memory, int32 accumulator in tensor memory) and, last, the kind::f16 MMAs of the low-rank term
+//     (A = U tile, B = T as three bf16 terms, fp32 accumulator in tensor memory);
+//   * warps 3..6 read both accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
+//     scales and store bf16.
 // The shift-and-mask expansion meets the weights of a 32-group in the order k = j + 8*i (register j, byte i), so the
 // codes are stored in that interleaved order by the quantiser.
 //
 // Every wait is bounded: on give-up the CTA records where in the workspace status words, stops issuing work, lets
-// in-flight copies land, frees its tensor memory and returns.
+// in-flight copies land, still takes part in the cluster barriers, frees its tensor memory and returns.
 #include <cuda_bf16.h>
 
 #include "bwla_common.cuh"
@@ -30,16 +38,22 @@ using namespace ptx;
 
 constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
-constexpr int kBlockK = 128;             // K per code stage / per tensor-memory A stage
-constexpr int kTmemCols = 256;           // per CTA, so that two CTAs share an SM's 512 columns
+constexpr int kBlockK = 128;             // K per code sub-block / per tensor-memory A stage
 constexpr int kThreads = 224;            // warp 0: weight TMA, 1: MMA, 2: code TMA, 3..6: expand + epilogue
 constexpr uint32_t kWaitLimit = 1u << 20;   // polls per wait before giving up (tens of milliseconds)
 
 struct UmmaParams {
     int M, N, K;
-    int total_units, units_per_split;
-    int32_t* acc;        // [M][N] raw accumulator D
-    int use_atomics;
+    int total_units, splits;
+    int r;                       // low-rank width, 0..kLowrankPad
+    const float* scales;         // [M]
+    const int32_t* qsum;         // [M]
+    const float* alpha;          // [N]
+    const float* mu;             // [N] or NULL
+    const __nv_bfloat16* U;      // [N][r] or NULL
+    __nv_bfloat16* out;          // [M][ldo] or NULL
+    int64_t ldo;
+    int32_t* acc_debug;          // [M][N] or NULL
     uint32_t* status;
 };
 
@@ -47,18 +61,29 @@ struct UmmaParams {
 //   weights: WS stages of 128 rows x 128 bytes (one K-unit of 1024 weights per row);
 //   codes:   BS stages of 16 KB = SUBS k-blocks of (N_TOK rows x 128 bytes), so that small token tiles still move
 //            16 KB per barrier round trip;
-//   tensor memory: D in columns [0, DCOLS), then AS stages of 32 columns (one k-block of expanded weights each).
-template <int N_TOK, int WS, int BS>
+//   U tile:  128 rows x 64 bf16 (128 bytes), zero padded beyond r;  T tiles: 3 x (N_TOK rows x 64 bf16);
+//   tensor memory: D in columns [0, DCOLS), D2 in [DCOLS, 2*DCOLS), then AS stages of 32 columns (one k-block of
+//   expanded weights each).
+// The cluster reduction buffers (int32 and fp32, N_TOK x 128 each) reuse the stage memory once the K loop is over.
+template <int N_TOK, int WS, int BS, int TMEM_COLS>
 struct UmmaCfg {
     static constexpr int w_bytes = kRowsPerCta * 128;
     static constexpr int sub_bytes = N_TOK * 128;
     static constexpr int SUBS = (128 / N_TOK) < 1 ? 1 : ((128 / N_TOK) > 8 ? 8 : (128 / N_TOK));
     static constexpr int b_bytes = SUBS * sub_bytes;
     static constexpr int DCOLS = N_TOK <= 64 ? 64 : 128;
-    static constexpr int AS = (kTmemCols - DCOLS) / 32;
-    static constexpr int bars_off = WS * w_bytes + BS * b_bytes;
-    static constexpr int n_bars = 2 * WS + 2 * BS + 2 * AS + 1;
-    static constexpr int total = bars_off + n_bars * 8 + 64 + 1024;   // + slack for 1024-byte alignment
+    static constexpr int AS = (TMEM_COLS - 2 * DCOLS) / 32;
+    static constexpr int u_off = WS * w_bytes + BS * b_bytes;
+    static constexpr int t_off = u_off + kRowsPerCta * 128;
+    static constexpr int bars_off = t_off + 3 * sub_bytes;
+    static constexpr int n_bars = 2 * WS + 2 * BS + 2 * AS + 3;
+    static constexpr int misc_off = bars_off + n_bars * 8;            // tmem slot, abort flag
+    static constexpr int tok_off = misc_off + 16;                      // scales[N_TOK], qsum[N_TOK]
+    static constexpr int used = tok_off + 8 * N_TOK;
+    static constexpr int total = used + 1024;                          // + slack for 1024-byte alignment
+    static constexpr int red_bytes = 2 * N_TOK * kRowsPerCta * 4;
+    static constexpr bool can_split = red_bytes <= u_off;
+    static_assert(AS >= 2, "tensor memory: no room for the expanded-weight ring");
 };
 
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
@@ -79,16 +104,31 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
     return false;
 }
 
-template <int N_TOK, int WS, int BS>
+// One output element from its two accumulators.
+__device__ __forceinline__ void finish_element(const UmmaParams& p, int64_t t, int n, int32_t d, float l, float sc,
+                                               int32_t qs, float alpha_n, float mu_n) {
+    const int32_t acc = -(d >> 6) - qs;
+    if (p.acc_debug) p.acc_debug[t * p.N + n] = acc;
+    if (p.out) {
+        float y = __fmul_rn(__fmul_rn(alpha_n, sc), (float)acc) + l;
+        if (p.mu) y = fmaf(__fmul_rn(mu_n, sc), (float)qs, y);
+        p.out[t * p.ldo + n] = __float2bfloat16_rn(y);
+    }
+}
+
+template <int N_TOK, int WS, int BS, int TMEM_COLS>
 __global__ void __launch_bounds__(kThreads, 1)
-umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map, UmmaParams p) {
+umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map,
+                const __grid_constant__ CUtensorMap t_map, UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
-    using L = UmmaCfg<N_TOK, WS, BS>;
+    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS>;
     constexpr int AS = L::AS;
     constexpr int SUBS = L::SUBS;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* wbuf = smem;
     uint8_t* bbuf = smem + WS * L::w_bytes;
+    uint8_t* ubuf = smem + L::u_off;
+    uint8_t* tbuf = smem + L::t_off;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::bars_off);
     uint64_t* w_full = bars;                 // [WS]
     uint64_t* w_empty = bars + WS;           // [WS]
@@ -97,39 +137,50 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     uint64_t* a_full = b_empty + BS;         // [AS]
     uint64_t* a_empty = a_full + AS;         // [AS]
     uint64_t* d_full = a_empty + AS;         // [1]
-    __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag_s;
-    volatile int* abort_flag = &abort_flag_s;
+    uint64_t* u_full = d_full + 1;           // [1] U tile staged by the four expander warps
+    uint64_t* t_full = u_full + 1;           // [1] the three terms of T landed
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + L::misc_off);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
+    float* scale_s = reinterpret_cast<float*>(smem + L::tok_off);
+    int32_t* qsum_s = reinterpret_cast<int32_t*>(smem + L::tok_off + 4 * N_TOK);
+    int32_t* red_i = reinterpret_cast<int32_t*>(smem);                                 // [N_TOK][128], after the K loop
+    float* red_f = reinterpret_cast<float*>(smem + N_TOK * kRowsPerCta * 4);           // [N_TOK][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * kRowsPerCta;
     const int t0 = blockIdx.y * N_TOK;
-    const int unit_begin = blockIdx.z * p.units_per_split;
-    const int unit_end = min(p.total_units, unit_begin + p.units_per_split);
+    const int split = blockIdx.z;                      // == rank in the (1,1,splits) cluster
+    const int unit_begin = (int)(((int64_t)split * p.total_units) / p.splits);
+    const int unit_end = (int)(((int64_t)(split + 1) * p.total_units) / p.splits);
+    const bool lowrank = p.r > 0;
+    const bool lowrank_here = lowrank && split == 0;   // the low-rank accumulator lives in the first CTA of a cluster
 
     if (threadIdx.x == 0) {
-        // a CTA of this launch that already gave up makes the rest of the grid skip its work
-        abort_flag_s = (p.status && *reinterpret_cast<volatile uint32_t*>(p.status) != 0) ? 1 : 0;
+        *abort_flag = 0;
         for (int i = 0; i < WS; ++i) { mbar_init(&w_full[i], 1); mbar_init(&w_empty[i], 4); }
         for (int i = 0; i < BS; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < AS; ++i) { mbar_init(&a_full[i], 4); mbar_init(&a_empty[i], 1); }
         mbar_init(d_full, 1);
+        mbar_init(u_full, 4);
+        mbar_init(t_full, 1);
         fence_barrier_init();
         fence_proxy_async();
     }
     if (warp == 1) {
-        tmem_alloc(&tmem_base_slot, kTmemCols);
+        tmem_alloc(tmem_base_slot, TMEM_COLS);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t tmem_base = *tmem_base_slot;
+    // the next kernel of the stream may start its own independent preamble now
+    griddep_launch_dependents();
 
     auto sub_count = [&](int u) { return min(kUnitK / kBlockK, (p.K - u * kUnitK) / kBlockK); };
 
     if (warp == 0) {
-        // ---------------- packed sign words: HBM -> shared memory ----------------
+        // ---------------- packed sign words: HBM -> shared memory (independent of the preceding kernel) ----------------
         if (elect_one()) {
             tma_prefetch_desc(&w_map);
             int ws = 0; uint32_t wph = 0;
@@ -142,9 +193,16 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);   // let copies in flight land
         }
     } else if (warp == 2) {
-        // ---------------- activation codes: L2/HBM -> shared memory ----------------
+        // ---------------- activation codes and T: L2 -> shared memory ----------------
         if (elect_one()) {
             tma_prefetch_desc(&b_map);
+            if (lowrank_here) tma_prefetch_desc(&t_map);
+            griddep_wait();                       // codes, scales and T come from the preceding kernel
+            if (p.status && *reinterpret_cast<volatile uint32_t*>(p.status) != 0) *abort_flag = 1;   // the call already failed
+            if (lowrank_here && !*abort_flag) {
+                mbar_expect_tx(t_full, 3 * L::sub_bytes);
+                for (int h = 0; h < 3; ++h) tma_load_3d(tbuf + h * L::sub_bytes, &t_map, 0, t0, h, t_full);
+            }
             int bs = 0; uint32_t bph = 0;
             bool ok = true;
             for (int u = unit_begin; u < unit_end && ok && !*abort_flag; ++u) {
@@ -163,8 +221,10 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     } else if (warp == 1) {
         // ---------------- MMA issue ----------------
         if (elect_one()) {
-            // instruction descriptor: D = s32, A = s8 (tensor memory, K-major), B = s8 (shared, K-major), M = 128
+            // instruction descriptors: D = s32, A = s8 (tensor memory, K-major), B = s8 (shared, K-major), M = 128;
+            // and D = f32, A = B = bf16 (shared, K-major), M = 128
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
+            const uint32_t idesc_lr = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
             int as = 0; uint32_t aph = 0; int bs = 0; uint32_t bph = 0; uint32_t first = 1;
             bool ok = true;
             for (int u = unit_begin; u < unit_end && ok; ++u) {
@@ -175,7 +235,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
                     tc_fence_after();
                     const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
-                    const uint32_t a_addr = tmem_base + L::DCOLS + 32 * as;
+                    const uint32_t a_addr = tmem_base + 2 * L::DCOLS + 32 * as;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         mma_i8_ts(tmem_base, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, first ? 0u : 1u);
@@ -189,13 +249,56 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     }
                 }
             }
+            if (ok && lowrank_here) {
+                if (!wait_or_abort(u_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x32); ok = false; }
+                if (ok && !wait_or_abort(t_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x33); ok = false; }
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t u_addr = smem_u32(ubuf);
+#pragma unroll
+                    for (int h = 0; h < 3; ++h) {
+                        const uint32_t t_addr = smem_u32(tbuf + h * L::sub_bytes);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            mma_f16_ss(tmem_base + L::DCOLS, smem_desc_sw128(u_addr, 32 * i), smem_desc_sw128(t_addr, 32 * i),
+                                       idesc_lr, (h | i) ? 1u : 0u);
+                    }
+                }
+            }
             tc_commit(d_full);
         }
     } else {
-        // ---------------- expand sign bits into tensor memory, then drain the accumulator ----------------
+        // ---------------- U tile, expansion of sign bits into tensor memory, then the epilogue ----------------
         const int q = warp & 3;                       // tensor-memory lane quarter this warp may touch
         const int row = q * 32 + lane;
+        const int e = threadIdx.x - 96;               // 0..127 among the expander threads
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        if (lowrank_here) {
+            // 128 rows x 8 chunks of 16 bytes, 128B-swizzled K-major; rows beyond N and columns beyond r are zero
+            const bool vec = (p.r % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.U) & 15) == 0);
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const int idx = it * 128 + e;
+                const int ur = idx >> 3, ch = idx & 7;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                const int n = n0 + ur;
+                if (n < p.N && ch * 8 < p.r) {
+                    const __nv_bfloat16* src = p.U + (int64_t)n * p.r + ch * 8;
+                    if (vec) {
+                        v = __ldg(reinterpret_cast<const uint4*>(src));
+                    } else {
+                        uint32_t w[4] = {0u, 0u, 0u, 0u};
+                        for (int c = 0; c < 8 && ch * 8 + c < p.r; ++c)
+                            w[c >> 1] |= (uint32_t)__bfloat16_as_ushort(src[c]) << (16 * (c & 1));
+                        v = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+                *reinterpret_cast<uint4*>(ubuf + ur * 128 + ((ch ^ (ur & 7)) << 4)) = v;
+            }
+            fence_proxy_async();                      // generic-proxy stores -> visible to the tensor core's reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(u_full);
+        }
         int ws = 0; uint32_t wph = 0; int as = 0; uint32_t aph = 0;
         bool ok = true;
         for (int u = unit_begin; u < unit_end && ok; ++u) {
@@ -212,7 +315,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     for (int j = 0; j < 8; ++j) v[8 * i + j] = (w[i] << (7 - j)) & 0x80808080u;
                 if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&a_empty[as], aph ^ 1, abort_flag))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
                 tc_fence_after();
-                tmem_st_32x32(tmem_base + lane_addr + L::DCOLS + 32 * as, v);
+                tmem_st_32x32(tmem_base + lane_addr + 2 * L::DCOLS + 32 * as, v);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -223,26 +326,55 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (lane == 0) mbar_arrive(&w_empty[ws]);
             if (++ws == WS) { ws = 0; wph ^= 1; }
         }
-        if (ok && unit_begin < unit_end) {
+        // per-token scale and code sum of this tile (written by the preceding kernel)
+        griddep_wait();
+        if (e < N_TOK) {
+            const int t = t0 + e;
+            scale_s[e] = t < p.M ? p.scales[t] : 0.f;
+            qsum_s[e] = t < p.M ? p.qsum[t] : 0;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");     // the four expander warps only
+        if (ok) {
             if (!__all_sync(0xFFFFFFFFu, wait_or_abort(d_full, 0, abort_flag))) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
-        if (ok && unit_begin < unit_end) {
+        if (ok) {
             tc_fence_after();
             const int n = n0 + row;
+            if (p.splits == 1) {
+                const float alpha_n = n < p.N ? p.alpha[n] : 0.f;
+                const float mu_n = (p.mu && n < p.N) ? p.mu[n] : 0.f;
 #pragma unroll 1
-            for (int c = 0; c < N_TOK / 16; ++c) {
-                uint32_t v[16];
-                tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
-                tc_wait_ld();
-                if (n < p.N) {
+                for (int c = 0; c < N_TOK / 16; ++c) {
+                    if (t0 + 16 * c >= p.M) break;                 // warp-uniform
+                    uint32_t v[16], l[16];
+                    tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
+                    if (lowrank) tmem_ld_32x16(tmem_base + lane_addr + L::DCOLS + 16 * c, l);
+                    tc_wait_ld();
+                    if (n < p.N) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int t = t0 + 16 * c + j;
-                        if (t < p.M) {
-                            int32_t* dst = p.acc + (int64_t)t * p.N + n;
-                            if (p.use_atomics) atomicAdd(dst, (int32_t)v[j]);
-                            else *dst = (int32_t)v[j];
+                        for (int j = 0; j < 16; ++j) {
+                            const int tt = 16 * c + j;
+                            if (t0 + tt < p.M)
+                                finish_element(p, t0 + tt, n, (int32_t)v[j], lowrank ? __uint_as_float(l[j]) : 0.f,
+                                               scale_s[tt], qsum_s[tt], alpha_n, mu_n);
                         }
+                    }
+                }
+            } else if (L::can_split) {
+                // partial sums of this K slice -> shared memory, transposed so that a token's 128 rows are contiguous
+#pragma unroll 1
+                for (int c = 0; c < N_TOK / 16; ++c) {
+                    if (t0 + 16 * c >= p.M) break;
+                    uint32_t v[16];
+                    tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) red_i[(16 * c + j) * kRowsPerCta + row] = (int32_t)v[j];
+                    if (lowrank_here) {
+                        tmem_ld_32x16(tmem_base + lane_addr + L::DCOLS + 16 * c, v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) red_f[(16 * c + j) * kRowsPerCta + row] = __uint_as_float(v[j]);
                     }
                 }
             }
@@ -250,36 +382,35 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
+    if (p.splits > 1) {
+        // every thread of every CTA of the cluster takes part, whether or not its CTA gave up
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        if (L::can_split && warp >= 3 && !*abort_flag) {
+            const int row = (warp & 3) * 32 + lane;
+            const int n = n0 + row;
+            if (n < p.N) {
+                const float alpha_n = p.alpha[n];
+                const float mu_n = p.mu ? p.mu[n] : 0.f;
+                // tokens of the tile are dealt round-robin to the CTAs of the cluster
+                for (int tt = split; tt < N_TOK && t0 + tt < p.M; tt += p.splits) {
+                    const uint32_t off_i = smem_u32(&red_i[tt * kRowsPerCta + row]);
+                    int32_t d = 0;
+                    for (int c = 0; c < p.splits; ++c) d += (int32_t)ld_shared_cluster_u32(map_shared_rank(off_i, c));
+                    float l = 0.f;
+                    if (lowrank) l = __uint_as_float(ld_shared_cluster_u32(map_shared_rank(smem_u32(&red_f[tt * kRowsPerCta + row]), 0)));
+                    finish_element(p, t0 + tt, n, d, l, scale_s[tt], qsum_s[tt], alpha_n, mu_n);
+                }
+            }
+        }
+        // nobody leaves while a neighbour may still read its shared memory
+        cluster_arrive_release();
+        cluster_wait_acquire();
+    }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
-    }
-}
-
-// -------------------------------------------------------------------------------------------------
-// epilogue from the raw int32 accumulator: acc = -D/64 - qsum; out = bf16(alpha * s * acc + U.T + mu * s * qsum)
-// -------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) finalize_kernel(GemmArgs a, int32_t* raw) {
-    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= a.M * a.N) return;
-    const int64_t t = idx / a.N, n = idx - t * a.N;
-    const int32_t d = raw[idx];
-    const int32_t qs = a.qsum[t];
-    const int32_t acc = -(d >> 6) - qs;
-    if (a.acc_debug) a.acc_debug[idx] = acc;        // may alias raw: same element, read before written
-    if (a.out) {
-        const float sc = a.scales[t];
-        float y = __fmul_rn(__fmul_rn(a.alpha[n], sc), (float)acc);
-        if (a.r > 0) {
-            const __nv_bfloat16* u = (const __nv_bfloat16*)a.U + n * a.r;
-            const float* tr = a.T + t * a.r;
-            float l = 0.f;
-            for (int j = 0; j < a.r; ++j) l = fmaf(__bfloat162float(u[j]), tr[j], l);
-            y += l;
-        }
-        if (a.mu) y = fmaf(__fmul_rn(a.mu[n], sc), (float)qs, y);
-        ((__nv_bfloat16*)a.out)[t * a.ldo + n] = __float2bfloat16_rn(y);
+        tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -302,80 +433,112 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-static int make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t inner, uint64_t outer,
-                       uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle sw,
-                       CUtensorMapL2promotion promo) {
+// rank 2 or 3; dims/box innermost first; strides in bytes for dimensions 1..rank-1
+static int make_map(CUtensorMap* map, CUtensorMapDataType dt, int rank, const void* base, const uint64_t* dims,
+                    const uint64_t* strides, const uint32_t* box, CUtensorMapSwizzle sw, CUtensorMapL2promotion promo) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return BWLA_ERR_CUDA;
-    cuuint64_t dims[2] = {inner, outer};
-    cuuint64_t strides[1] = {row_stride_bytes};
-    cuuint32_t box[2] = {box_inner, box_outer};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+    cuuint64_t d[3]; cuuint64_t s[2]; cuuint32_t b[3]; cuuint32_t estr[3] = {1, 1, 1};
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) s[i] = strides[i];
+    CUresult r = fn(map, dt, (cuuint32_t)rank, const_cast<void*>(base), d, s, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                     promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return BWLA_ERR_CUDA; }
     return BWLA_OK;
 }
 
-template <int N_TOK, int WS, int BS>
-static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const UmmaParams& p, dim3 grid, cudaStream_t s) {
-    using L = UmmaCfg<N_TOK, WS, BS>;
-    constexpr int AS = L::AS;
-    constexpr int SUBS = L::SUBS;
+template <int N_TOK, int WS, int BS, int TMEM_COLS>
+static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUtensorMap& tm, const UmmaParams& p,
+                         dim3 grid, cudaStream_t s) {
+    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS>;
+    auto kernel = umma_w1a_kernel<N_TOK, WS, BS, TMEM_COLS>;
     static thread_local int configured = -1;
     int dev = 0;
     BWLA_CUDA_TRY(cudaGetDevice(&dev));
     if (configured != dev) {
-        BWLA_CUDA_TRY(cudaFuncSetAttribute(umma_w1a_kernel<N_TOK, WS, BS>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total));
+        BWLA_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::total));
         configured = dev;
     }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = L::total;
+    cfg.stream = s;
+    cudaLaunchAttribute attrs[2];
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = 1; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = grid.z;
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = 2;
     ProfScope prof(kProfContraction, s);
-    umma_w1a_kernel<N_TOK, WS, BS><<<grid, kThreads, L::total, s>>>(wm, bm, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, wm, bm, tm, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return cuda_fail(e); }
     return after_launch();
 }
 
-bool umma_supports(int64_t M, int64_t K, int64_t N) {
-    return M > 0 && N > 0 && K % 128 == 0 && M * N < (int64_t)1 << 31 && encode_tiled_fn() != nullptr;
+bool umma_supports(int64_t M, int64_t K, int64_t N, int r) {
+    return M > 0 && N > 0 && K % 128 == 0 && r <= kLowrankPad && M * N < (int64_t)1 << 31 && M < (int64_t)1 << 30 &&
+           encode_tiled_fn() != nullptr;
 }
 
-// codes_interleaved: int8 [M][K] in the interleaved order.  raw: int32 [M][N] scratch (or the caller's acc_debug).
-int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, int32_t* raw, cudaStream_t stream) {
+// How many CTAs share a tile and split K.  Enough to put about one CTA on every SM, never more than the units there
+// are, never more than the portable cluster size, and only powers of two.
+static int choose_splits(int tiles, int units, bool can_split) {
+    if (!can_split) return 1;
+    int s = 1;
+    while (s * 2 <= 8 && s * 2 <= units && tiles * s * 2 <= 148 + 148 / 4) s *= 2;
+    return s;
+}
+
+// codes_interleaved: int8 [M][K] in the interleaved order.  a.Thl: bf16 [3][M][64], T = hi + mid + lo.
+int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream) {
     const int M = (int)a.M, N = (int)a.N, K = (int)a.K;
     const int n_tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
     const int row_tiles = (N + kRowsPerCta - 1) / kRowsPerCta;
     const int tok_tiles = (M + n_tok - 1) / n_tok;
     const int units = (K + kUnitK - 1) / kUnitK;
-    // split K until there are about two CTAs per SM
-    int split = 1;
-    const int target = 148 * 2;
-    while (split < units && row_tiles * tok_tiles * split < target) ++split;
-    int ups = (units + split - 1) / split;
-    split = (units + ups - 1) / ups;
+    const int split = choose_splits(row_tiles * tok_tiles, units, n_tok <= 64);
 
-    CUtensorMap wm, bm;
-    int st = make_map_2d(&wm, CU_TENSOR_MAP_DATA_TYPE_UINT32, a.packed, (uint64_t)K / 32, (uint64_t)N, (uint64_t)K / 8,
-                         32, kRowsPerCta, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
-    if (st != BWLA_OK) return st;
-    st = make_map_2d(&bm, CU_TENSOR_MAP_DATA_TYPE_UINT8, codes_interleaved, (uint64_t)K, (uint64_t)M, (uint64_t)K,
-                     kBlockK, (uint32_t)n_tok, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
-    if (st != BWLA_OK) return st;
+    CUtensorMap wm, bm, tm;
+    {
+        const uint64_t dims[2] = {(uint64_t)K / 32, (uint64_t)N};
+        const uint64_t strides[1] = {(uint64_t)K / 8};
+        const uint32_t box[2] = {32, kRowsPerCta};
+        int st = make_map(&wm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, a.packed, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+        if (st != BWLA_OK) return st;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+        const uint64_t strides[1] = {(uint64_t)K};
+        const uint32_t box[2] = {kBlockK, (uint32_t)n_tok};
+        int st = make_map(&bm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, codes_interleaved, dims, strides, box,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+        if (st != BWLA_OK) return st;
+    }
+    if (a.r > 0) {
+        const uint64_t dims[3] = {(uint64_t)kLowrankPad, (uint64_t)M, 3};
+        const uint64_t strides[2] = {(uint64_t)kLowrankPad * 2, (uint64_t)M * kLowrankPad * 2};
+        const uint32_t box[3] = {(uint32_t)kLowrankPad, (uint32_t)n_tok, 1};
+        int st = make_map(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, a.Thl, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+        if (st != BWLA_OK) return st;
+    } else {
+        tm = bm;   // never dereferenced
+    }
 
     UmmaParams p{};
-    p.M = M; p.N = N; p.K = K; p.total_units = units; p.units_per_split = ups; p.acc = raw;
-    p.use_atomics = split > 1; p.status = a.status;
-    if (split > 1) BWLA_CUDA_TRY(cudaMemsetAsync(raw, 0, (size_t)M * N * 4, stream));
+    p.M = M; p.N = N; p.K = K; p.total_units = units; p.splits = split; p.r = a.r;
+    p.scales = a.scales; p.qsum = a.qsum; p.alpha = a.alpha; p.mu = a.mu; p.U = (const __nv_bfloat16*)a.U;
+    p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug; p.status = a.status;
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     switch (n_tok) {
-        case 16: st = launch_umma_t<16, 3, 3>(wm, bm, p, grid, stream); break;
-        case 32: st = launch_umma_t<32, 3, 3>(wm, bm, p, grid, stream); break;
-        case 64: st = launch_umma_t<64, 3, 3>(wm, bm, p, grid, stream); break;
-        default: st = launch_umma_t<128, 2, 4>(wm, bm, p, grid, stream); break;
+        case 16: return launch_umma_t<16, 3, 2, 256>(wm, bm, tm, p, grid, stream);
+        case 32: return launch_umma_t<32, 3, 2, 256>(wm, bm, tm, p, grid, stream);
+        case 64: return launch_umma_t<64, 2, 2, 256>(wm, bm, tm, p, grid, stream);
+        default: return launch_umma_t<128, 2, 4, 512>(wm, bm, tm, p, grid, stream);
     }
-    if (st != BWLA_OK) return st;
-    const int64_t total = (int64_t)M * N;
-    ProfScope prof(kProfFinalize, stream);
-    finalize_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(a, raw);
-    return after_launch();
 }
 
 }  // namespace bwla

@@ -1,17 +1,49 @@
-// Online OKT + per-token symmetric quantiser, fused: one block per token.
+// The per-call prologue, one launch: online OKT + per-token symmetric quantiser, and the first stage of the PSP
+// low-rank branch.
 //
 //   X = reshape(x_t, n1 x n2) (row-major), Z = X * P2, Y = P1^T * Z, amax = max|Y|,
-//   q = clamp(rne(Y * (qmax / amax)), +-qmax), s_t = amax / qmax.
+//   q = clamp(rne(Y * (qmax / amax)), +-qmax), s_t = amax / qmax;          T[t][j] = sum_k V[j][k] * x_t[k]
 //
 // (Sec. 3.1: R = R1 (x) R2 evaluated as two small contractions on the reshaped vector; Sec. 4.1: per-token
-// activation quantisation.)  X, Z and Y live in shared memory (2*K floats); Y never touches HBM.  The two
-// contractions are register-tiled 4x4 fp32 FMA loops; the absmax is a warp-shuffle + shared-memory reduction;
-// codes leave as 128-bit stores.
+// activation quantisation; Sec. 3.2: W x = (W - M) x + A (B x).)
+//
+// Rotation blocks: a thread-block cluster of C CTAs owns one token.  CTA c owns a slab of rows of X: it computes
+// that slab of Z and stores it into the full-size Z buffer of every CTA of the cluster (distributed shared memory),
+// then computes the same slab of rows of Y from the full Z, exchanges its absmax and its code sum the same way and
+// quantises its slab.  With few tokens this spreads one token's 2*K*(n1+n2) flops over C SMs; with many tokens C = 1.
+// X, Z and Y never touch HBM.  Both contractions are register-tiled 4x4 fp32 FMA loops; codes leave as 128-bit stores.
+//
+// Low-rank blocks (after the rotation blocks in the same grid): each reduces two rows of V against a tile of 16
+// tokens with 128-bit loads and writes T split into three bf16 terms (T = hi + mid + lo, all 24 bits of the fp32 sum), the form
+// the tensor-core epilogue of the contraction consumes.
+//
+// The kernel is launched with programmatic stream serialisation: everything up to the first global store may
+// overlap the preceding kernel of the stream; every block waits for that kernel before it stores anything.
 #include <cuda_bf16.h>
 
 #include "bwla_common.cuh"
+#include "umma_ptx.cuh"
 
 namespace bwla {
+
+using namespace ptx;
+
+constexpr int kLrTokens = 16;     // tokens per low-rank block
+constexpr int kLrRows = 2;        // rows of V per low-rank block
+constexpr int kLrMaxWarps = 16;   // blocks have at most 512 threads
+
+struct PrologueParams {
+    const __nv_bfloat16* x; int64_t M; int K; int64_t ldx;
+    // rotation + quantiser (rot_blocks == 0 skips them)
+    const float* P1; int n1; const float* P2; int n2; int bits;
+    int8_t* codes; int codes_layout; float* scales; int32_t* qsum;
+    int C;              // CTAs per token (cluster size)
+    int rot_blocks;     // M * C
+    int row_gran;       // slab boundaries are multiples of this many rows of X
+    int slab_cap;       // floats reserved for one slab
+    // low-rank
+    const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
+};
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -25,120 +57,43 @@ __device__ __forceinline__ int warp_sum(int v) {
     return v;
 }
 
-// Generic contraction used when n2 is not a multiple of 4 (odd test shapes): one output per thread step.
-__device__ void rotate_scalar(const float* __restrict__ X, float* __restrict__ Z, float* __restrict__ Y,
-                              const float* __restrict__ P1, int n1, const float* __restrict__ P2, int n2,
-                              float& amax) {
-    const int K = n1 * n2;
-    for (int o = threadIdx.x; o < K; o += blockDim.x) {
-        const int a = o / n2, d = o - a * n2;
-        float s = 0.f;
-        for (int b = 0; b < n2; ++b) s = fmaf(X[a * n2 + b], __ldg(P2 + b * n2 + d), s);
-        Z[o] = s;
-    }
-    __syncthreads();
-    for (int o = threadIdx.x; o < K; o += blockDim.x) {
-        const int c = o / n2, d = o - c * n2;
-        float s = 0.f;
-        for (int a = 0; a < n1; ++a) s = fmaf(__ldg(P1 + a * n1 + c), Z[a * n2 + d], s);
-        Y[o] = s;
-        amax = fmaxf(amax, fabsf(s));
-    }
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float4 v) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
-// Register-tiled contraction, n2 % 4 == 0: each thread owns 4 rows x 4 columns of the output.
-__device__ void rotate_tiled(const float* __restrict__ X, float* __restrict__ Z, float* __restrict__ Y,
-                             const float* __restrict__ P1, int n1, const float* __restrict__ P2, int n2,
-                             float& amax) {
-    const int dt_count = n2 >> 2;
-    const int mt_count = (n1 + 3) >> 2;
-    const int tiles = dt_count * mt_count;
-    // Z = X * P2
-    for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
-        const int mt = tile / dt_count, d0 = (tile - mt * dt_count) << 2;
-        const int a0 = mt << 2;
-        const float* xr[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) xr[i] = X + min(a0 + i, n1 - 1) * n2;
-        float acc[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-        const float* p = P2 + d0;
-#pragma unroll 4
-        for (int b = 0; b < n2; ++b) {
-            const float4 pv = __ldg(reinterpret_cast<const float4*>(p + (size_t)b * n2));
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float xa = xr[i][b];
-                acc[i][0] = fmaf(xa, pv.x, acc[i][0]);
-                acc[i][1] = fmaf(xa, pv.y, acc[i][1]);
-                acc[i][2] = fmaf(xa, pv.z, acc[i][2]);
-                acc[i][3] = fmaf(xa, pv.w, acc[i][3]);
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (a0 + i < n1)
-                *reinterpret_cast<float4*>(Z + (a0 + i) * n2 + d0) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-    }
-    __syncthreads();
-    // Y = P1^T * Z   (Y overwrites X, which is dead now)
-    for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
-        const int mt = tile / dt_count, d0 = (tile - mt * dt_count) << 2;
-        const int c0 = mt << 2;
-        int cc[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) cc[i] = min(c0 + i, n1 - 1);
-        float acc[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-#pragma unroll 4
-        for (int a = 0; a < n1; ++a) {
-            const float4 zv = *reinterpret_cast<const float4*>(Z + a * n2 + d0);
-            const float* prow = P1 + (size_t)a * n1;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float pa = __ldg(prow + cc[i]);
-                acc[i][0] = fmaf(pa, zv.x, acc[i][0]);
-                acc[i][1] = fmaf(pa, zv.y, acc[i][1]);
-                acc[i][2] = fmaf(pa, zv.z, acc[i][2]);
-                acc[i][3] = fmaf(pa, zv.w, acc[i][3]);
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (c0 + i < n1) {
-                *reinterpret_cast<float4*>(Y + (c0 + i) * n2 + d0) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                amax = fmaxf(amax, fmaxf(fmaxf(fabsf(acc[i][0]), fabsf(acc[i][1])), fmaxf(fabsf(acc[i][2]), fabsf(acc[i][3]))));
-            }
-    }
+__device__ __forceinline__ int slab_begin(int c, int C, int n1, int gran) {
+    if (c >= C) return n1;
+    return (int)(((int64_t)n1 * c / C) / gran * gran);
 }
 
-// codes_layout 0: byte p of a 32-group holds k = p.  1: byte 4*j + i holds k = j + 8*i (j < 8, i < 4), the
-// order in which the tensor-core contraction meets the weights after its shift-and-mask expansion.
-__global__ void rotate_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int K, int64_t ldx,
-                                    const float* __restrict__ P1, int n1, const float* __restrict__ P2, int n2,
-                                    int bits, int8_t* __restrict__ codes, int codes_layout,
-                                    float* __restrict__ scales, int32_t* __restrict__ qsum,
-                                    uint32_t* __restrict__ planes, uint32_t* __restrict__ status) {
-    if (status && blockIdx.x == 0 && threadIdx.x == 0) status[0] = 0;   // this call's status starts clean
-    extern __shared__ __align__(16) float smem[];
-    float* bufX = smem;        // X, later Y
-    float* bufZ = smem + K;    // Z
+// ---------------------------------------------------------------------------------------------
+// rotation + quantiser
+// ---------------------------------------------------------------------------------------------
+__device__ void rotate_role(const PrologueParams& p, float* smem) {
+    const int C = p.C;
+    const int rank = C > 1 ? (int)cluster_ctarank() : 0;
+    const int64_t t = blockIdx.x / C;
+    const int n1 = p.n1, n2 = p.n2, K = p.K;
+    const int a_lo = slab_begin(rank, C, n1, p.row_gran), a_hi = slab_begin(rank + 1, C, n1, p.row_gran);
+    const int rows = a_hi - a_lo;
+    float* Xs = smem;                          // this CTA's slab of X, later of Y
+    float* Zf = smem + p.slab_cap;             // all of Z
+    float* slots = Zf + K;                     // [0..7] absmax per rank, [8..15] code sum per rank (int)
     __shared__ float red_max[32];
     __shared__ int red_sum;
-    const int qmax = (1 << (bits - 1)) - 1;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int qmax = (1 << (p.bits - 1)) - 1;
 
-    for (int64_t t = blockIdx.x; t < M; t += gridDim.x) {
-        const __nv_bfloat16* xt = x + t * ldx;
-        if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0) {
+    // ---- this slab of x_t -> fp32 in shared memory
+    {
+        const __nv_bfloat16* xt = p.x + t * p.ldx + (int64_t)a_lo * n2;
+        const int len = rows * n2;
+        if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0 && (len & 7) == 0) {
             const uint4* xv = reinterpret_cast<const uint4*>(xt);
-            for (int i = threadIdx.x; i < (K >> 3); i += blockDim.x) {
+            for (int i = threadIdx.x; i < (len >> 3); i += blockDim.x) {
                 const uint4 v = __ldg(xv + i);
                 const uint32_t w[4] = {v.x, v.y, v.z, v.w};
                 float f[8];
@@ -147,103 +102,350 @@ __global__ void rotate_quant_kernel(const __nv_bfloat16* __restrict__ x, int64_t
                     f[2 * j] = __uint_as_float(w[j] << 16);
                     f[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
                 }
-                *reinterpret_cast<float4*>(bufX + 8 * i) = make_float4(f[0], f[1], f[2], f[3]);
-                *reinterpret_cast<float4*>(bufX + 8 * i + 4) = make_float4(f[4], f[5], f[6], f[7]);
+                *reinterpret_cast<float4*>(Xs + 8 * i) = make_float4(f[0], f[1], f[2], f[3]);
+                *reinterpret_cast<float4*>(Xs + 8 * i + 4) = make_float4(f[4], f[5], f[6], f[7]);
             }
         } else {
-            for (int k = threadIdx.x; k < K; k += blockDim.x) bufX[k] = __bfloat162float(xt[k]);
+            for (int k = threadIdx.x; k < len; k += blockDim.x) Xs[k] = __bfloat162float(xt[k]);
         }
-        if (threadIdx.x == 0) red_sum = 0;
-        __syncthreads();
+    }
+    if (threadIdx.x == 0) red_sum = 0;
+    // every CTA of the cluster must be running before its shared memory is written from outside
+    if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
+    griddep_launch_dependents();
 
-        float amax = 0.f;
-        if ((n2 & 3) == 0) rotate_tiled(bufX, bufZ, bufX, P1, n1, P2, n2, amax);
-        else {
-            // the scalar variant may not alias: Y goes to bufX only after Z is complete (it syncs inside)
-            rotate_scalar(bufX, bufZ, bufX, P1, n1, P2, n2, amax);
-        }
-        amax = warp_max(amax);
-        if (lane == 0) red_max[warp] = amax;
-        __syncthreads();
-        amax = (lane < nwarps) ? red_max[lane] : 0.f;
-        amax = warp_max(amax);
-
-        float inv, scale;
-        if (amax == 0.f) { inv = 0.f; scale = 1.f; }
-        else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
-
-        int local_sum = 0;
-        int8_t* ct = codes + t * (int64_t)K;
-        const int words = K >> 5;
-        for (int g = threadIdx.x; g < words; g += blockDim.x) {
-            const float* y = bufX + 32 * g;
-            int q[32];
+    float amax = 0.f;
+    if ((n2 & 3) == 0) {
+        const int dt_count = n2 >> 2;
+        const int tiles = ((rows + 3) >> 2) * dt_count;
+        // ---- Z slab = X slab * P2, stored into every CTA's full Z
+        for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
+            const int mt = tile / dt_count, d0 = (tile - mt * dt_count) << 2;
+            const int r0 = mt << 2;
+            const float* xr[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float4 v = *reinterpret_cast<const float4*>(y + 4 * i);
-                const float f[4] = {v.x, v.y, v.z, v.w};
+            for (int i = 0; i < 4; ++i) xr[i] = Xs + min(r0 + i, rows - 1) * n2;
+            float acc[4][4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    int c = __float2int_rn(__fmul_rn(f[j], inv));
-                    c = max(-qmax, min(qmax, c));
-                    q[4 * i + j] = c;
-                    local_sum += c;
-                }
-            }
-            uint32_t w[8];
+            for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint32_t v = 0;
+                for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+            const float* pp = p.P2 + d0;
+#pragma unroll 4
+            for (int b = 0; b < n2; ++b) {
+                const float4 pv = __ldg(reinterpret_cast<const float4*>(pp + (size_t)b * n2));
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int k = codes_layout ? (j + 8 * i) : (4 * j + i);
-                    v |= (uint32_t)(q[k] & 0xFF) << (8 * i);
+                    const float xa = xr[i][b];
+                    acc[i][0] = fmaf(xa, pv.x, acc[i][0]);
+                    acc[i][1] = fmaf(xa, pv.y, acc[i][1]);
+                    acc[i][2] = fmaf(xa, pv.z, acc[i][2]);
+                    acc[i][3] = fmaf(xa, pv.w, acc[i][3]);
                 }
-                w[j] = v;
             }
-            uint4* dst = reinterpret_cast<uint4*>(ct + 32 * g);
-            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-            if (planes) {
-                // plane i of u = q + qmax, LSB-first like the weight words; plane index `bits` is all ones
-                uint32_t* pt = planes + (t * 8) * (int64_t)words;
-                for (int i = 0; i < bits; ++i) {
-                    uint32_t pw = 0;
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) pw |= (uint32_t)(((q[k] + qmax) >> i) & 1) << k;
-                    pt[(int64_t)i * words + g] = pw;
+            for (int i = 0; i < 4; ++i)
+                if (r0 + i < rows) {
+                    float* dst = Zf + (a_lo + r0 + i) * n2 + d0;
+                    const float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                    if (C == 1) {
+                        *reinterpret_cast<float4*>(dst) = v;
+                    } else {
+                        const uint32_t local = smem_u32(dst);
+                        for (int c = 0; c < C; ++c) st_cluster_v4(map_shared_rank(local, c), v);
+                    }
                 }
-                for (int i = bits; i < 8; ++i) pt[(int64_t)i * words + g] = (i == bits) ? 0xFFFFFFFFu : 0u;
+        }
+        if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
+        // ---- Y slab = (P1^T * Z) rows [a_lo, a_hi); Y overwrites the X slab, which is dead now
+        for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
+            const int mt = tile / dt_count, d0 = (tile - mt * dt_count) << 2;
+            const int r0 = mt << 2;
+            int cc[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) cc[i] = a_lo + min(r0 + i, rows - 1);
+            float acc[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+            for (int a = 0; a < n1; ++a) {
+                const float4 zv = *reinterpret_cast<const float4*>(Zf + a * n2 + d0);
+                const float* prow = p.P1 + (size_t)a * n1;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float pa = __ldg(prow + cc[i]);
+                    acc[i][0] = fmaf(pa, zv.x, acc[i][0]);
+                    acc[i][1] = fmaf(pa, zv.y, acc[i][1]);
+                    acc[i][2] = fmaf(pa, zv.z, acc[i][2]);
+                    acc[i][3] = fmaf(pa, zv.w, acc[i][3]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (r0 + i < rows) {
+                    *reinterpret_cast<float4*>(Xs + (r0 + i) * n2 + d0) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(acc[i][0]), fabsf(acc[i][1])), fmaxf(fabsf(acc[i][2]), fabsf(acc[i][3]))));
+                }
+        }
+    } else {
+        // generic shapes (n2 not a multiple of 4; C == 1): one output per thread step
+        for (int o = threadIdx.x; o < K; o += blockDim.x) {
+            const int a = o / n2, d = o - a * n2;
+            float s = 0.f;
+            for (int b = 0; b < n2; ++b) s = fmaf(Xs[a * n2 + b], __ldg(p.P2 + b * n2 + d), s);
+            Zf[o] = s;
+        }
+        __syncthreads();
+        for (int o = threadIdx.x; o < K; o += blockDim.x) {
+            const int c = o / n2, d = o - c * n2;
+            float s = 0.f;
+            for (int a = 0; a < n1; ++a) s = fmaf(__ldg(p.P1 + a * n1 + c), Zf[a * n2 + d], s);
+            Xs[o] = s;
+            amax = fmaxf(amax, fabsf(s));
+        }
+    }
+    // ---- absmax over the block, then over the cluster
+    amax = warp_max(amax);
+    if (lane == 0) red_max[warp] = amax;
+    __syncthreads();
+    amax = (lane < nwarps) ? red_max[lane] : 0.f;
+    amax = warp_max(amax);
+    if (C > 1) {
+        if (threadIdx.x < C) st_cluster_u32(map_shared_rank(smem_u32(slots + rank), threadIdx.x), __float_as_uint(amax));
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        float m = (lane < C) ? slots[lane] : 0.f;
+        amax = warp_max(m);
+    }
+
+    float inv, scale;
+    if (amax == 0.f) { inv = 0.f; scale = 1.f; }
+    else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
+
+    // nothing is stored to global memory before the preceding kernel of the stream has completed
+    griddep_wait();
+
+    int local_sum = 0;
+    int8_t* ct = p.codes + t * (int64_t)K + (int64_t)a_lo * n2;
+    const int words = (rows * n2) >> 5;
+    for (int g = threadIdx.x; g < words; g += blockDim.x) {
+        const float* y = Xs + 32 * g;
+        int q[32];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 v = *reinterpret_cast<const float4*>(y + 4 * i);
+            const float f[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int c = __float2int_rn(__fmul_rn(f[j], inv));
+                c = max(-qmax, min(qmax, c));
+                q[4 * i + j] = c;
+                local_sum += c;
             }
         }
-        local_sum = warp_sum(local_sum);
-        if (lane == 0 && local_sum != 0) atomicAdd(&red_sum, local_sum);
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            scales[t] = scale;
-            if (qsum) qsum[t] = red_sum;
+        uint32_t w[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint32_t v = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int k = p.codes_layout ? (j + 8 * i) : (4 * j + i);
+                v |= (uint32_t)(q[k] & 0xFF) << (8 * i);
+            }
+            w[j] = v;
         }
-        __syncthreads();
+        uint4* dst = reinterpret_cast<uint4*>(ct + 32 * g);
+        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+    local_sum = warp_sum(local_sum);
+    if (lane == 0 && local_sum != 0) atomicAdd(&red_sum, local_sum);
+    __syncthreads();
+    if (C > 1) {
+        if (threadIdx.x == 0) st_cluster_u32(map_shared_rank(smem_u32(slots + 8 + rank), 0), (uint32_t)red_sum);
+        cluster_arrive_release();
+        cluster_wait_acquire();
+    }
+    if (rank == 0 && threadIdx.x == 0) {
+        int s = red_sum;
+        if (C > 1) { s = 0; for (int c = 0; c < C; ++c) s += (int)__float_as_uint(slots[8 + c]); }
+        p.scales[t] = scale;
+        if (p.qsum) p.qsum[t] = s;
     }
 }
 
-int launch_rotate_quant(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1,
-                        const float* P2, int n2, int bits, int8_t* codes, int codes_layout, float* scales,
-                        int32_t* qsum, uint32_t* planes, uint32_t* status, cudaStream_t stream) {
+// ---------------------------------------------------------------------------------------------
+// T = V x, written as three bf16 terms
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void fma8(float (&acc)[kLrTokens], int tt, const uint4& v, const uint4& xv) {
+    const uint32_t a[4] = {v.x, v.y, v.z, v.w}, b[4] = {xv.x, xv.y, xv.z, xv.w};
+    float s = acc[tt];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        s = fmaf(__uint_as_float(a[i] << 16), __uint_as_float(b[i] << 16), s);
+        s = fmaf(__uint_as_float(a[i] & 0xFFFF0000u), __uint_as_float(b[i] & 0xFFFF0000u), s);
+    }
+    acc[tt] = s;
+}
+
+__device__ void lowrank_role(const PrologueParams& p, int b) {
+    const int jblocks = p.lr_cols / kLrRows;
+    const int jb = b % jblocks;
+    const int64_t t0 = (int64_t)(b / jblocks) * kLrTokens;
+    if (t0 >= p.M) return;
+    const int j0 = jb * kLrRows;
+    const int nt = (int)min((int64_t)kLrTokens, p.M - t0);
+    float acc[kLrRows][kLrTokens];
+#pragma unroll
+    for (int j = 0; j < kLrRows; ++j)
+#pragma unroll
+        for (int i = 0; i < kLrTokens; ++i) acc[j][i] = 0.f;
+    griddep_launch_dependents();
+    if (j0 < p.r) {
+        const int K = p.K;
+        const bool two = j0 + 1 < p.r;
+        const __nv_bfloat16* v0 = p.V + (int64_t)j0 * K;
+        const __nv_bfloat16* v1 = p.V + (int64_t)(two ? j0 + 1 : j0) * K;
+        const __nv_bfloat16* xt = p.x + t0 * p.ldx;
+        const bool vec = ((reinterpret_cast<uintptr_t>(p.V) | reinterpret_cast<uintptr_t>(p.x)) & 15) == 0 && (p.ldx & 7) == 0;
+        if (vec) {
+            for (int kc = threadIdx.x; kc < (K >> 3); kc += blockDim.x) {
+                const uint4 a0 = __ldg(reinterpret_cast<const uint4*>(v0) + kc);
+                const uint4 a1 = __ldg(reinterpret_cast<const uint4*>(v1) + kc);
+#pragma unroll
+                for (int tt = 0; tt < kLrTokens; ++tt) {
+                    if (tt < nt) {
+                        const uint4 xv = __ldg(reinterpret_cast<const uint4*>(xt + tt * p.ldx) + kc);
+                        fma8(acc[0], tt, a0, xv);
+                        fma8(acc[1], tt, a1, xv);
+                    }
+                }
+            }
+        } else {
+            for (int k = threadIdx.x; k < K; k += blockDim.x) {
+                const float a0 = __bfloat162float(v0[k]), a1 = __bfloat162float(v1[k]);
+#pragma unroll
+                for (int tt = 0; tt < kLrTokens; ++tt) {
+                    if (tt < nt) {
+                        const float xv = __bfloat162float(xt[tt * p.ldx + k]);
+                        acc[0][tt] = fmaf(a0, xv, acc[0][tt]);
+                        acc[1][tt] = fmaf(a1, xv, acc[1][tt]);
+                    }
+                }
+            }
+        }
+        if (!two) {
+#pragma unroll
+            for (int i = 0; i < kLrTokens; ++i) acc[1][i] = 0.f;
+        }
+    }
+    __shared__ float red[kLrMaxWarps][kLrRows * kLrTokens];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int j = 0; j < kLrRows; ++j)
+#pragma unroll
+        for (int i = 0; i < kLrTokens; ++i) {
+            float v = acc[j][i];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+            if (lane == 0) red[warp][j * kLrTokens + i] = v;
+        }
+    __syncthreads();
+    griddep_wait();
+    if (threadIdx.x < kLrRows * kLrTokens) {
+        const int j = threadIdx.x / kLrTokens, i = threadIdx.x % kLrTokens;
+        if (i < nt) {
+            float s = 0.f;
+#pragma unroll
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w][threadIdx.x];
+            // three bf16 terms carry all 24 bits of the fp32 sum
+            const __nv_bfloat16 hi = __float2bfloat16_rn(s);
+            const float r1 = s - __bfloat162float(hi);
+            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+            const int64_t o = (t0 + i) * p.lr_cols + j0 + j;
+            p.Thl[o] = hi;
+            p.Thl[p.M * p.lr_cols + o] = mid;
+            p.Thl[2 * p.M * p.lr_cols + o] = lo;
+        }
+    }
+}
+
+__global__ void prologue_kernel(PrologueParams p) {
+    extern __shared__ __align__(16) float smem[];
+    if ((int)blockIdx.x < p.rot_blocks) rotate_role(p, smem);
+    else lowrank_role(p, (int)blockIdx.x - p.rot_blocks);
+}
+
+static int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
+
+int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2, int n2,
+                    int bits, int8_t* codes, int codes_layout, float* scales, int32_t* qsum, const void* V, int r,
+                    void* Thl, cudaStream_t stream) {
     if (M == 0) return BWLA_OK;
-    const size_t smem = (size_t)K * 8;
+    const bool rotate = codes != nullptr;
+    PrologueParams p{};
+    p.x = (const __nv_bfloat16*)x; p.M = M; p.K = (int)K; p.ldx = ldx;
+    p.P1 = P1; p.n1 = n1; p.P2 = P2; p.n2 = n2; p.bits = bits;
+    p.codes = codes; p.codes_layout = codes_layout; p.scales = scales; p.qsum = qsum;
+    p.V = (const __nv_bfloat16*)V; p.r = r; p.Thl = (__nv_bfloat16*)Thl;
+    p.lr_cols = lowrank_cols(r);
+
+    int C = 1;
+    int threads = 256;
+    size_t smem = 0;
+    if (rotate) {
+        const int gran = 32 / gcd_int(n2, 32);
+        if ((n2 & 3) == 0) {
+            // spread one token over several SMs while there are few tokens and the token is worth splitting
+            const double flops = 2.0 * (double)K * (n1 + n2);
+            while (C < 8 && M * (C * 2) <= 160 && flops / (C * 2) >= 2.5e5 && n1 / (C * 2) >= gran) C *= 2;
+        }
+        int cap = 0;
+        for (int c = 0; c < C; ++c) {
+            const int lo = (int)(((int64_t)n1 * c / C) / gran * gran);
+            const int hi = (c + 1 >= C) ? n1 : (int)(((int64_t)n1 * (c + 1) / C) / gran * gran);
+            cap = cap > (hi - lo) ? cap : (hi - lo);
+        }
+        p.C = C; p.rot_blocks = (int)(M * C); p.row_gran = gran; p.slab_cap = (cap * n2 + 3) / 4 * 4;
+        smem = ((size_t)p.slab_cap + (size_t)K + 16) * 4;
+        const int tiles = ((cap + 3) / 4) * (n2 / 4 > 0 ? n2 / 4 : 1);
+        threads = (n2 & 3) ? 256 : (tiles > 384 ? 512 : (tiles > 192 ? 384 : 256));
+    } else {
+        p.C = 1; p.rot_blocks = 0;
+    }
+    int lr_blocks = 0;
+    if (r > 0 && Thl) {
+        lr_blocks = (p.lr_cols / kLrRows) * (int)((M + kLrTokens - 1) / kLrTokens);
+    }
+    int grid = p.rot_blocks + lr_blocks;
+    grid = (grid + C - 1) / C * C;
+    if (grid == 0) return BWLA_OK;
+
     static thread_local int configured_device = -1;
     int dev = 0;
     BWLA_CUDA_TRY(cudaGetDevice(&dev));
     if (configured_device != dev) {
-        BWLA_CUDA_TRY(cudaFuncSetAttribute(rotate_quant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 25600 * 8));
+        BWLA_CUDA_TRY(cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 25600 * 8 + 64));
         configured_device = dev;
     }
-    const int threads = (K >= 8192) ? 512 : 256;
-    const unsigned grid = (unsigned)(M < 148 * 64 ? M : 148 * 64);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attrs[2];
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = (unsigned)C; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = 2;
     ProfScope prof(kProfRotateQuant, stream);
-    rotate_quant_kernel<<<grid, threads, smem, stream>>>((const __nv_bfloat16*)x, M, (int)K, ldx, P1, n1, P2, n2, bits,
-                                                         codes, codes_layout, scales, qsum, planes, status);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, prologue_kernel, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return cuda_fail(e); }
     return after_launch();
 }
 
@@ -251,9 +453,7 @@ int launch_rotate_quant(const void* x, int64_t M, int64_t K, int64_t ldx, const 
 // qsum and interleaving for codes supplied by the caller
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) prepare_codes_kernel(const int8_t* __restrict__ codes, int64_t M, int K,
-                                                            int8_t* __restrict__ inter, int32_t* __restrict__ qsum,
-                                                            uint32_t* __restrict__ status) {
-    if (status && blockIdx.x == 0 && threadIdx.x == 0) status[0] = 0;   // this call's status starts clean
+                                                            int8_t* __restrict__ inter, int32_t* __restrict__ qsum) {
     __shared__ int red_sum;
     const int64_t t = blockIdx.x;
     if (threadIdx.x == 0) red_sum = 0;
@@ -293,10 +493,10 @@ __global__ void __launch_bounds__(256) prepare_codes_kernel(const int8_t* __rest
 }
 
 int launch_prepare_codes(const int8_t* codes, int64_t M, int64_t K, int8_t* codes_interleaved, int32_t* qsum,
-                         uint32_t* status, cudaStream_t stream) {
+                         cudaStream_t stream) {
     if (M == 0) return BWLA_OK;
     ProfScope prof(kProfPrepare, stream);
-    prepare_codes_kernel<<<(unsigned)M, 256, 0, stream>>>(codes, M, (int)K, codes_interleaved, qsum, status);
+    prepare_codes_kernel<<<(unsigned)M, 256, 0, stream>>>(codes, M, (int)K, codes_interleaved, qsum);
     return after_launch();
 }
 

@@ -7,9 +7,13 @@ Tolerances (all stated here, used by every parity test):
     exactly +-1 and are counted.
   * per-token scale: within 2e-6 relative of amax / qmax (amax comes out of two fp32 contractions of up to
     n1 + n2 = 320 terms; sqrt(320) * 2^-24 ~ 1e-6 of the row's scale).
-  * bf16 output: relative L2 error <= 2e-3 (asserted for outputs of >= 1024 elements); every element within 1 bf16 ulp of the correctly rounded oracle value
-    or within 1e-2 * rms(y) + 2^-8 * |y| of the fp64 oracle value (a correctly rounded bf16 is already up to
-    2^-9 * |y| away, so the absolute bound alone cannot hold for elements several rms large).
+  * bf16 output: relative L2 error <= 2e-3 (asserted for outputs of >= 1024 elements); every element within
+    1e-2 * rms(y) + 2^-8 * |y| of the fp64 oracle value (a correctly rounded bf16 is already up to 2^-9 * |y| away,
+    so the absolute bound alone cannot hold for elements several rms large).
+  * where the test also knows the two summands of the output (the scaled integer term and the low-rank term):
+    every element within 1 bf16 step of the correctly rounded oracle value plus 2^-18 * (|term1| + |term2|).  The
+    kernel evaluates the sum in fp32 (tensor-core fp32 accumulation for the low-rank term), whose error is
+    proportional to the summands, not to a sum that may cancel; 2^-18 leaves 6 bits over the fp32 unit roundoff.
 """
 from __future__ import annotations
 
@@ -59,6 +63,12 @@ class DeviceLayer:
             self.packed_host = words_to_host(self.packed)
 
 
+def summand_magnitude(ref: dict, alpha: np.ndarray) -> np.ndarray:
+    """|alpha * s * acc| + |y - alpha * s * acc| of an oracle result: the size of what the output sum adds up."""
+    main = alpha.astype(np.float64)[None, :] * ref["scales"].astype(np.float64)[:, None] * ref["acc"].astype(np.float64)
+    return np.abs(main) + np.abs(ref["y"] - main)
+
+
 def check_codes(gpu_codes: np.ndarray, gpu_scales: np.ndarray, Y: np.ndarray, bits: int) -> dict:
     """The benchmark spec rule for the integer codes; returns counts for the report."""
     ref = oracle.quantize(Y, bits, "f64")
@@ -79,7 +89,7 @@ def check_codes(gpu_codes: np.ndarray, gpu_scales: np.ndarray, Y: np.ndarray, bi
             "scale_rel_err": float(scale_err.max())}
 
 
-def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray) -> dict:
+def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray, mag: np.ndarray = None) -> dict:
     got = gen.f32_from_bf16_bits(gpu_bits).astype(np.float64)
     err = got - y_ref
     rel_l2 = float(np.linalg.norm(err) / max(np.linalg.norm(y_ref), 1e-300))
@@ -94,6 +104,7 @@ def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray) -> dict:
     ref_bits = oracle.bf16_round(y_ref)
     ref_val = gen.f32_from_bf16_bits(ref_bits).astype(np.float64)
     step = np.maximum(np.abs(ref_val), 2.0 ** -126) * 2.0 ** -7
-    ulps = np.abs(got - ref_val) / step
+    slack = 0.0 if mag is None else 2.0 ** -18 * mag
+    ulps = np.maximum(np.abs(got - ref_val) - slack, 0.0) / step
     return {"rel_l2": rel_l2, "max_abs_over_rms": float(np.abs(err).max() / max(rms, 1e-300)),
             "max_bf16_steps": float(ulps.max()), "exact_bf16": float(np.mean(gpu_bits == ref_bits))}

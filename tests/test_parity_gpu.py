@@ -56,6 +56,10 @@ ROT_CASES = [
     (86, 128, 4, 6),      # LLaMA down_proj, n1 not a multiple of 4
     (64, 128, 4, 8),
     (160, 160, 3, 4),     # largest K (25600)
+    (64, 80, 1, 6),       # one token spread over a cluster of CTAs
+    (160, 160, 1, 8),
+    (86, 128, 2, 6),      # uneven row slabs
+    (24, 8, 1, 6),        # slab boundaries must stay on 32-element groups
 ]
 
 
@@ -124,7 +128,7 @@ def _run_layer_case(bwla, cfg, shape, M, bits, with_mu=False, direct_words=False
                                              want_acc=True, workspace=ws)
         assert bwla.bwla_check_status(ws) == 0
         assert np.array_equal(acc.cpu().numpy().astype(np.int64), ref["acc"])
-        rep2 = H.check_output(H.bf16_to_host(out2), ref["y"])
+        rep2 = H.check_output(H.bf16_to_host(out2), ref["y"], H.summand_magnitude(ref, lay.alpha))
         assert rep2["max_bf16_steps"] <= 1.0 + 1e-9
     finally:
         bwla.bwla_force_path(bwla.BWLA_PATH_AUTO)
