@@ -86,9 +86,14 @@ size_t bwla_workspace_bytes(int64_t M, int64_t K, int64_t N, int r, int bits);
  *   packed device uint32 [N][K/32];  alpha device fp32 [N];  mu device fp32 [N] or NULL   (Eq. 4)
  *   U_bf16 device bf16 [N][r], V_bf16 device bf16 [r][K]; both may be NULL iff r == 0      (Sec. 3.2, M = A B)
  *   out_bf16 device bf16 [M][ldo], ldo >= N
- *   workspace device, 256-byte aligned, >= bwla_workspace_bytes(M,K,N,r,bits); contents are scratch.
- *     Its first word is a status word that bounded device-side waits set; read it with bwla_check_status.
+ *   workspace device, 256-byte aligned, >= bwla_workspace_bytes(M,K,N,r,bits); contents are scratch, except that
+ *     its first 256 bytes must be zero before the first call that uses it.  The first word is a status word that
+ *     bounded device-side waits set and that stays set (later calls on this workspace then skip their work) until
+ *     bwla_check_status reads and clears it.
  *   Two calls that share a workspace must be ordered on one stream.
+ *   The kernels are launched with programmatic stream serialisation: the part of a call that does not depend on
+ *   earlier work (streaming the sign words into shared memory) may overlap the tail of the preceding kernel of
+ *   `stream`; every global store waits for that kernel to finish.
  */
 int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
                      const float* P1, int n1, const float* P2, int n2, int bits,
@@ -133,9 +138,11 @@ int bwla_last_launch_count(void);
 
 /*
  * Per-kernel timing for benchmarks.  While enabled (per calling thread), every kernel the library launches is
- * bracketed by CUDA events recorded on the launching stream.  bwla_profile_collect waits for them, adds the
+ * bracketed by CUDA events recorded on the launching stream and launched without programmatic overlap, so that an
+ * event pair times one kernel alone.  bwla_profile_collect waits for them, adds the
  * elapsed milliseconds and launch counts per kernel kind into two caller arrays of 8 entries
- * (0 rotate+quantise, 1 low-rank V x, 2 contraction, 3 accumulator epilogue, 4 code preparation, 5 pack_signs)
+ * (0 prologue: rotate + quantise + V x, 2 contraction with its fused epilogue, 4 code preparation, 5 pack_signs;
+ * the other entries stay zero)
  * and forgets the events.  Host arrays.  Do not enable during stream capture.
  */
 int bwla_profile_enable(int on);

@@ -13,7 +13,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbwla.so")
+LIB_PATH = os.environ.get("BWLA_LIBRARY", os.path.join(_HERE, "libbwla.so"))   # override: another build of the same ABI
 
 BWLA_OK = 0
 BWLA_ERR_INVALID_ARG = -1
@@ -228,7 +228,7 @@ def bwla_check_status(workspace: torch.Tensor) -> int:
     return int(_lib.bwla_check_status(_ptr(workspace), _stream()))
 
 
-PROFILE_KINDS = ("rotate_quant", "lowrank_vx", "contraction", "acc_epilogue", "prepare_codes", "pack_signs")
+PROFILE_KINDS = ("prologue", "unused1", "contraction", "unused3", "prepare_codes", "pack_signs")
 
 
 def bwla_profile_enable(on: bool) -> None:

@@ -15,6 +15,8 @@ static thread_local bool g_prof_on = false;
 static thread_local std::vector<ProfPair>* g_prof = nullptr;       // pairs recorded since the last collect
 static thread_local std::vector<ProfPair>* g_prof_pool = nullptr;  // idle pairs, reused so that recording stays cheap
 
+unsigned launch_overlap_allowed() { return g_prof_on ? 0u : 1u; }
+
 void prof_begin(int kind, cudaStream_t stream) {
     if (!g_prof_on) return;
     if (!g_prof) { g_prof = new std::vector<ProfPair>(); g_prof_pool = new std::vector<ProfPair>(); }

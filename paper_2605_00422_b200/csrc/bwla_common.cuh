@@ -40,8 +40,11 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // optional per-kernel timing (bwla_profile_enable / bwla_profile_collect): CUDA events recorded on the launching
 // stream right around each kernel launch, summed per kernel kind.  Off by default; not usable under stream capture.
 // ---------------------------------------------------------------------------------------------
-enum ProfKind { kProfRotateQuant = 0, kProfLowrankT = 1, kProfContraction = 2, kProfFinalize = 3, kProfPrepare = 4,
+enum ProfKind { kProfRotateQuant = 0, kProfContraction = 2, kProfPrepare = 4,
                 kProfPack = 5, kProfKinds = 8 };
+// 1 unless per-kernel timing is on: timed kernels are launched fully serialised so that each event pair brackets
+// one kernel alone.
+unsigned launch_overlap_allowed();
 void prof_begin(int kind, cudaStream_t stream);
 void prof_end(int kind, cudaStream_t stream);
 struct ProfScope {

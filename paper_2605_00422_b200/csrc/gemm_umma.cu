@@ -11,17 +11,20 @@
 //   * warp 0 streams packed sign words by TMA (128 rows x 128 bytes = 1024 weights per row, 128B-swizzled); these
 //     loads do not depend on the activations and start before the preceding kernel of the stream has finished
 //     (programmatic dependent launch);
-//   * warp 2 waits for the preceding kernel, then streams the activation codes (tokens x 128 bytes per k-block, the
-//     canonical K-major 128B-swizzled UMMA layout) and the three bf16 terms of T;
-//   * warps 3..6 (one per tensor-memory lane quarter, thread = output row) stage the U tile in shared memory, then
-//     turn each 32-bit sign word into eight registers of four int8 with one shift and one mask per register
-//     ((w << (7-j)) & 0x80808080) and write them with tcgen05.st into tensor memory, where they are the A operand:
-//     expanded weights never touch shared memory;
-//   * one thread of warp 1 issues tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor memory, B from
-//     shared memory, int32 accumulator in tensor memory) and, last, the kind::f16 MMAs of the low-rank term
-//     (A = U tile, B = T as three bf16 terms, fp32 accumulator in tensor memory);
-//   * warps 3..6 read both accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
-//     scales and store bf16.
+//   * warp 1 waits for the preceding kernel, then streams the three bf16 terms of T and the activation codes
+//     (tokens x 128 bytes per k-block, the canonical K-major 128B-swizzled UMMA layout);
+//   * warps 6..13 (two per tensor-memory lane quarter, thread = output row, the two warps of a quarter taking
+//     alternate k-blocks) stage the U tile in shared memory, then turn each 32-bit sign word into eight registers
+//     of four int8 with one shift and one mask per register ((w << (7-j)) & 0x80808080) and write them with
+//     tcgen05.st into tensor memory, where they are the A operand: expanded weights never touch shared memory.
+//     A warp expands its next k-block while the store of the previous one completes;
+//   * NISS threads (one each in warps 2..5) issue tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor
+//     memory, B from shared memory), taking k-blocks round-robin, each into an int32 accumulator of its own in
+//     tensor memory: with few tokens an MMA is short and the issue latency of one thread would be the bottleneck.
+//     The first of them also issues the kind::f16 MMAs of the low-rank term (A = U tile, B = T as three bf16
+//     terms, fp32 accumulator in tensor memory);
+//   * warps 6..13 read the accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
+//     scales, transpose through shared memory and store bf16 with 128-bit stores.
 // The shift-and-mask expansion meets the weights of a 32-group in the order k = j + 8*i (register j, byte i), so the
 // codes are stored in that interleaved order by the quantiser.
 //
@@ -39,7 +42,9 @@ using namespace ptx;
 constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
 constexpr int kBlockK = 128;             // K per code sub-block / per tensor-memory A stage
-constexpr int kThreads = 224;            // warp 0: weight TMA, 1: MMA, 2: code TMA, 3..6: expand + epilogue
+constexpr int kFirstExpander = 192;      // warps 0, 1: TMA; warps 2..5: MMA issue; warps 6..13: expand + epilogue
+constexpr int kExpanders = 256;
+constexpr int kThreads = kFirstExpander + kExpanders;
 constexpr uint32_t kWaitLimit = 1u << 20;   // polls per wait before giving up (tens of milliseconds)
 
 struct UmmaParams {
@@ -62,17 +67,19 @@ struct UmmaParams {
 //   codes:   BS stages of 16 KB = SUBS k-blocks of (N_TOK rows x 128 bytes), so that small token tiles still move
 //            16 KB per barrier round trip;
 //   U tile:  128 rows x 64 bf16 (128 bytes), zero padded beyond r;  T tiles: 3 x (N_TOK rows x 64 bf16);
-//   tensor memory: D in columns [0, DCOLS), D2 in [DCOLS, 2*DCOLS), then AS stages of 32 columns (one k-block of
-//   expanded weights each).
-// The cluster reduction buffers (int32 and fp32, N_TOK x 128 each) reuse the stage memory once the K loop is over.
-template <int N_TOK, int WS, int BS, int TMEM_COLS>
+//   tensor memory: NISS int32 accumulators of N_TOK columns, the fp32 low-rank accumulator (N_TOK columns), then AS
+//   stages of 32 columns (one k-block of expanded weights each).
+// The cluster reduction buffers (int32 and fp32, N_TOK x 128 each) and the bf16 output tile reuse the stage memory
+// once the K loop is over.
+template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS>
 struct UmmaCfg {
     static constexpr int w_bytes = kRowsPerCta * 128;
     static constexpr int sub_bytes = N_TOK * 128;
     static constexpr int SUBS = (128 / N_TOK) < 1 ? 1 : ((128 / N_TOK) > 8 ? 8 : (128 / N_TOK));
     static constexpr int b_bytes = SUBS * sub_bytes;
-    static constexpr int DCOLS = N_TOK <= 64 ? 64 : 128;
-    static constexpr int AS = (TMEM_COLS - 2 * DCOLS) / 32;
+    static constexpr int D2_COL = NISS * N_TOK;
+    static constexpr int A_COL = ((NISS + 1) * N_TOK + 31) / 32 * 32;
+    static constexpr int AS = ((TMEM_COLS - A_COL) / 32) & ~1;        // even: the two warps of a quarter alternate
     static constexpr int u_off = WS * w_bytes + BS * b_bytes;
     static constexpr int t_off = u_off + kRowsPerCta * 128;
     static constexpr int bars_off = t_off + 3 * sub_bytes;
@@ -83,7 +90,9 @@ struct UmmaCfg {
     static constexpr int total = used + 1024;                          // + slack for 1024-byte alignment
     static constexpr int red_bytes = 2 * N_TOK * kRowsPerCta * 4;
     static constexpr bool can_split = red_bytes <= u_off;
+    static_assert(NISS >= 1 && NISS <= 4, "one to four issuing warps");
     static_assert(AS >= 2, "tensor memory: no room for the expanded-weight ring");
+    static_assert(N_TOK * kRowsPerCta * 2 <= u_off, "output tile does not fit the stage memory");
 };
 
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
@@ -99,29 +108,27 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (i > 32) __nanosleep(32);
+        if (i > 8192) __nanosleep(64);             // a sleeping warp wakes up late: only back off on long waits
     }
     return false;
 }
 
-// One output element from its two accumulators.
-__device__ __forceinline__ void finish_element(const UmmaParams& p, int64_t t, int n, int32_t d, float l, float sc,
-                                               int32_t qs, float alpha_n, float mu_n) {
+// One output value from its two accumulators.
+__device__ __forceinline__ float finish_value(const UmmaParams& p, int64_t t, int n, int32_t d, float l, float sc,
+                                              int32_t qs, float alpha_n, float mu_n) {
     const int32_t acc = -(d >> 6) - qs;
     if (p.acc_debug) p.acc_debug[t * p.N + n] = acc;
-    if (p.out) {
-        float y = __fmul_rn(__fmul_rn(alpha_n, sc), (float)acc) + l;
-        if (p.mu) y = fmaf(__fmul_rn(mu_n, sc), (float)qs, y);
-        p.out[t * p.ldo + n] = __float2bfloat16_rn(y);
-    }
+    float y = __fmul_rn(__fmul_rn(alpha_n, sc), (float)acc) + l;
+    if (p.mu) y = fmaf(__fmul_rn(mu_n, sc), (float)qs, y);
+    return y;
 }
 
-template <int N_TOK, int WS, int BS, int TMEM_COLS>
+template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map,
                 const __grid_constant__ CUtensorMap t_map, UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
-    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS>;
+    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS>;
     constexpr int AS = L::AS;
     constexpr int SUBS = L::SUBS;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -136,15 +143,17 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     uint64_t* b_empty = b_full + BS;         // [BS]
     uint64_t* a_full = b_empty + BS;         // [AS]
     uint64_t* a_empty = a_full + AS;         // [AS]
-    uint64_t* d_full = a_empty + AS;         // [1]
-    uint64_t* u_full = d_full + 1;           // [1] U tile staged by the four expander warps
+    uint64_t* d_full = a_empty + AS;         // [1] every issuing thread's MMAs have completed
+    uint64_t* u_full = d_full + 1;           // [1] U tile staged by the expander warps
     uint64_t* t_full = u_full + 1;           // [1] the three terms of T landed
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + L::misc_off);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
     float* scale_s = reinterpret_cast<float*>(smem + L::tok_off);
     int32_t* qsum_s = reinterpret_cast<int32_t*>(smem + L::tok_off + 4 * N_TOK);
-    int32_t* red_i = reinterpret_cast<int32_t*>(smem);                                 // [N_TOK][128], after the K loop
-    float* red_f = reinterpret_cast<float*>(smem + N_TOK * kRowsPerCta * 4);           // [N_TOK][128]
+    // after the K loop the stage memory is free:
+    int32_t* red_i = reinterpret_cast<int32_t*>(smem);                                 // [N_TOK][128] partial sums
+    float* red_f = reinterpret_cast<float*>(smem + N_TOK * kRowsPerCta * 4);           // [N_TOK][128] low-rank term
+    __nv_bfloat16* otile = reinterpret_cast<__nv_bfloat16*>(smem);                     // [N_TOK][128] finished outputs
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * kRowsPerCta;
@@ -155,18 +164,22 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     const bool lowrank = p.r > 0;
     const bool lowrank_here = lowrank && split == 0;   // the low-rank accumulator lives in the first CTA of a cluster
 
+    auto sub_count = [&](int u) { return min(kUnitK / kBlockK, (p.K - u * kUnitK) / kBlockK); };
+    // k-blocks this CTA contracts; every unit but the last of the matrix has eight
+    const int my_blocks = (unit_end - unit_begin - 1) * (kUnitK / kBlockK) + sub_count(unit_end - 1);
+
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        for (int i = 0; i < WS; ++i) { mbar_init(&w_full[i], 1); mbar_init(&w_empty[i], 4); }
-        for (int i = 0; i < BS; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
+        for (int i = 0; i < WS; ++i) { mbar_init(&w_full[i], 1); mbar_init(&w_empty[i], kExpanders / 32); }
+        for (int i = 0; i < BS; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], NISS); }
         for (int i = 0; i < AS; ++i) { mbar_init(&a_full[i], 4); mbar_init(&a_empty[i], 1); }
-        mbar_init(d_full, 1);
-        mbar_init(u_full, 4);
+        mbar_init(d_full, NISS);
+        mbar_init(u_full, kExpanders / 32);
         mbar_init(t_full, 1);
         fence_barrier_init();
         fence_proxy_async();
     }
-    if (warp == 1) {
+    if (warp == 2) {
         tmem_alloc(tmem_base_slot, TMEM_COLS);
         tmem_relinquish();
     }
@@ -176,8 +189,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     const uint32_t tmem_base = *tmem_base_slot;
     // the next kernel of the stream may start its own independent preamble now
     griddep_launch_dependents();
-
-    auto sub_count = [&](int u) { return min(kUnitK / kBlockK, (p.K - u * kUnitK) / kBlockK); };
 
     if (warp == 0) {
         // ---------------- packed sign words: HBM -> shared memory (independent of the preceding kernel) ----------------
@@ -192,8 +203,8 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);   // let copies in flight land
         }
-    } else if (warp == 2) {
-        // ---------------- activation codes and T: L2 -> shared memory ----------------
+    } else if (warp == 1) {
+        // ---------------- T and the activation codes: L2 -> shared memory ----------------
         if (elect_one()) {
             tma_prefetch_desc(&b_map);
             if (lowrank_here) tma_prefetch_desc(&t_map);
@@ -218,38 +229,16 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issue ----------------
-        if (elect_one()) {
+    } else if (warp < 6) {
+        // ---------------- MMA issue: thread `iss` takes k-blocks kb = iss, iss + NISS, ... ----------------
+        const int iss = warp - 2;
+        if (iss < NISS && elect_one()) {
             // instruction descriptors: D = s32, A = s8 (tensor memory, K-major), B = s8 (shared, K-major), M = 128;
             // and D = f32, A = B = bf16 (shared, K-major), M = 128
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc_lr = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
-            int as = 0; uint32_t aph = 0; int bs = 0; uint32_t bph = 0; uint32_t first = 1;
             bool ok = true;
-            for (int u = unit_begin; u < unit_end && ok; ++u) {
-                const int ns = sub_count(u);
-                for (int s = 0; s < ns; ++s) {
-                    const int sb = s % SUBS;
-                    if (sb == 0 && !wait_or_abort(&b_full[bs], bph, abort_flag)) { give_up(p.status, abort_flag, 0x30); ok = false; break; }
-                    if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
-                    const uint32_t a_addr = tmem_base + 2 * L::DCOLS + 32 * as;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        mma_i8_ts(tmem_base, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, first ? 0u : 1u);
-                        first = 0;
-                    }
-                    tc_commit(&a_empty[as]);
-                    if (++as == AS) { as = 0; aph ^= 1; }
-                    if (sb == SUBS - 1 || s == ns - 1) {
-                        tc_commit(&b_empty[bs]);
-                        if (++bs == BS) { bs = 0; bph ^= 1; }
-                    }
-                }
-            }
-            if (ok && lowrank_here) {
+            if (iss == 0 && lowrank_here) {
                 if (!wait_or_abort(u_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x32); ok = false; }
                 if (ok && !wait_or_abort(t_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x33); ok = false; }
                 if (ok) {
@@ -260,8 +249,36 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         const uint32_t t_addr = smem_u32(tbuf + h * L::sub_bytes);
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            mma_f16_ss(tmem_base + L::DCOLS, smem_desc_sw128(u_addr, 32 * i), smem_desc_sw128(t_addr, 32 * i),
+                            mma_f16_ss(tmem_base + L::D2_COL, smem_desc_sw128(u_addr, 32 * i), smem_desc_sw128(t_addr, 32 * i),
                                        idesc_lr, (h | i) ? 1u : 0u);
+                    }
+                }
+            }
+            const uint32_t d_addr = tmem_base + iss * N_TOK;
+            int bs = 0; uint32_t bph = 0; int kb = 0;
+            for (int u = unit_begin; u < unit_end && ok; ++u) {
+                const int ns = sub_count(u);
+                for (int s = 0; s < ns; ++s, ++kb) {
+                    const int sb = s % SUBS;
+                    // every issuing thread sees each code stage filled before it releases it, whether or not one of
+                    // the stage's k-blocks is its own: its release can then never run a whole ring ahead
+                    if (sb == 0 && !wait_or_abort(&b_full[bs], bph, abort_flag)) { give_up(p.status, abort_flag, 0x30); ok = false; break; }
+                    if (kb % NISS == iss) {
+                        const int as = kb % AS;
+                        const uint32_t aph = (uint32_t)(kb / AS) & 1u;
+                        if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
+                        const uint32_t a_addr = tmem_base + L::A_COL + 32 * as;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            mma_i8_ts(d_addr, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, (kb < NISS && i == 0) ? 0u : 1u);
+                        tc_commit(&a_empty[as]);
+                    }
+                    if (sb == SUBS - 1 || s == ns - 1) {
+                        // this thread is done with the code stage once its MMAs so far have completed
+                        tc_commit(&b_empty[bs]);
+                        if (++bs == BS) { bs = 0; bph ^= 1; }
                     }
                 }
             }
@@ -270,15 +287,16 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     } else {
         // ---------------- U tile, expansion of sign bits into tensor memory, then the epilogue ----------------
         const int q = warp & 3;                       // tensor-memory lane quarter this warp may touch
+        const int half = (warp - 6) >> 2;             // which of the two warps of that quarter
         const int row = q * 32 + lane;
-        const int e = threadIdx.x - 96;               // 0..127 among the expander threads
+        const int e = threadIdx.x - kFirstExpander;   // 0..255 among the expander threads
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         if (lowrank_here) {
             // 128 rows x 8 chunks of 16 bytes, 128B-swizzled K-major; rows beyond N and columns beyond r are zero
             const bool vec = (p.r % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.U) & 15) == 0);
 #pragma unroll
-            for (int it = 0; it < 8; ++it) {
-                const int idx = it * 128 + e;
+            for (int it = 0; it < 1024 / kExpanders; ++it) {
+                const int idx = it * kExpanders + e;
                 const int ur = idx >> 3, ch = idx & 7;
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
                 const int n = n0 + ur;
@@ -299,32 +317,60 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(u_full);
         }
-        int ws = 0; uint32_t wph = 0; int as = 0; uint32_t aph = 0;
+        // This warp expands k-blocks kb = half, half + 2, ... of the CTA (stage kb % AS; AS is even).  The store of one
+        // k-block is left in flight while the next one is expanded; `pending` is the stage whose store has not been
+        // waited for and announced yet.
+        int ws = 0; uint32_t wph = 0;
+        int pending = -1;
         bool ok = true;
+        int kb0 = 0;                                   // k-block index of sub-block 0 of the current unit
         for (int u = unit_begin; u < unit_end && ok; ++u) {
             if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&w_full[ws], wph, abort_flag))) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
-            for (int s = 0; s < ns; ++s) {
-                const uint4 w4 = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
-                uint32_t v[32];
-                const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+            const int s_first = (kb0 + half) & 1;      // kb0 + s has the parity of `half`
+            // the sign words of this warp's k-blocks of the unit, loaded together
+            uint4 w4[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[8 * i + j] = (w[i] << (7 - j)) & 0x80808080u;
-                if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&a_empty[as], aph ^ 1, abort_flag))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
-                tc_fence_after();
-                tmem_st_32x32(tmem_base + lane_addr + 2 * L::DCOLS + 32 * as, v);
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[as]);
-                if (++as == AS) { as = 0; aph ^= 1; }
+            for (int i = 0; i < 4; ++i) {
+                const int s = 2 * i + s_first;
+                if (s < ns) w4[i] = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&w_empty[ws]);
+            if (lane == 0) mbar_arrive(&w_empty[ws]);      // the stage is in registers now
             if (++ws == WS) { ws = 0; wph ^= 1; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int s = 2 * i + s_first;
+                if (s >= ns) break;
+                const int kb = kb0 + s;
+                const int as = kb % AS;
+                const uint32_t aph = (uint32_t)(kb / AS) & 1u;
+                uint32_t v[32];
+                const uint32_t w[4] = {w4[i].x, w4[i].y, w4[i].z, w4[i].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
+                if (pending >= 0) {
+                    tc_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&a_full[pending]);
+                    pending = -1;
+                }
+                if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&a_empty[as], aph ^ 1, abort_flag))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
+                tc_fence_after();
+                tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
+                pending = as;
+            }
+            kb0 += ns;
+        }
+        if (pending >= 0) {
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&a_full[pending]);
         }
         // per-token scale and code sum of this tile (written by the preceding kernel)
         griddep_wait();
@@ -333,48 +379,67 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             scale_s[e] = t < p.M ? p.scales[t] : 0.f;
             qsum_s[e] = t < p.M ? p.qsum[t] : 0;
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");     // the four expander warps only
+        asm volatile("bar.sync 1, 256;" ::: "memory");     // the expander warps only
         if (ok) {
             if (!__all_sync(0xFFFFFFFFu, wait_or_abort(d_full, 0, abort_flag))) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
         if (ok) {
             tc_fence_after();
             const int n = n0 + row;
-            if (p.splits == 1) {
-                const float alpha_n = n < p.N ? p.alpha[n] : 0.f;
-                const float mu_n = (p.mu && n < p.N) ? p.mu[n] : 0.f;
+            const int nacc = min(NISS, my_blocks);             // accumulators that hold something
+            const bool single = p.splits == 1;
+            const float alpha_n = n < p.N ? p.alpha[n] : 0.f;
+            const float mu_n = (p.mu && n < p.N) ? p.mu[n] : 0.f;
+            // the two warps of a quarter take alternate chunks of 16 tokens
 #pragma unroll 1
-                for (int c = 0; c < N_TOK / 16; ++c) {
-                    if (t0 + 16 * c >= p.M) break;                 // warp-uniform
-                    uint32_t v[16], l[16];
-                    tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
-                    if (lowrank) tmem_ld_32x16(tmem_base + lane_addr + L::DCOLS + 16 * c, l);
-                    tc_wait_ld();
-                    if (n < p.N) {
+            for (int c = half; c < N_TOK / 16; c += 2) {
+                if (t0 + 16 * c >= p.M) break;                 // warp-uniform
+                uint32_t v[16], l[16];
+                tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
+                if (lowrank_here) tmem_ld_32x16(tmem_base + lane_addr + L::D2_COL + 16 * c, l);
+                tc_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int tt = 16 * c + j;
-                            if (t0 + tt < p.M)
-                                finish_element(p, t0 + tt, n, (int32_t)v[j], lowrank ? __uint_as_float(l[j]) : 0.f,
-                                               scale_s[tt], qsum_s[tt], alpha_n, mu_n);
-                        }
-                    }
-                }
-            } else if (L::can_split) {
-                // partial sums of this K slice -> shared memory, transposed so that a token's 128 rows are contiguous
-#pragma unroll 1
-                for (int c = 0; c < N_TOK / 16; ++c) {
-                    if (t0 + 16 * c >= p.M) break;
-                    uint32_t v[16];
-                    tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) red_i[(16 * c + j) * kRowsPerCta + row] = (int32_t)v[j];
-                    if (lowrank_here) {
-                        tmem_ld_32x16(tmem_base + lane_addr + L::DCOLS + 16 * c, v);
+                for (int a = 1; a < NISS; ++a) {
+                    if (a < nacc) {
+                        uint32_t v2[16];
+                        tmem_ld_32x16(tmem_base + lane_addr + a * N_TOK + 16 * c, v2);
                         tc_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) red_f[(16 * c + j) * kRowsPerCta + row] = __uint_as_float(v[j]);
+                        for (int j = 0; j < 16; ++j) v[j] += v2[j];
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int tt = 16 * c + j;
+                    const int32_t d = (int32_t)v[j];
+                    const float lr = lowrank_here ? __uint_as_float(l[j]) : 0.f;
+                    if (single) {
+                        // finished value -> bf16 tile in shared memory, [token][row]
+                        float y = 0.f;
+                        if (n < p.N && t0 + tt < p.M) y = finish_value(p, t0 + tt, n, d, lr, scale_s[tt], qsum_s[tt], alpha_n, mu_n);
+                        otile[tt * kRowsPerCta + row] = __float2bfloat16_rn(y);
+                    } else if (L::can_split) {
+                        red_i[tt * kRowsPerCta + row] = d;
+                        if (lowrank_here) red_f[tt * kRowsPerCta + row] = lr;
+                    }
+                }
+            }
+        }
+        if (p.splits == 1) {
+            asm volatile("bar.sync 1, 256;" ::: "memory");   // the output tile is complete (all expander warps, always)
+            if (ok && p.out) {
+                // 16 threads move one token's 128 outputs (256 bytes) with 128-bit stores
+                const bool vec = ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) && (p.ldo % 8 == 0) && (n0 + kRowsPerCta <= p.N);
+                for (int tt = e >> 4; tt < N_TOK && t0 + tt < p.M; tt += kExpanders / 16) {
+                    const int c8 = (e & 15) * 8;
+                    __nv_bfloat16* dst = p.out + (int64_t)(t0 + tt) * p.ldo + n0 + c8;
+                    const uint4 val = *reinterpret_cast<const uint4*>(otile + tt * kRowsPerCta + c8);
+                    if (vec) {
+                        *reinterpret_cast<uint4*>(dst) = val;
+                    } else {
+                        const __nv_bfloat16* sv = reinterpret_cast<const __nv_bfloat16*>(&val);
+                        for (int j = 0; j < 8; ++j)
+                            if (n0 + c8 + j < p.N) dst[j] = sv[j];
                     }
                 }
             }
@@ -386,20 +451,43 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         // every thread of every CTA of the cluster takes part, whether or not its CTA gave up
         cluster_arrive_release();
         cluster_wait_acquire();
-        if (L::can_split && warp >= 3 && !*abort_flag) {
-            const int row = (warp & 3) * 32 + lane;
-            const int n = n0 + row;
-            if (n < p.N) {
-                const float alpha_n = p.alpha[n];
-                const float mu_n = p.mu ? p.mu[n] : 0.f;
-                // tokens of the tile are dealt round-robin to the CTAs of the cluster
-                for (int tt = split; tt < N_TOK && t0 + tt < p.M; tt += p.splits) {
-                    const uint32_t off_i = smem_u32(&red_i[tt * kRowsPerCta + row]);
-                    int32_t d = 0;
-                    for (int c = 0; c < p.splits; ++c) d += (int32_t)ld_shared_cluster_u32(map_shared_rank(off_i, c));
-                    float l = 0.f;
-                    if (lowrank) l = __uint_as_float(ld_shared_cluster_u32(map_shared_rank(smem_u32(&red_f[tt * kRowsPerCta + row]), 0)));
-                    finish_element(p, t0 + tt, n, d, l, scale_s[tt], qsum_s[tt], alpha_n, mu_n);
+        if (L::can_split && warp >= 6 && !*abort_flag) {
+            // the tokens of the tile are dealt round-robin to the CTAs of the cluster; a thread sums four consecutive
+            // rows of one token over all CTAs with 128-bit distributed-shared-memory loads
+            const int e = threadIdx.x - kFirstExpander;
+            const int r4 = (e & 31) * 4;
+            const int n = n0 + r4;
+            for (int ti = e >> 5; ; ti += kExpanders / 32) {
+                const int tt = split + ti * p.splits;
+                if (tt >= N_TOK || t0 + tt >= p.M) break;
+                const uint32_t off_i = smem_u32(&red_i[tt * kRowsPerCta + r4]);
+                uint4 part[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    if (c < p.splits) part[c] = ld_shared_cluster_v4(map_shared_rank(off_i, c));
+                uint4 lf = make_uint4(0u, 0u, 0u, 0u);
+                if (lowrank) lf = ld_shared_cluster_v4(map_shared_rank(smem_u32(&red_f[tt * kRowsPerCta + r4]), 0));
+                int32_t d[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    if (c < p.splits) { d[0] += (int32_t)part[c].x; d[1] += (int32_t)part[c].y; d[2] += (int32_t)part[c].z; d[3] += (int32_t)part[c].w; }
+                const float l4[4] = {__uint_as_float(lf.x), __uint_as_float(lf.y), __uint_as_float(lf.z), __uint_as_float(lf.w)};
+                __align__(8) __nv_bfloat16 y4[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float y = 0.f;
+                    if (n + j < p.N)
+                        y = finish_value(p, t0 + tt, n + j, d[j], l4[j], scale_s[tt], qsum_s[tt], p.alpha[n + j], p.mu ? p.mu[n + j] : 0.f);
+                    y4[j] = __float2bfloat16_rn(y);
+                }
+                if (p.out) {
+                    __nv_bfloat16* dst = p.out + (int64_t)(t0 + tt) * p.ldo + n;
+                    if (((reinterpret_cast<uintptr_t>(dst) & 7) == 0) && n + 3 < p.N) {
+                        *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(y4);
+                    } else {
+                        for (int j = 0; j < 4; ++j)
+                            if (n + j < p.N) dst[j] = y4[j];
+                    }
                 }
             }
         }
@@ -407,7 +495,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         cluster_arrive_release();
         cluster_wait_acquire();
     }
-    if (warp == 1) {
+    if (warp == 2) {
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
@@ -447,11 +535,11 @@ static int make_map(CUtensorMap* map, CUtensorMapDataType dt, int rank, const vo
     return BWLA_OK;
 }
 
-template <int N_TOK, int WS, int BS, int TMEM_COLS>
+template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS>
 static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUtensorMap& tm, const UmmaParams& p,
                          dim3 grid, cudaStream_t s) {
-    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS>;
-    auto kernel = umma_w1a_kernel<N_TOK, WS, BS, TMEM_COLS>;
+    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS>;
+    auto kernel = umma_w1a_kernel<N_TOK, WS, BS, TMEM_COLS, NISS>;
     static thread_local int configured = -1;
     int dev = 0;
     BWLA_CUDA_TRY(cudaGetDevice(&dev));
@@ -468,7 +556,7 @@ static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUt
     attrs[0].id = cudaLaunchAttributeClusterDimension;
     attrs[0].val.clusterDim.x = 1; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = grid.z;
     attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    attrs[1].val.programmaticStreamSerializationAllowed = launch_overlap_allowed();
     cfg.attrs = attrs;
     cfg.numAttrs = 2;
     ProfScope prof(kProfContraction, s);
@@ -534,10 +622,10 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
     p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug; p.status = a.status;
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     switch (n_tok) {
-        case 16: return launch_umma_t<16, 3, 2, 256>(wm, bm, tm, p, grid, stream);
-        case 32: return launch_umma_t<32, 3, 2, 256>(wm, bm, tm, p, grid, stream);
-        case 64: return launch_umma_t<64, 2, 2, 256>(wm, bm, tm, p, grid, stream);
-        default: return launch_umma_t<128, 2, 4, 512>(wm, bm, tm, p, grid, stream);
+        case 16: return launch_umma_t<16, 3, 2, 256, 2>(wm, bm, tm, p, grid, stream);
+        case 32: return launch_umma_t<32, 3, 2, 256, 2>(wm, bm, tm, p, grid, stream);
+        case 64: return launch_umma_t<64, 4, 3, 512, 2>(wm, bm, tm, p, grid, stream);
+        default: return launch_umma_t<128, 2, 6, 512, 1>(wm, bm, tm, p, grid, stream);
     }
 }
 

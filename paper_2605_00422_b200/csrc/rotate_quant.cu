@@ -21,6 +21,8 @@
 // overlap the preceding kernel of the stream; every block waits for that kernel before it stores anything.
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "bwla_common.cuh"
 #include "umma_ptx.cuh"
 
@@ -31,6 +33,7 @@ using namespace ptx;
 constexpr int kLrTokens = 16;     // tokens per low-rank block
 constexpr int kLrRows = 2;        // rows of V per low-rank block
 constexpr int kLrMaxWarps = 16;   // blocks have at most 512 threads
+constexpr int kPrologueSmemFloats = 56 * 1024;   // dynamic shared memory of a prologue block, in floats (224 KB)
 
 struct PrologueParams {
     const __nv_bfloat16* x; int64_t M; int K; int64_t ldx;
@@ -41,6 +44,9 @@ struct PrologueParams {
     int rot_blocks;     // M * C
     int row_gran;       // slab boundaries are multiples of this many rows of X
     int slab_cap;       // floats reserved for one slab
+    int ps_cap;         // floats reserved for a staged chunk of P2 / P1
+    int ch1, ch2;       // columns of P2 / of P1 staged at a time
+    int tr1, tr2;       // rows per thread in the two contractions
     // low-rank
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
 };
@@ -69,6 +75,106 @@ __device__ __forceinline__ int slab_begin(int c, int C, int n1, int gran) {
     return (int)(((int64_t)n1 * c / C) / gran * gran);
 }
 
+// Z[rows of this slab][dc .. dc+cw) = X slab * P2[:, dc .. dc+cw).  Ps holds that chunk of P2 (row stride cw).
+// Each thread owns TR rows x 4 columns; the sum runs over b in increasing order.
+template <int TR>
+__device__ __forceinline__ void stage1_chunk(const float* __restrict__ Xs, int rows, int n2, const float* __restrict__ Ps,
+                                             int dc, int cw, float* Zf, int a_lo, int C) {
+    const int ct = cw >> 2;
+    const int tiles = ((rows + TR - 1) / TR) * ct;
+    for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
+        const int mt = tile / ct, dl = (tile - mt * ct) << 2;
+        const int r0 = mt * TR;
+        const float* xr[TR];
+#pragma unroll
+        for (int i = 0; i < TR; ++i) xr[i] = Xs + min(r0 + i, rows - 1) * n2;
+        float acc[TR][4];
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        const float* pp = Ps + dl;
+#pragma unroll 2
+        for (int b = 0; b < n2; b += 4) {
+            float4 xa[TR];
+#pragma unroll
+            for (int i = 0; i < TR; ++i) xa[i] = *reinterpret_cast<const float4*>(xr[i] + b);
+#pragma unroll
+            for (int bb = 0; bb < 4; ++bb) {
+                const float4 pv = *reinterpret_cast<const float4*>(pp + (b + bb) * cw);
+#pragma unroll
+                for (int i = 0; i < TR; ++i) {
+                    const float x = bb == 0 ? xa[i].x : bb == 1 ? xa[i].y : bb == 2 ? xa[i].z : xa[i].w;
+                    acc[i][0] = fmaf(x, pv.x, acc[i][0]);
+                    acc[i][1] = fmaf(x, pv.y, acc[i][1]);
+                    acc[i][2] = fmaf(x, pv.z, acc[i][2]);
+                    acc[i][3] = fmaf(x, pv.w, acc[i][3]);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+            if (r0 + i < rows) {
+                float* dst = Zf + (a_lo + r0 + i) * n2 + dc + dl;
+                const float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                if (C == 1) {
+                    *reinterpret_cast<float4*>(dst) = v;
+                } else {
+                    const uint32_t local = smem_u32(dst);
+                    for (int c = 0; c < C; ++c) st_cluster_v4(map_shared_rank(local, c), v);
+                }
+            }
+    }
+}
+
+// Y[c0 .. c0+cw)[all d] = sum_a P1[a][a_lo + c0 + .] * Z[a][d].  Ps holds P1[:, a_lo+c0 .. a_lo+c0+cw) with row
+// stride cwp (cw rounded up to 4, padding zero).  Each thread owns TR output rows x 4 columns.
+template <int TR>
+__device__ __forceinline__ void stage2_chunk(const float* __restrict__ Zf, int n1, int n2, const float* __restrict__ Ps,
+                                             int cwp, int c0, int cw, float* Ys, float& amax) {
+    const int dt = n2 >> 2;
+    const int tiles = ((cw + TR - 1) / TR) * dt;
+    for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
+        const int mt = tile / dt, d0 = (tile - mt * dt) << 2;
+        const int r0 = mt * TR;
+        float acc[TR][4];
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        const float* zp = Zf + d0;
+        const float* pp = Ps + r0;
+#pragma unroll 4
+        for (int a = 0; a < n1; ++a) {
+            const float4 zv = *reinterpret_cast<const float4*>(zp + a * n2);
+            float pa[TR];
+            if (TR % 4 == 0) {
+#pragma unroll
+                for (int i = 0; i < TR; i += 4) {
+                    const float4 v = *reinterpret_cast<const float4*>(pp + a * cwp + i);
+                    pa[i] = v.x; pa[i + 1] = v.y; pa[i + 2] = v.z; pa[i + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < TR; ++i) pa[i] = pp[a * cwp + min(i, cw - 1 - r0)];
+            }
+#pragma unroll
+            for (int i = 0; i < TR; ++i) {
+                acc[i][0] = fmaf(pa[i], zv.x, acc[i][0]);
+                acc[i][1] = fmaf(pa[i], zv.y, acc[i][1]);
+                acc[i][2] = fmaf(pa[i], zv.z, acc[i][2]);
+                acc[i][3] = fmaf(pa[i], zv.w, acc[i][3]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+            if (r0 + i < cw) {
+                *reinterpret_cast<float4*>(Ys + (c0 + r0 + i) * n2 + d0) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                amax = fmaxf(amax, fmaxf(fmaxf(fabsf(acc[i][0]), fabsf(acc[i][1])), fmaxf(fabsf(acc[i][2]), fabsf(acc[i][3]))));
+            }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // rotation + quantiser
 // ---------------------------------------------------------------------------------------------
@@ -81,7 +187,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     const int rows = a_hi - a_lo;
     float* Xs = smem;                          // this CTA's slab of X, later of Y
     float* Zf = smem + p.slab_cap;             // all of Z
-    float* slots = Zf + K;                     // [0..7] absmax per rank, [8..15] code sum per rank (int)
+    float* slots = Zf + K + p.ps_cap;          // [0..7] absmax per rank, [8..15] code sum per rank (int)
     __shared__ float red_max[32];
     __shared__ int red_sum;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -116,78 +222,40 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
 
     float amax = 0.f;
     if ((n2 & 3) == 0) {
-        const int dt_count = n2 >> 2;
-        const int tiles = ((rows + 3) >> 2) * dt_count;
-        // ---- Z slab = X slab * P2, stored into every CTA's full Z
-        for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
-            const int mt = tile / dt_count, d0 = (tile - mt * dt_count) << 2;
-            const int r0 = mt << 2;
-            const float* xr[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) xr[i] = Xs + min(r0 + i, rows - 1) * n2;
-            float acc[4][4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-            const float* pp = p.P2 + d0;
-#pragma unroll 4
-            for (int b = 0; b < n2; ++b) {
-                const float4 pv = __ldg(reinterpret_cast<const float4*>(pp + (size_t)b * n2));
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float xa = xr[i][b];
-                    acc[i][0] = fmaf(xa, pv.x, acc[i][0]);
-                    acc[i][1] = fmaf(xa, pv.y, acc[i][1]);
-                    acc[i][2] = fmaf(xa, pv.z, acc[i][2]);
-                    acc[i][3] = fmaf(xa, pv.w, acc[i][3]);
-                }
+        float* Ps = Zf + K;                    // staged chunk of P2, later of P1
+        // ---- Z slab = X slab * P2, one chunk of columns of P2 at a time, stored into every CTA's full Z
+        for (int dc = 0; dc < n2; dc += p.ch1) {
+            const int cw = min(p.ch1, n2 - dc);
+            for (int i = threadIdx.x; i < n2 * (cw >> 2); i += blockDim.x) {
+                const int b = i / (cw >> 2), j = (i - b * (cw >> 2)) << 2;
+                *reinterpret_cast<float4*>(Ps + b * cw + j) = __ldg(reinterpret_cast<const float4*>(p.P2 + (size_t)b * n2 + dc + j));
             }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (r0 + i < rows) {
-                    float* dst = Zf + (a_lo + r0 + i) * n2 + d0;
-                    const float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                    if (C == 1) {
-                        *reinterpret_cast<float4*>(dst) = v;
-                    } else {
-                        const uint32_t local = smem_u32(dst);
-                        for (int c = 0; c < C; ++c) st_cluster_v4(map_shared_rank(local, c), v);
-                    }
-                }
+            __syncthreads();
+            switch (p.tr1) {
+                case 8: stage1_chunk<8>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
+                case 4: stage1_chunk<4>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
+                case 2: stage1_chunk<2>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
+                default: stage1_chunk<1>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
+            }
+            __syncthreads();
         }
-        if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
-        // ---- Y slab = (P1^T * Z) rows [a_lo, a_hi); Y overwrites the X slab, which is dead now
-        for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
-            const int mt = tile / dt_count, d0 = (tile - mt * dt_count) << 2;
-            const int r0 = mt << 2;
-            int cc[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) cc[i] = a_lo + min(r0 + i, rows - 1);
-            float acc[4][4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-#pragma unroll 4
-            for (int a = 0; a < n1; ++a) {
-                const float4 zv = *reinterpret_cast<const float4*>(Zf + a * n2 + d0);
-                const float* prow = p.P1 + (size_t)a * n1;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float pa = __ldg(prow + cc[i]);
-                    acc[i][0] = fmaf(pa, zv.x, acc[i][0]);
-                    acc[i][1] = fmaf(pa, zv.y, acc[i][1]);
-                    acc[i][2] = fmaf(pa, zv.z, acc[i][2]);
-                    acc[i][3] = fmaf(pa, zv.w, acc[i][3]);
-                }
+        if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); }
+        // ---- Y slab = (P1^T * Z) rows [a_lo, a_hi), one chunk of output rows (columns of P1) at a time;
+        //      Y overwrites the X slab, which is dead now
+        for (int c0 = 0; c0 < rows; c0 += p.ch2) {
+            const int cw = min(p.ch2, rows - c0), cwp = (cw + 3) & ~3;
+            for (int i = threadIdx.x; i < n1 * cwp; i += blockDim.x) {
+                const int a = i / cwp, j = i - a * cwp;
+                Ps[i] = j < cw ? __ldg(p.P1 + (size_t)a * n1 + a_lo + c0 + j) : 0.f;
             }
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (r0 + i < rows) {
-                    *reinterpret_cast<float4*>(Xs + (r0 + i) * n2 + d0) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                    amax = fmaxf(amax, fmaxf(fmaxf(fabsf(acc[i][0]), fabsf(acc[i][1])), fmaxf(fabsf(acc[i][2]), fabsf(acc[i][3]))));
-                }
+            __syncthreads();
+            switch (p.tr2) {
+                case 8: stage2_chunk<8>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
+                case 4: stage2_chunk<4>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
+                case 2: stage2_chunk<2>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
+                default: stage2_chunk<1>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
+            }
+            __syncthreads();
         }
     } else {
         // generic shapes (n2 not a multiple of 4; C == 1): one output per thread step
@@ -410,9 +478,35 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
             cap = cap > (hi - lo) ? cap : (hi - lo);
         }
         p.C = C; p.rot_blocks = (int)(M * C); p.row_gran = gran; p.slab_cap = (cap * n2 + 3) / 4 * 4;
-        smem = ((size_t)p.slab_cap + (size_t)K + 16) * 4;
-        const int tiles = ((cap + 3) / 4) * (n2 / 4 > 0 ? n2 / 4 : 1);
-        threads = (n2 & 3) ? 256 : (tiles > 384 ? 512 : (tiles > 192 ? 384 : 256));
+        if ((n2 & 3) == 0) {
+            // chunks of P2 (ch1 columns) and of P1 (ch2 columns) that fit beside the X slab and Z
+            const int64_t avail = kPrologueSmemFloats - p.slab_cap - K - 16 - 8;
+            const int max1 = (int)std::min<int64_t>(n2, avail / n2 / 4 * 4);
+            const int max2 = (int)std::min<int64_t>((cap + 3) / 4 * 4, avail / n1 / 4 * 4);
+            if (max1 < 4 || max2 < 4) return BWLA_ERR_INVALID_ARG;
+            // equal chunks rather than full ones and a sliver
+            const int nch1 = (n2 + max1 - 1) / max1, nch2 = (cap + max2 - 1) / max2;
+            const int ch1 = ((n2 + nch1 - 1) / nch1 + 3) / 4 * 4;
+            const int ch2 = std::min(cap, ((cap + nch2 - 1) / nch2 + 3) / 4 * 4);
+            p.ch1 = ch1; p.ch2 = ch2;
+            p.ps_cap = std::max(n2 * ch1, n1 * ((ch2 + 3) / 4 * 4)) + 8;
+            // rows per thread: as many as still leave a few hundred tiles
+            auto pick = [](int rows, int cols4) {
+                for (int tr = 8; tr > 1; tr >>= 1)
+                    if (((rows + tr - 1) / tr) * cols4 >= 256) return tr;
+                return 1;
+            };
+            p.tr1 = pick(cap, ch1 / 4);
+            p.tr2 = pick(ch2, n2 / 4);
+            const int tiles = std::max(((cap + p.tr1 - 1) / p.tr1) * (ch1 / 4), ((ch2 + p.tr2 - 1) / p.tr2) * (n2 / 4));
+            const int rounds = (tiles + 511) / 512;
+            threads = ((tiles + rounds - 1) / rounds + 31) / 32 * 32;
+            threads = threads < 128 ? 128 : (threads > 512 ? 512 : threads);
+        } else {
+            p.ps_cap = 0; p.ch1 = p.ch2 = 4; p.tr1 = p.tr2 = 1;
+            threads = 256;
+        }
+        smem = ((size_t)p.slab_cap + (size_t)K + (size_t)p.ps_cap + 16) * 4;
     } else {
         p.C = 1; p.rot_blocks = 0;
     }
@@ -428,7 +522,7 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     int dev = 0;
     BWLA_CUDA_TRY(cudaGetDevice(&dev));
     if (configured_device != dev) {
-        BWLA_CUDA_TRY(cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 25600 * 8 + 64));
+        BWLA_CUDA_TRY(cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrologueSmemFloats * 4));
         configured_device = dev;
     }
     cudaLaunchConfig_t cfg{};
@@ -440,7 +534,7 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     attrs[0].id = cudaLaunchAttributeClusterDimension;
     attrs[0].val.clusterDim.x = (unsigned)C; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
     attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    attrs[1].val.programmaticStreamSerializationAllowed = launch_overlap_allowed();
     cfg.attrs = attrs;
     cfg.numAttrs = 2;
     ProfScope prof(kProfRotateQuant, stream);
