@@ -56,7 +56,11 @@ struct ProfScope {
 // ---------------------------------------------------------------------------------------------
 // workspace layout (byte offsets into the caller's scratch buffer; every section 256-byte aligned)
 // ---------------------------------------------------------------------------------------------
+#ifdef BWLA_TRACE
+constexpr int kStatusBytes = 8192;       // tuning builds keep a timeline behind the status words
+#else
 constexpr int kStatusBytes = 256;        // word 0: status; words 1..: where a bounded wait gave up
+#endif
 constexpr int kLowrankPad = 64;          // T is kept as bf16 [3][M][64] (T = hi + mid + lo), zero beyond r <= 64
 
 __host__ __device__ inline int lowrank_cols(int r) { return r > kLowrankPad ? (r + 1) / 2 * 2 : kLowrankPad; }

@@ -13,17 +13,17 @@
 //     (programmatic dependent launch);
 //   * warp 1 waits for the preceding kernel, then streams the three bf16 terms of T and the activation codes
 //     (tokens x 128 bytes per k-block, the canonical K-major 128B-swizzled UMMA layout);
-//   * warps 6..13 (two per tensor-memory lane quarter, thread = output row, the two warps of a quarter taking
+//   * warps 4..11 (two per tensor-memory lane quarter, thread = output row, the two warps of a quarter taking
 //     alternate k-blocks) stage the U tile in shared memory, then turn each 32-bit sign word into eight registers
 //     of four int8 with one shift and one mask per register ((w << (7-j)) & 0x80808080) and write them with
 //     tcgen05.st into tensor memory, where they are the A operand: expanded weights never touch shared memory.
 //     A warp expands its next k-block while the store of the previous one completes;
-//   * NISS threads (one each in warps 2..5) issue tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor
+//   * NISS threads (one each in warps 2 and 3) issue tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor
 //     memory, B from shared memory), taking k-blocks round-robin, each into an int32 accumulator of its own in
 //     tensor memory: with few tokens an MMA is short and the issue latency of one thread would be the bottleneck.
 //     The first of them also issues the kind::f16 MMAs of the low-rank term (A = U tile, B = T as three bf16
 //     terms, fp32 accumulator in tensor memory);
-//   * warps 6..13 read the accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
+//   * warps 4..11 read the accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
 //     scales, transpose through shared memory and store bf16 with 128-bit stores.
 // The shift-and-mask expansion meets the weights of a 32-group in the order k = j + 8*i (register j, byte i), so the
 // codes are stored in that interleaved order by the quantiser.
@@ -42,7 +42,7 @@ using namespace ptx;
 constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
 constexpr int kBlockK = 128;             // K per code sub-block / per tensor-memory A stage
-constexpr int kFirstExpander = 192;      // warps 0, 1: TMA; warps 2..5: MMA issue; warps 6..13: expand + epilogue
+constexpr int kFirstExpander = 128;      // warps 0, 1: TMA; warps 2, 3: MMA issue; warps 4..11: expand + epilogue
 constexpr int kExpanders = 256;
 constexpr int kThreads = kFirstExpander + kExpanders;
 constexpr uint32_t kWaitLimit = 1u << 20;   // polls per wait before giving up (tens of milliseconds)
@@ -90,10 +90,18 @@ struct UmmaCfg {
     static constexpr int total = used + 1024;                          // + slack for 1024-byte alignment
     static constexpr int red_bytes = 2 * N_TOK * kRowsPerCta * 4;
     static constexpr bool can_split = red_bytes <= u_off;
-    static_assert(NISS >= 1 && NISS <= 4, "one to four issuing warps");
+    static_assert(NISS >= 1 && NISS <= 2, "one or two issuing warps");
     static_assert(AS >= 2, "tensor memory: no room for the expanded-weight ring");
     static_assert(N_TOK * kRowsPerCta * 2 <= u_off, "output tile does not fit the stage memory");
 };
+
+// Optional timeline of CTA (0,0,0) for tuning: clock64 stamps behind the status words (compiled out by default).
+#ifdef BWLA_TRACE
+#define BWLA_STAMP(i) do { if (p.status && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
+        reinterpret_cast<long long*>(p.status + 16)[i] = clock64(); } while (0)
+#else
+#define BWLA_STAMP(i) do { } while (0)
+#endif
 
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
     if (status) {
@@ -104,8 +112,9 @@ __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_fl
     *abort_flag = 1;
 }
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t* polls = nullptr) {
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (polls) *polls = i;
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (i > 8192) __nanosleep(64);             // a sleeping warp wakes up late: only back off on long waits
@@ -124,7 +133,7 @@ __device__ __forceinline__ float finish_value(const UmmaParams& p, int64_t t, in
 }
 
 template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, TMEM_COLS == 256 ? 2 : 1)
 umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map,
                 const __grid_constant__ CUtensorMap t_map, UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -163,6 +172,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     const int unit_end = (int)(((int64_t)(split + 1) * p.total_units) / p.splits);
     const bool lowrank = p.r > 0;
     const bool lowrank_here = lowrank && split == 0;   // the low-rank accumulator lives in the first CTA of a cluster
+    if (threadIdx.x == 0) BWLA_STAMP(0);
 
     auto sub_count = [&](int u) { return min(kUnitK / kBlockK, (p.K - u * kUnitK) / kBlockK); };
     // k-blocks this CTA contracts; every unit but the last of the matrix has eight
@@ -229,7 +239,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);
         }
-    } else if (warp < 6) {
+    } else if (warp < 4) {
         // ---------------- MMA issue: thread `iss` takes k-blocks kb = iss, iss + NISS, ... ----------------
         const int iss = warp - 2;
         if (iss < NISS && elect_one()) {
@@ -267,6 +277,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         const int as = kb % AS;
                         const uint32_t aph = (uint32_t)(kb / AS) & 1u;
                         if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
+                        if (kb < 96) BWLA_STAMP(32 + kb);
                         tc_fence_after();
                         const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
                         const uint32_t a_addr = tmem_base + L::A_COL + 32 * as;
@@ -274,6 +285,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         for (int i = 0; i < 4; ++i)
                             mma_i8_ts(d_addr, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, (kb < NISS && i == 0) ? 0u : 1u);
                         tc_commit(&a_empty[as]);
+                        if (kb < 96) BWLA_STAMP(416 + kb);
                     }
                     if (sb == SUBS - 1 || s == ns - 1) {
                         // this thread is done with the code stage once its MMAs so far have completed
@@ -287,7 +299,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     } else {
         // ---------------- U tile, expansion of sign bits into tensor memory, then the epilogue ----------------
         const int q = warp & 3;                       // tensor-memory lane quarter this warp may touch
-        const int half = (warp - 6) >> 2;             // which of the two warps of that quarter
+        const int half = (warp - 4) >> 2;             // which of the two warps of that quarter
         const int row = q * 32 + lane;
         const int e = threadIdx.x - kFirstExpander;   // 0..255 among the expander threads
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
@@ -346,6 +358,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 const int kb = kb0 + s;
                 const int as = kb % AS;
                 const uint32_t aph = (uint32_t)(kb / AS) & 1u;
+                if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(800 + kb);
                 uint32_t v[32];
                 const uint32_t w[4] = {w4[i].x, w4[i].y, w4[i].z, w4[i].w};
 #pragma unroll
@@ -353,15 +366,26 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
                 if (pending >= 0) {
+                    if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(896 + kb);
                     tc_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&a_full[pending]);
+                    if (kb < 98 && (e == 64 || e == 192)) BWLA_STAMP(320 + kb - 2);
+                    if (kb < 98 && (e == 0 || e == 128)) BWLA_STAMP(512 + kb - 2);
+                    if (kb < 98 && (e == 32 || e == 160)) BWLA_STAMP(608 + kb - 2);
+                    if (kb < 98 && (e == 96 || e == 224)) BWLA_STAMP(704 + kb - 2);
                     pending = -1;
                 }
-                if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&a_empty[as], aph ^ 1, abort_flag))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
+                uint32_t polls = 0;
+                if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&a_empty[as], aph ^ 1, abort_flag, &polls))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
+                if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(128 + kb);
+#ifdef BWLA_TRACE
+                if (kb < 96 && (e == 64 || e == 192) && p.status && blockIdx.x == 0 && blockIdx.z == 0) reinterpret_cast<long long*>(p.status + 16)[800 + kb] = polls;
+#endif
                 tc_fence_after();
                 tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
+                if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(224 + kb);
                 pending = as;
             }
             kb0 += ns;
@@ -372,6 +396,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(&a_full[pending]);
         }
+        if (e == 64) BWLA_STAMP(4);
         // per-token scale and code sum of this tile (written by the preceding kernel)
         griddep_wait();
         if (e < N_TOK) {
@@ -383,6 +408,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         if (ok) {
             if (!__all_sync(0xFFFFFFFFu, wait_or_abort(d_full, 0, abort_flag))) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
+        if (e == 64) BWLA_STAMP(5);
         if (ok) {
             tc_fence_after();
             const int n = n0 + row;
@@ -445,13 +471,14 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
         }
     }
+    if (threadIdx.x == kFirstExpander) BWLA_STAMP(6);
     tc_fence_before();
     __syncthreads();
     if (p.splits > 1) {
         // every thread of every CTA of the cluster takes part, whether or not its CTA gave up
         cluster_arrive_release();
         cluster_wait_acquire();
-        if (L::can_split && warp >= 6 && !*abort_flag) {
+        if (L::can_split && warp >= 4 && !*abort_flag) {
             // the tokens of the tile are dealt round-robin to the CTAs of the cluster; a thread sums four consecutive
             // rows of one token over all CTAs with 128-bit distributed-shared-memory loads
             const int e = threadIdx.x - kFirstExpander;
@@ -499,6 +526,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
+        if (lane == 0) BWLA_STAMP(7);
     }
 }
 
