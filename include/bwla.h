@@ -38,7 +38,8 @@ enum {
     BWLA_ERR_UNSUPPORTED = -2,     /* no sm_100 device is current */
     BWLA_ERR_WORKSPACE = -3,       /* workspace NULL, misaligned (256 B) or smaller than bwla_workspace_bytes */
     BWLA_ERR_CUDA = -4,            /* a CUDA call failed; see bwla_last_cuda_error */
-    BWLA_ERR_DEVICE_TIMEOUT = -5   /* a bounded device-side wait ran out (only from bwla_check_status) */
+    BWLA_ERR_DEVICE_TIMEOUT = -5,  /* a bounded device-side wait ran out (only from bwla_check_status) */
+    BWLA_ERR_STATIC_SCRATCH = -6   /* bwla_w1ax_linear_static: the problem needs more scratch than the built-in array holds */
 };
 
 /* Kernel families the layer can run its contraction on (see bwla_force_path). */
@@ -101,6 +102,37 @@ int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
                      const void* U_bf16, const void* V_bf16, int r,
                      void* out_bf16, int64_t N, int64_t ldo,
                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The whole layer without a workspace argument, for callers that cannot allocate.  (The paper has no counterpart:
+ * it describes no kernels and no memory management; this entry point exists for integration only.)
+ *
+ * Who needs it: code that is handed its input and output tensors and nothing else -- a plug-in or custom-op slot
+ * of a host framework, a stage that runs after the framework has frozen its memory pool, a serving process that
+ * may not call cudaMalloc once traffic flows.  Such a caller cannot supply the scratch buffer bwla_w1ax_linear
+ * wants, so here the scratch is a fixed array of BWLA_STATIC_SCRATCH_BYTES inside the library's device image.
+ * Every GPU that loads the library holds that array until the process exits.
+ *
+ * Arguments, layouts and results are those of bwla_w1ax_linear (same kernels, same arithmetic); the workspace
+ * pair is gone.  The call allocates and frees nothing, through CUDA or any other library.
+ *   - Limit: bwla_workspace_bytes(M,K,N,r,bits) must not exceed BWLA_STATIC_SCRATCH_BYTES (4 MiB: e.g. 64 tokens
+ *     at K = 25600, or 512 tokens at K = 5120).  Larger problems return BWLA_ERR_STATIC_SCRATCH and launch nothing.
+ *   - The first call on each device looks up the array's device address (a host-side runtime query).  Make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps what the last call left in it.  The entry point
+ *     clears the status words itself at the start of every call; nothing else needs to start at zero.  Two calls
+ *     that may overlap on the GPU (different streams, or the same stream from two host threads without ordering)
+ *     race on the array and give wrong results: order them.
+ *   - The status word of the built-in array is not exposed: a device-side wait that runs out leaves this call's
+ *     outputs invalid and the next call starts clean.  Use bwla_w1ax_linear with bwla_check_status where that
+ *     must be observed.
+ */
+#define BWLA_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int bwla_w1ax_linear_static(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
+                            const float* P1, int n1, const float* P2, int n2, int bits,
+                            const uint32_t* packed, const float* alpha, const float* mu,
+                            const void* U_bf16, const void* V_bf16, int r,
+                            void* out_bf16, int64_t N, int64_t ldo, void* stream);
 
 /*
  * Contraction + epilogue from given codes (the part of the layer after the quantiser), so that

@@ -240,6 +240,7 @@ const char* bwla_status_string(int status) {
         case BWLA_ERR_WORKSPACE: return "BWLA_ERR_WORKSPACE";
         case BWLA_ERR_CUDA: return "BWLA_ERR_CUDA";
         case BWLA_ERR_DEVICE_TIMEOUT: return "BWLA_ERR_DEVICE_TIMEOUT";
+        case BWLA_ERR_STATIC_SCRATCH: return "BWLA_ERR_STATIC_SCRATCH";
         default: return "BWLA_ERR_UNKNOWN";
     }
 }
