@@ -17,7 +17,6 @@
 //     alternate k-blocks) stage the U tile in shared memory, then turn each 32-bit sign word into eight registers
 //     of four int8 with one shift and one mask per register ((w << (7-j)) & 0x80808080) and write them with
 //     tcgen05.st into tensor memory, where they are the A operand: expanded weights never touch shared memory.
-//     A warp expands its next k-block while the store of the previous one completes;
 //   * NISS threads (one each in warps 2 and 3) issue tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor
 //     memory, B from shared memory), taking k-blocks round-robin, each into an int32 accumulator of its own in
 //     tensor memory: with few tokens an MMA is short and the issue latency of one thread would be the bottleneck.
@@ -60,6 +59,9 @@ struct UmmaParams {
     int64_t ldo;
     int32_t* acc_debug;          // [M][N] or NULL
     uint32_t* status;
+#ifdef BWLA_TRACE
+    const uint32_t* packed_dbg;  // tuning builds compare what the expanders read from shared memory with global memory
+#endif
 };
 
 // Shared-memory and tensor-memory budget of one CTA.
@@ -95,6 +97,11 @@ struct UmmaCfg {
     static_assert(N_TOK * kRowsPerCta * 2 <= u_off, "output tile does not fit the stage memory");
 };
 
+#ifdef BWLA_TRACE
+__device__ uint32_t* g_xor_dbg = nullptr;   // [N][2]: XOR of the sign words each expander thread read from shared memory
+extern "C" int bwla_trace_set_xor_buffer(void* p) { return cudaMemcpyToSymbol(g_xor_dbg, &p, sizeof(p)) == cudaSuccess ? 0 : -4; }
+#endif
+
 // Optional timeline of CTA (0,0,0) for tuning: clock64 stamps behind the status words (compiled out by default).
 #ifdef BWLA_TRACE
 #define BWLA_STAMP(i) do { if (p.status && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
@@ -120,6 +127,17 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
         if (i > 8192) __nanosleep(64);             // a sleeping warp wakes up late: only back off on long waits
     }
     return false;
+}
+
+// A whole warp waits on a barrier: lane 0 polls, the result is broadcast and the warp leaves the call converged, as the
+// .sync.aligned tcgen05 instructions that follow such a wait require (lanes that each ran their own polling loop may
+// come out of it at different times, and a warp-wide tensor-memory store issued by part of a warp lands late).
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
+    int ok = 1;
+    if (lane == 0) ok = wait_or_abort(bar, parity, abort_flag) ? 1 : 0;
+    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+    __syncwarp();
+    return ok != 0;
 }
 
 // One output value from its two accumulators.
@@ -329,15 +347,17 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(u_full);
         }
-        // This warp expands k-blocks kb = half, half + 2, ... of the CTA (stage kb % AS; AS is even).  The store of one
-        // k-block is left in flight while the next one is expanded; `pending` is the stage whose store has not been
-        // waited for and announced yet.
+        // This warp expands k-blocks kb = half, half + 2, ... of the CTA (stage kb % AS; AS is even).  tcgen05.st reads
+        // its source registers asynchronously, so they are left alone until tcgen05.wait::st has returned; the other
+        // warp of the quarter and the second CTA of the SM fill the store's latency.
         int ws = 0; uint32_t wph = 0;
-        int pending = -1;
         bool ok = true;
         int kb0 = 0;                                   // k-block index of sub-block 0 of the current unit
+#ifdef BWLA_TRACE
+        uint32_t xor_dbg = 0;
+#endif
         for (int u = unit_begin; u < unit_end && ok; ++u) {
-            if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&w_full[ws], wph, abort_flag))) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
+            if (!warp_wait(&w_full[ws], wph, abort_flag, lane)) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
             const int s_first = (kb0 + half) & 1;      // kb0 + s has the parity of `half`
@@ -348,9 +368,11 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 const int s = 2 * i + s_first;
                 if (s < ns) w4[i] = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&w_empty[ws]);      // the stage is in registers now
-            if (++ws == WS) { ws = 0; wph ^= 1; }
+#ifdef BWLA_TRACE
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (2 * i + s_first < ns) xor_dbg ^= w4[i].x ^ w4[i].y ^ w4[i].z ^ w4[i].w;
+#endif
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int s = 2 * i + s_first;
@@ -358,44 +380,30 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 const int kb = kb0 + s;
                 const int as = kb % AS;
                 const uint32_t aph = (uint32_t)(kb / AS) & 1u;
-                if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(800 + kb);
                 uint32_t v[32];
                 const uint32_t w[4] = {w4[i].x, w4[i].y, w4[i].z, w4[i].w};
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
-                if (pending >= 0) {
-                    if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(896 + kb);
-                    tc_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&a_full[pending]);
-                    if (kb < 98 && (e == 64 || e == 192)) BWLA_STAMP(320 + kb - 2);
-                    if (kb < 98 && (e == 0 || e == 128)) BWLA_STAMP(512 + kb - 2);
-                    if (kb < 98 && (e == 32 || e == 160)) BWLA_STAMP(608 + kb - 2);
-                    if (kb < 98 && (e == 96 || e == 224)) BWLA_STAMP(704 + kb - 2);
-                    pending = -1;
-                }
-                uint32_t polls = 0;
-                if (!__all_sync(0xFFFFFFFFu, wait_or_abort(&a_empty[as], aph ^ 1, abort_flag, &polls))) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
-                if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(128 + kb);
-#ifdef BWLA_TRACE
-                if (kb < 96 && (e == 64 || e == 192) && p.status && blockIdx.x == 0 && blockIdx.z == 0) reinterpret_cast<long long*>(p.status + 16)[800 + kb] = polls;
-#endif
+                if (!warp_wait(&a_empty[as], aph ^ 1, abort_flag, lane)) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
                 tc_fence_after();
                 tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
-                if (kb < 96 && (e == 64 || e == 192)) BWLA_STAMP(224 + kb);
-                pending = as;
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&a_full[as]);
             }
+            // The stage is released only here, after every word loaded from it has gone through the expansion: an
+            // arrive placed right behind the loads let the copy of a later unit overwrite words not yet read.
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&w_empty[ws]);
+            if (++ws == WS) { ws = 0; wph ^= 1; }
             kb0 += ns;
         }
-        if (pending >= 0) {
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&a_full[pending]);
-        }
+#ifdef BWLA_TRACE
+        if (g_xor_dbg && n0 + row < p.N) g_xor_dbg[(int64_t)(n0 + row) * 2 + half] = xor_dbg;
+#endif
         if (e == 64) BWLA_STAMP(4);
         // per-token scale and code sum of this tile (written by the preceding kernel)
         griddep_wait();
@@ -406,7 +414,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");     // the expander warps only
         if (ok) {
-            if (!__all_sync(0xFFFFFFFFu, wait_or_abort(d_full, 0, abort_flag))) { give_up(p.status, abort_flag, 0x50); ok = false; }
+            if (!warp_wait(d_full, 0, abort_flag, lane)) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
         if (e == 64) BWLA_STAMP(5);
         if (ok) {
@@ -648,9 +656,15 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
     p.M = M; p.N = N; p.K = K; p.total_units = units; p.splits = split; p.r = a.r;
     p.scales = a.scales; p.qsum = a.qsum; p.alpha = a.alpha; p.mu = a.mu; p.U = (const __nv_bfloat16*)a.U;
     p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug; p.status = a.status;
+#ifdef BWLA_TRACE
+    p.packed_dbg = a.packed;
+#endif
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     switch (n_tok) {
-        case 16: return launch_umma_t<16, 3, 2, 256, 2>(wm, bm, tm, p, grid, stream);
+        #ifndef BWLA_DBG_NISS
+#define BWLA_DBG_NISS 2
+#endif
+        case 16: return launch_umma_t<16, 3, 2, 256, BWLA_DBG_NISS>(wm, bm, tm, p, grid, stream);
         case 32: return launch_umma_t<32, 3, 2, 256, 2>(wm, bm, tm, p, grid, stream);
         case 64: return launch_umma_t<64, 4, 3, 512, 2>(wm, bm, tm, p, grid, stream);
         default: return launch_umma_t<128, 2, 6, 512, 1>(wm, bm, tm, p, grid, stream);

@@ -35,6 +35,17 @@ constexpr int kLrRows = 2;        // rows of V per low-rank block
 constexpr int kLrMaxWarps = 16;   // blocks have at most 512 threads
 constexpr int kPrologueSmemFloats = 56 * 1024;   // dynamic shared memory of a prologue block, in floats (224 KB)
 
+// Optional phase timeline of rotation block 0 for tuning (compiled out by default).
+#ifdef BWLA_TRACE
+__device__ long long g_prologue_trace[32];
+#define BWLA_PSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_prologue_trace[i] = clock64(); } while (0)
+extern "C" int bwla_trace_prologue(long long* host32) {
+    return cudaMemcpyFromSymbol(host32, g_prologue_trace, sizeof(long long) * 32) == cudaSuccess ? 0 : -4;
+}
+#else
+#define BWLA_PSTAMP(i) do { } while (0)
+#endif
+
 struct PrologueParams {
     const __nv_bfloat16* x; int64_t M; int K; int64_t ldx;
     // rotation + quantiser (rot_blocks == 0 skips them)
@@ -46,6 +57,8 @@ struct PrologueParams {
     int slab_cap;       // floats reserved for one slab
     int ps_cap;         // floats reserved for a staged chunk of P2 / P1
     int ch1, ch2;       // columns of P2 / of P1 staged at a time
+    int prefetch;       // 1: all of P2 and this CTA's columns of P1 are fetched at the start, with x
+    int p1_cap;         // floats reserved for the prefetched columns of P1
     int tr1, tr2;       // rows per thread in the two contractions
     // low-rank
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
@@ -187,12 +200,14 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     const int rows = a_hi - a_lo;
     float* Xs = smem;                          // this CTA's slab of X, later of Y
     float* Zf = smem + p.slab_cap;             // all of Z
-    float* slots = Zf + K + p.ps_cap;          // [0..7] absmax per rank, [8..15] code sum per rank (int)
+    float* P1s = Zf + K + p.ps_cap;            // this CTA's columns of P1 when they are prefetched
+    float* slots = P1s + p.p1_cap;             // [0..7] absmax per rank, [8..15] code sum per rank (int)
     __shared__ float red_max[32];
     __shared__ int red_sum;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int qmax = (1 << (p.bits - 1)) - 1;
 
+    BWLA_PSTAMP(0);
     // ---- this slab of x_t -> fp32 in shared memory
     {
         const __nv_bfloat16* xt = p.x + t * p.ldx + (int64_t)a_lo * n2;
@@ -215,10 +230,22 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             for (int k = threadIdx.x; k < len; k += blockDim.x) Xs[k] = __bfloat162float(xt[k]);
         }
     }
+    if (p.prefetch) {
+        // one round trip for everything this block reads: P2 and the needed columns of P1 are requested with x
+        float* Ps = Zf + K;
+        for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x)
+            *reinterpret_cast<float4*>(Ps + 4 * i) = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
+        const int cwp = (rows + 3) & ~3;
+        for (int i = threadIdx.x; i < n1 * cwp; i += blockDim.x) {
+            const int a = i / cwp, j = i - a * cwp;
+            P1s[i] = j < rows ? __ldg(p.P1 + (size_t)a * n1 + a_lo + j) : 0.f;
+        }
+    }
     if (threadIdx.x == 0) red_sum = 0;
     // every CTA of the cluster must be running before its shared memory is written from outside
     if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
     griddep_launch_dependents();
+    BWLA_PSTAMP(1);
 
     float amax = 0.f;
     if ((n2 & 3) == 0) {
@@ -226,11 +253,12 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         // ---- Z slab = X slab * P2, one chunk of columns of P2 at a time, stored into every CTA's full Z
         for (int dc = 0; dc < n2; dc += p.ch1) {
             const int cw = min(p.ch1, n2 - dc);
-            for (int i = threadIdx.x; i < n2 * (cw >> 2); i += blockDim.x) {
+            if (!p.prefetch) for (int i = threadIdx.x; i < n2 * (cw >> 2); i += blockDim.x) {
                 const int b = i / (cw >> 2), j = (i - b * (cw >> 2)) << 2;
                 *reinterpret_cast<float4*>(Ps + b * cw + j) = __ldg(reinterpret_cast<const float4*>(p.P2 + (size_t)b * n2 + dc + j));
             }
             __syncthreads();
+            BWLA_PSTAMP(2);
             switch (p.tr1) {
                 case 8: stage1_chunk<8>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
                 case 4: stage1_chunk<4>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
@@ -239,21 +267,25 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             }
             __syncthreads();
         }
+        BWLA_PSTAMP(3);
         if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); }
+        BWLA_PSTAMP(4);
         // ---- Y slab = (P1^T * Z) rows [a_lo, a_hi), one chunk of output rows (columns of P1) at a time;
         //      Y overwrites the X slab, which is dead now
         for (int c0 = 0; c0 < rows; c0 += p.ch2) {
             const int cw = min(p.ch2, rows - c0), cwp = (cw + 3) & ~3;
-            for (int i = threadIdx.x; i < n1 * cwp; i += blockDim.x) {
+            const float* Pc = p.prefetch ? P1s : Ps;
+            if (!p.prefetch) for (int i = threadIdx.x; i < n1 * cwp; i += blockDim.x) {
                 const int a = i / cwp, j = i - a * cwp;
                 Ps[i] = j < cw ? __ldg(p.P1 + (size_t)a * n1 + a_lo + c0 + j) : 0.f;
             }
             __syncthreads();
+            BWLA_PSTAMP(5);
             switch (p.tr2) {
-                case 8: stage2_chunk<8>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
-                case 4: stage2_chunk<4>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
-                case 2: stage2_chunk<2>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
-                default: stage2_chunk<1>(Zf, n1, n2, Ps, cwp, c0, cw, Xs, amax); break;
+                case 8: stage2_chunk<8>(Zf, n1, n2, Pc, cwp, c0, cw, Xs, amax); break;
+                case 4: stage2_chunk<4>(Zf, n1, n2, Pc, cwp, c0, cw, Xs, amax); break;
+                case 2: stage2_chunk<2>(Zf, n1, n2, Pc, cwp, c0, cw, Xs, amax); break;
+                default: stage2_chunk<1>(Zf, n1, n2, Pc, cwp, c0, cw, Xs, amax); break;
             }
             __syncthreads();
         }
@@ -274,6 +306,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             amax = fmaxf(amax, fabsf(s));
         }
     }
+    BWLA_PSTAMP(6);
     // ---- absmax over the block, then over the cluster
     amax = warp_max(amax);
     if (lane == 0) red_max[warp] = amax;
@@ -292,8 +325,10 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     if (amax == 0.f) { inv = 0.f; scale = 1.f; }
     else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
 
+    BWLA_PSTAMP(7);
     // nothing is stored to global memory before the preceding kernel of the stream has completed
     griddep_wait();
+    BWLA_PSTAMP(8);
 
     int local_sum = 0;
     int8_t* ct = p.codes + t * (int64_t)K + (int64_t)a_lo * n2;
@@ -331,6 +366,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     local_sum = warp_sum(local_sum);
     if (lane == 0 && local_sum != 0) atomicAdd(&red_sum, local_sum);
     __syncthreads();
+    BWLA_PSTAMP(9);
     if (C > 1) {
         if (threadIdx.x == 0) st_cluster_u32(map_shared_rank(smem_u32(slots + 8 + rank), 0), (uint32_t)red_sum);
         cluster_arrive_release();
@@ -342,6 +378,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         p.scales[t] = scale;
         if (p.qsum) p.qsum[t] = s;
     }
+    BWLA_PSTAMP(10);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -447,6 +484,34 @@ __global__ void prologue_kernel(PrologueParams p) {
     else lowrank_role(p, (int)blockIdx.x - p.rot_blocks);
 }
 
+// How many clusters of `c` prologue blocks (threads, dynamic shared memory) the device holds at once; cached.
+__global__ void prologue_kernel(PrologueParams p);
+static int clusters_resident(int c, int threads, size_t smem) {
+    struct Key { int dev, c, threads; size_t smem; int n; };
+    static thread_local Key cache[16];
+    static thread_local int used = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    for (int i = 0; i < used; ++i)
+        if (cache[i].dev == dev && cache[i].c == c && cache[i].threads == threads && cache[i].smem == smem) return cache[i].n;
+    if (cudaFuncSetAttribute(prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrologueSmemFloats * 4) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(c * 148), 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, prologue_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+    if (used < 16) cache[used++] = Key{dev, c, threads, smem, n};
+    return n;
+}
+
 static int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
 
 int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2, int n2,
@@ -466,47 +531,63 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     size_t smem = 0;
     if (rotate) {
         const int gran = 32 / gcd_int(n2, 32);
+        // lays the block out for clusters of `c` CTAs per token; false if it does not fit
+        auto plan = [&](int c) -> bool {
+            int cap = 0;
+            for (int i = 0; i < c; ++i) {
+                const int lo = (int)(((int64_t)n1 * i / c) / gran * gran);
+                const int hi = (i + 1 >= c) ? n1 : (int)(((int64_t)n1 * (i + 1) / c) / gran * gran);
+                cap = cap > (hi - lo) ? cap : (hi - lo);
+            }
+            p.C = c; p.rot_blocks = (int)(M * c); p.row_gran = gran; p.slab_cap = (cap * n2 + 3) / 4 * 4;
+            p.prefetch = 0; p.p1_cap = 0;
+            if ((n2 & 3) == 0) {
+                // chunks of P2 (ch1 columns) and of P1 (ch2 columns) that fit beside the X slab and Z
+                const int64_t avail = kPrologueSmemFloats - p.slab_cap - K - 16 - 8;
+                const int max1 = (int)std::min<int64_t>(n2, avail / n2 / 4 * 4);
+                const int max2 = (int)std::min<int64_t>((cap + 3) / 4 * 4, avail / n1 / 4 * 4);
+                if (max1 < 4 || max2 < 4) return false;
+                // equal chunks rather than full ones and a sliver
+                const int nch1 = (n2 + max1 - 1) / max1, nch2 = (cap + max2 - 1) / max2;
+                const int ch1 = ((n2 + nch1 - 1) / nch1 + 3) / 4 * 4;
+                const int ch2 = std::min(cap, ((cap + nch2 - 1) / nch2 + 3) / 4 * 4);
+                p.ch1 = ch1; p.ch2 = ch2;
+                p.ps_cap = std::max(n2 * ch1, n1 * ((ch2 + 3) / 4 * 4)) + 8;
+                // all of P2 and this CTA's columns of P1 at once, fetched together with x, when both fit
+                const int64_t p1_need = (int64_t)n1 * ((cap + 3) / 4 * 4) + 8;
+                if (nch1 == 1 && nch2 == 1 && (int64_t)n2 * n2 + 8 + p1_need <= avail) {
+                    p.prefetch = 1; p.ps_cap = n2 * n2 + 8; p.p1_cap = (int)p1_need;
+                }
+                // rows per thread: as many as still leave a hundred-odd tiles
+                auto pick = [](int rows, int cols4) {
+                    for (int tr = 8; tr > 1; tr >>= 1)
+                        if (((rows + tr - 1) / tr) * cols4 >= 128) return tr;
+                    return 1;
+                };
+                p.tr1 = pick(cap, ch1 / 4);
+                p.tr2 = pick(ch2, n2 / 4);
+                const int tiles = std::max(((cap + p.tr1 - 1) / p.tr1) * (ch1 / 4), ((ch2 + p.tr2 - 1) / p.tr2) * (n2 / 4));
+                const int rounds = (tiles + 511) / 512;
+                threads = ((tiles + rounds - 1) / rounds + 31) / 32 * 32;
+                threads = threads < 128 ? 128 : (threads > 512 ? 512 : threads);
+            } else {
+                p.ps_cap = 0; p.ch1 = p.ch2 = 4; p.tr1 = p.tr2 = 1;
+                threads = 256;
+            }
+            smem = ((size_t)p.slab_cap + (size_t)K + (size_t)p.ps_cap + (size_t)p.p1_cap + 16) * 4;
+            return true;
+        };
         if ((n2 & 3) == 0) {
-            // spread one token over several SMs while there are few tokens and the token is worth splitting
+            // spread one token over several SMs while there are few tokens and the token is worth splitting, as long as
+            // every token's cluster is resident at once (a second wave of clusters would double the latency)
             const double flops = 2.0 * (double)K * (n1 + n2);
             while (C < 8 && M * (C * 2) <= 160 && flops / (C * 2) >= 2.5e5 && n1 / (C * 2) >= gran) C *= 2;
+            for (; C > 1; C >>= 1) {
+                if (!plan(C)) continue;
+                if (clusters_resident(C, threads, smem) >= M) break;
+            }
         }
-        int cap = 0;
-        for (int c = 0; c < C; ++c) {
-            const int lo = (int)(((int64_t)n1 * c / C) / gran * gran);
-            const int hi = (c + 1 >= C) ? n1 : (int)(((int64_t)n1 * (c + 1) / C) / gran * gran);
-            cap = cap > (hi - lo) ? cap : (hi - lo);
-        }
-        p.C = C; p.rot_blocks = (int)(M * C); p.row_gran = gran; p.slab_cap = (cap * n2 + 3) / 4 * 4;
-        if ((n2 & 3) == 0) {
-            // chunks of P2 (ch1 columns) and of P1 (ch2 columns) that fit beside the X slab and Z
-            const int64_t avail = kPrologueSmemFloats - p.slab_cap - K - 16 - 8;
-            const int max1 = (int)std::min<int64_t>(n2, avail / n2 / 4 * 4);
-            const int max2 = (int)std::min<int64_t>((cap + 3) / 4 * 4, avail / n1 / 4 * 4);
-            if (max1 < 4 || max2 < 4) return BWLA_ERR_INVALID_ARG;
-            // equal chunks rather than full ones and a sliver
-            const int nch1 = (n2 + max1 - 1) / max1, nch2 = (cap + max2 - 1) / max2;
-            const int ch1 = ((n2 + nch1 - 1) / nch1 + 3) / 4 * 4;
-            const int ch2 = std::min(cap, ((cap + nch2 - 1) / nch2 + 3) / 4 * 4);
-            p.ch1 = ch1; p.ch2 = ch2;
-            p.ps_cap = std::max(n2 * ch1, n1 * ((ch2 + 3) / 4 * 4)) + 8;
-            // rows per thread: as many as still leave a few hundred tiles
-            auto pick = [](int rows, int cols4) {
-                for (int tr = 8; tr > 1; tr >>= 1)
-                    if (((rows + tr - 1) / tr) * cols4 >= 256) return tr;
-                return 1;
-            };
-            p.tr1 = pick(cap, ch1 / 4);
-            p.tr2 = pick(ch2, n2 / 4);
-            const int tiles = std::max(((cap + p.tr1 - 1) / p.tr1) * (ch1 / 4), ((ch2 + p.tr2 - 1) / p.tr2) * (n2 / 4));
-            const int rounds = (tiles + 511) / 512;
-            threads = ((tiles + rounds - 1) / rounds + 31) / 32 * 32;
-            threads = threads < 128 ? 128 : (threads > 512 ? 512 : threads);
-        } else {
-            p.ps_cap = 0; p.ch1 = p.ch2 = 4; p.tr1 = p.tr2 = 1;
-            threads = 256;
-        }
-        smem = ((size_t)p.slab_cap + (size_t)K + (size_t)p.ps_cap + 16) * 4;
+        if (!plan(C)) return BWLA_ERR_INVALID_ARG;
     } else {
         p.C = 1; p.rot_blocks = 0;
     }
