@@ -13,16 +13,16 @@
 //     (programmatic dependent launch);
 //   * warp 1 waits for the preceding kernel, then streams the three bf16 terms of T and the activation codes
 //     (tokens x 128 bytes per k-block, the canonical K-major 128B-swizzled UMMA layout);
-//   * warps 4..11 (two per tensor-memory lane quarter, thread = output row, the two warps of a quarter taking
+//   * warps 6..13 (two per tensor-memory lane quarter, thread = output row, the two warps of a quarter taking
 //     alternate k-blocks) stage the U tile in shared memory, then turn each 32-bit sign word into eight registers
 //     of four int8 with one shift and one mask per register ((w << (7-j)) & 0x80808080) and write them with
 //     tcgen05.st into tensor memory, where they are the A operand: expanded weights never touch shared memory.
-//   * NISS threads (one each in warps 2 and 3) issue tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor
+//   * NISS threads (one each in warps 2..5) issue tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor
 //     memory, B from shared memory), taking k-blocks round-robin, each into an int32 accumulator of its own in
 //     tensor memory: with few tokens an MMA is short and the issue latency of one thread would be the bottleneck.
 //     The first of them also issues the kind::f16 MMAs of the low-rank term (A = U tile, B = T as three bf16
 //     terms, fp32 accumulator in tensor memory);
-//   * warps 4..11 read the accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
+//   * warps 6..13 read the accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
 //     scales, transpose through shared memory and store bf16 with 128-bit stores.
 // The shift-and-mask expansion meets the weights of a 32-group in the order k = j + 8*i (register j, byte i), so the
 // codes are stored in that interleaved order by the quantiser.
@@ -41,9 +41,7 @@ using namespace ptx;
 constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
 constexpr int kBlockK = 128;             // K per code sub-block / per tensor-memory A stage
-constexpr int kFirstExpander = 128;      // warps 0, 1: TMA; warps 2, 3: MMA issue; warps 4..11: expand + epilogue
-constexpr int kExpanders = 256;
-constexpr int kThreads = kFirstExpander + kExpanders;
+constexpr int kFirstExpander = 192;      // warps 0, 1: TMA; warps 2..5: MMA issue; warps 6..13: expand + epilogue
 constexpr uint32_t kWaitLimit = 1u << 20;   // polls per wait before giving up (tens of milliseconds)
 
 struct UmmaParams {
@@ -59,9 +57,6 @@ struct UmmaParams {
     int64_t ldo;
     int32_t* acc_debug;          // [M][N] or NULL
     uint32_t* status;
-#ifdef BWLA_TRACE
-    const uint32_t* packed_dbg;  // tuning builds compare what the expanders read from shared memory with global memory
-#endif
 };
 
 // Shared-memory and tensor-memory budget of one CTA.
@@ -73,34 +68,32 @@ struct UmmaParams {
 //   stages of 32 columns (one k-block of expanded weights each).
 // The cluster reduction buffers (int32 and fp32, N_TOK x 128 each) and the bf16 output tile reuse the stage memory
 // once the K loop is over.
-template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS>
+template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS, int EW>
 struct UmmaCfg {
+    static constexpr int kExpanders = 128 * EW;                        // EW warps per tensor-memory lane quarter
+    static constexpr int kThreads = kFirstExpander + kExpanders;
     static constexpr int w_bytes = kRowsPerCta * 128;
     static constexpr int sub_bytes = N_TOK * 128;
     static constexpr int SUBS = (128 / N_TOK) < 1 ? 1 : ((128 / N_TOK) > 8 ? 8 : (128 / N_TOK));
     static constexpr int b_bytes = SUBS * sub_bytes;
     static constexpr int D2_COL = NISS * N_TOK;
     static constexpr int A_COL = ((NISS + 1) * N_TOK + 31) / 32 * 32;
-    static constexpr int AS = ((TMEM_COLS - A_COL) / 32) & ~1;        // even: the two warps of a quarter alternate
+    static constexpr int AS = ((TMEM_COLS - A_COL) / 32) / EW * EW;   // a multiple of EW: the warps of a quarter take turns
     static constexpr int u_off = WS * w_bytes + BS * b_bytes;
     static constexpr int t_off = u_off + kRowsPerCta * 128;
     static constexpr int bars_off = t_off + 3 * sub_bytes;
-    static constexpr int n_bars = 2 * WS + 2 * BS + 2 * AS + 3;
+    static constexpr int n_bars = 2 * WS + 2 * BS + 2 * AS + 4;
     static constexpr int misc_off = bars_off + n_bars * 8;            // tmem slot, abort flag
     static constexpr int tok_off = misc_off + 16;                      // scales[N_TOK], qsum[N_TOK]
     static constexpr int used = tok_off + 8 * N_TOK;
     static constexpr int total = used + 1024;                          // + slack for 1024-byte alignment
     static constexpr int red_bytes = 2 * N_TOK * kRowsPerCta * 4;
     static constexpr bool can_split = red_bytes <= u_off;
-    static_assert(NISS >= 1 && NISS <= 2, "one or two issuing warps");
-    static_assert(AS >= 2, "tensor memory: no room for the expanded-weight ring");
+    static_assert(NISS >= 1 && NISS <= 4, "one to four issuing warps");
+    static_assert(EW == 2 || EW == 4, "two or four expander warps per lane quarter");
+    static_assert(AS >= 2 * EW, "tensor memory: no room for the expanded-weight ring");
     static_assert(N_TOK * kRowsPerCta * 2 <= u_off, "output tile does not fit the stage memory");
 };
-
-#ifdef BWLA_TRACE
-__device__ uint32_t* g_xor_dbg = nullptr;   // [N][2]: XOR of the sign words each expander thread read from shared memory
-extern "C" int bwla_trace_set_xor_buffer(void* p) { return cudaMemcpyToSymbol(g_xor_dbg, &p, sizeof(p)) == cudaSuccess ? 0 : -4; }
-#endif
 
 // Optional timeline of CTA (0,0,0) for tuning: clock64 stamps behind the status words (compiled out by default).
 #ifdef BWLA_TRACE
@@ -119,9 +112,8 @@ __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_fl
     *abort_flag = 1;
 }
 
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t* polls = nullptr) {
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (polls) *polls = i;
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (i > 8192) __nanosleep(64);             // a sleeping warp wakes up late: only back off on long waits
@@ -150,14 +142,15 @@ __device__ __forceinline__ float finish_value(const UmmaParams& p, int64_t t, in
     return y;
 }
 
-template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS>
-__global__ void __launch_bounds__(kThreads, TMEM_COLS == 256 ? 2 : 1)
+template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS, int EW>
+__global__ void __launch_bounds__(kFirstExpander + 128 * EW, TMEM_COLS == 256 ? 2 : 1)
 umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map,
                 const __grid_constant__ CUtensorMap t_map, UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
-    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS>;
+    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS, EW>;
     constexpr int AS = L::AS;
     constexpr int SUBS = L::SUBS;
+    constexpr int kExpanders = L::kExpanders;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* wbuf = smem;
     uint8_t* bbuf = smem + WS * L::w_bytes;
@@ -173,6 +166,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     uint64_t* d_full = a_empty + AS;         // [1] every issuing thread's MMAs have completed
     uint64_t* u_full = d_full + 1;           // [1] U tile staged by the expander warps
     uint64_t* t_full = u_full + 1;           // [1] the three terms of T landed
+    uint64_t* s_full = t_full + 1;           // [1] per-token scales and code sums staged in shared memory
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(smem + L::misc_off);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
     float* scale_s = reinterpret_cast<float*>(smem + L::tok_off);
@@ -204,6 +198,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         mbar_init(d_full, NISS);
         mbar_init(u_full, kExpanders / 32);
         mbar_init(t_full, 1);
+        mbar_init(s_full, 1);
         fence_barrier_init();
         fence_proxy_async();
     }
@@ -232,11 +227,18 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);   // let copies in flight land
         }
     } else if (warp == 1) {
-        // ---------------- T and the activation codes: L2 -> shared memory ----------------
+        // ---------------- per-token scales, T and the activation codes: L2 -> shared memory ----------------
+        griddep_wait();                           // all of them come from the preceding kernel
+        for (int i = lane; i < N_TOK; i += 32) {
+            const int t = t0 + i;
+            scale_s[i] = t < p.M ? p.scales[t] : 0.f;
+            qsum_s[i] = t < p.M ? p.qsum[t] : 0;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(s_full);
         if (elect_one()) {
             tma_prefetch_desc(&b_map);
             if (lowrank_here) tma_prefetch_desc(&t_map);
-            griddep_wait();                       // codes, scales and T come from the preceding kernel
             if (p.status && *reinterpret_cast<volatile uint32_t*>(p.status) != 0) *abort_flag = 1;   // the call already failed
             if (lowrank_here && !*abort_flag) {
                 mbar_expect_tx(t_full, 3 * L::sub_bytes);
@@ -257,7 +259,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);
         }
-    } else if (warp < 4) {
+    } else if (warp < 6) {
         // ---------------- MMA issue: thread `iss` takes k-blocks kb = iss, iss + NISS, ... ----------------
         const int iss = warp - 2;
         if (iss < NISS && elect_one()) {
@@ -295,7 +297,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         const int as = kb % AS;
                         const uint32_t aph = (uint32_t)(kb / AS) & 1u;
                         if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
-                        if (kb < 96) BWLA_STAMP(32 + kb);
+                        if (kb == 0) BWLA_STAMP(8);
                         tc_fence_after();
                         const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
                         const uint32_t a_addr = tmem_base + L::A_COL + 32 * as;
@@ -303,7 +305,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         for (int i = 0; i < 4; ++i)
                             mma_i8_ts(d_addr, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, (kb < NISS && i == 0) ? 0u : 1u);
                         tc_commit(&a_empty[as]);
-                        if (kb < 96) BWLA_STAMP(416 + kb);
                     }
                     if (sb == SUBS - 1 || s == ns - 1) {
                         // this thread is done with the code stage once its MMAs so far have completed
@@ -313,14 +314,18 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 }
             }
             tc_commit(d_full);
+            if (iss == 0) BWLA_STAMP(9);
         }
     } else {
         // ---------------- U tile, expansion of sign bits into tensor memory, then the epilogue ----------------
         const int q = warp & 3;                       // tensor-memory lane quarter this warp may touch
-        const int half = (warp - 4) >> 2;             // which of the two warps of that quarter
+        const int part = (warp - 6) >> 2;             // which of the EW warps of that quarter
         const int row = q * 32 + lane;
         const int e = threadIdx.x - kFirstExpander;   // 0..255 among the expander threads
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        // this row's weight scale and shift do not depend on the preceding kernel: fetched now, used in the epilogue
+        const float alpha_row = n0 + row < p.N ? __ldg(p.alpha + n0 + row) : 0.f;
+        const float mu_row = (p.mu && n0 + row < p.N) ? __ldg(p.mu + n0 + row) : 0.f;
         if (lowrank_here) {
             // 128 rows x 8 chunks of 16 bytes, 128B-swizzled K-major; rows beyond N and columns beyond r are zero
             const bool vec = (p.r % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.U) & 15) == 0);
@@ -347,35 +352,28 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(u_full);
         }
-        // This warp expands k-blocks kb = half, half + 2, ... of the CTA (stage kb % AS; AS is even).  tcgen05.st reads
-        // its source registers asynchronously, so they are left alone until tcgen05.wait::st has returned; the other
-        // warp of the quarter and the second CTA of the SM fill the store's latency.
+        // This warp expands k-blocks kb = part, part + EW, ... of the CTA (stage kb % AS; AS is a multiple of EW).  Its
+        // registers are left alone until tcgen05.wait::st has returned; the other warps of the quarter fill the
+        // store's latency.
         int ws = 0; uint32_t wph = 0;
         bool ok = true;
         int kb0 = 0;                                   // k-block index of sub-block 0 of the current unit
-#ifdef BWLA_TRACE
-        uint32_t xor_dbg = 0;
-#endif
         for (int u = unit_begin; u < unit_end && ok; ++u) {
             if (!warp_wait(&w_full[ws], wph, abort_flag, lane)) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
+            if (e == 64 && u == unit_begin) BWLA_STAMP(3);
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
-            const int s_first = (kb0 + half) & 1;      // kb0 + s has the parity of `half`
+            const int s_first = ((part - kb0) % EW + EW) % EW;      // kb0 + s_first = part (mod EW)
             // the sign words of this warp's k-blocks of the unit, loaded together
-            uint4 w4[4];
+            uint4 w4[8 / EW];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int s = 2 * i + s_first;
+            for (int i = 0; i < 8 / EW; ++i) {
+                const int s = EW * i + s_first;
                 if (s < ns) w4[i] = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
             }
-#ifdef BWLA_TRACE
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (2 * i + s_first < ns) xor_dbg ^= w4[i].x ^ w4[i].y ^ w4[i].z ^ w4[i].w;
-#endif
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int s = 2 * i + s_first;
+            for (int i = 0; i < 8 / EW; ++i) {
+                const int s = EW * i + s_first;
                 if (s >= ns) break;
                 const int kb = kb0 + s;
                 const int as = kb % AS;
@@ -401,18 +399,11 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (++ws == WS) { ws = 0; wph ^= 1; }
             kb0 += ns;
         }
-#ifdef BWLA_TRACE
-        if (g_xor_dbg && n0 + row < p.N) g_xor_dbg[(int64_t)(n0 + row) * 2 + half] = xor_dbg;
-#endif
         if (e == 64) BWLA_STAMP(4);
-        // per-token scale and code sum of this tile (written by the preceding kernel)
+        // the stores of the epilogue come after the preceding kernel; the per-token scales and code sums it wrote were
+        // staged in shared memory by warp 1 while the K loop ran
         griddep_wait();
-        if (e < N_TOK) {
-            const int t = t0 + e;
-            scale_s[e] = t < p.M ? p.scales[t] : 0.f;
-            qsum_s[e] = t < p.M ? p.qsum[t] : 0;
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");     // the expander warps only
+        if (!warp_wait(s_full, 0, abort_flag, lane)) { give_up(p.status, abort_flag, 0x51); ok = false; }
         if (ok) {
             if (!warp_wait(d_full, 0, abort_flag, lane)) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
@@ -422,11 +413,10 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             const int n = n0 + row;
             const int nacc = min(NISS, my_blocks);             // accumulators that hold something
             const bool single = p.splits == 1;
-            const float alpha_n = n < p.N ? p.alpha[n] : 0.f;
-            const float mu_n = (p.mu && n < p.N) ? p.mu[n] : 0.f;
-            // the two warps of a quarter take alternate chunks of 16 tokens
+            const float alpha_n = alpha_row, mu_n = mu_row;
+            // the warps of a quarter take chunks of 16 tokens in turn
 #pragma unroll 1
-            for (int c = half; c < N_TOK / 16; c += 2) {
+            for (int c = part; c < N_TOK / 16; c += EW) {
                 if (t0 + 16 * c >= p.M) break;                 // warp-uniform
                 uint32_t v[16], l[16];
                 tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
@@ -460,7 +450,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
         }
         if (p.splits == 1) {
-            asm volatile("bar.sync 1, 256;" ::: "memory");   // the output tile is complete (all expander warps, always)
+            asm volatile("bar.sync 1, %0;" ::"r"(kExpanders) : "memory");   // the output tile is complete (all expander warps, always)
             if (ok && p.out) {
                 // 16 threads move one token's 128 outputs (256 bytes) with 128-bit stores
                 const bool vec = ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) && (p.ldo % 8 == 0) && (n0 + kRowsPerCta <= p.N);
@@ -486,7 +476,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         // every thread of every CTA of the cluster takes part, whether or not its CTA gave up
         cluster_arrive_release();
         cluster_wait_acquire();
-        if (L::can_split && warp >= 4 && !*abort_flag) {
+        if (L::can_split && warp >= 6 && !*abort_flag) {
             // the tokens of the tile are dealt round-robin to the CTAs of the cluster; a thread sums four consecutive
             // rows of one token over all CTAs with 128-bit distributed-shared-memory loads
             const int e = threadIdx.x - kFirstExpander;
@@ -571,11 +561,11 @@ static int make_map(CUtensorMap* map, CUtensorMapDataType dt, int rank, const vo
     return BWLA_OK;
 }
 
-template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS>
+template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS, int EW>
 static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUtensorMap& tm, const UmmaParams& p,
                          dim3 grid, cudaStream_t s) {
-    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS>;
-    auto kernel = umma_w1a_kernel<N_TOK, WS, BS, TMEM_COLS, NISS>;
+    using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS, EW>;
+    auto kernel = umma_w1a_kernel<N_TOK, WS, BS, TMEM_COLS, NISS, EW>;
     static thread_local int configured = -1;
     int dev = 0;
     BWLA_CUDA_TRY(cudaGetDevice(&dev));
@@ -585,7 +575,7 @@ static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUt
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(L::kThreads, 1, 1);
     cfg.dynamicSmemBytes = L::total;
     cfg.stream = s;
     cudaLaunchAttribute attrs[2];
@@ -656,18 +646,13 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
     p.M = M; p.N = N; p.K = K; p.total_units = units; p.splits = split; p.r = a.r;
     p.scales = a.scales; p.qsum = a.qsum; p.alpha = a.alpha; p.mu = a.mu; p.U = (const __nv_bfloat16*)a.U;
     p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug; p.status = a.status;
-#ifdef BWLA_TRACE
-    p.packed_dbg = a.packed;
-#endif
+
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     switch (n_tok) {
-        #ifndef BWLA_DBG_NISS
-#define BWLA_DBG_NISS 2
-#endif
-        case 16: return launch_umma_t<16, 3, 2, 256, BWLA_DBG_NISS>(wm, bm, tm, p, grid, stream);
-        case 32: return launch_umma_t<32, 3, 2, 256, 2>(wm, bm, tm, p, grid, stream);
-        case 64: return launch_umma_t<64, 4, 3, 512, 2>(wm, bm, tm, p, grid, stream);
-        default: return launch_umma_t<128, 2, 6, 512, 1>(wm, bm, tm, p, grid, stream);
+                case 16: return launch_umma_t<16, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
+        case 32: return launch_umma_t<32, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
+        case 64: return launch_umma_t<64, 4, 3, 512, 2, 2>(wm, bm, tm, p, grid, stream);
+        default: return launch_umma_t<128, 2, 6, 512, 1, 2>(wm, bm, tm, p, grid, stream);
     }
 }
 

@@ -559,9 +559,12 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                     p.prefetch = 1; p.ps_cap = n2 * n2 + 8; p.p1_cap = (int)p1_need;
                 }
                 // rows per thread: as many as still leave a hundred-odd tiles
-                auto pick = [](int rows, int cols4) {
+                // (a block that shares a token wants its short chain done soon; a block that owns a whole token
+                // wants enough threads to hide latency)
+                const int want_tiles = c > 1 ? 128 : 256;
+                auto pick = [want_tiles](int rows, int cols4) {
                     for (int tr = 8; tr > 1; tr >>= 1)
-                        if (((rows + tr - 1) / tr) * cols4 >= 128) return tr;
+                        if (((rows + tr - 1) / tr) * cols4 >= want_tiles) return tr;
                     return 1;
                 };
                 p.tr1 = pick(cap, ch1 / 4);
