@@ -30,10 +30,8 @@ namespace bwla {
 
 using namespace ptx;
 
-constexpr int kLrTokens = 16;     // tokens per low-rank block
-constexpr int kLrRows = 2;        // rows of V per low-rank block
 constexpr int kLrMaxWarps = 16;   // blocks have at most 512 threads
-constexpr int kPrologueSmemFloats = 56 * 1024;   // dynamic shared memory of a prologue block, in floats (224 KB)
+constexpr int kPrologueSmemFloats = 55 * 1024;   // dynamic shared memory of a prologue block, in floats (220 KB; about 6 KB are static)
 
 // Optional phase timeline of rotation block 0 for tuning (compiled out by default).
 #ifdef BWLA_TRACE
@@ -62,6 +60,7 @@ struct PrologueParams {
     int tr1, tr2;       // rows per thread in the two contractions
     // low-rank
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
+    int lr_wide;        // 1: blocks of 8 rows of V x 8 tokens (many tokens), 0: 2 rows x 16 tokens
 };
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -384,96 +383,104 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
 // ---------------------------------------------------------------------------------------------
 // T = V x, written as three bf16 terms
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void fma8(float (&acc)[kLrTokens], int tt, const uint4& v, const uint4& xv) {
+// acc += dot of eight bf16 pairs (two packed 128-bit words)
+__device__ __forceinline__ float dot8(float acc, const uint4& v, const uint4& xv) {
     const uint32_t a[4] = {v.x, v.y, v.z, v.w}, b[4] = {xv.x, xv.y, xv.z, xv.w};
-    float s = acc[tt];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        s = fmaf(__uint_as_float(a[i] << 16), __uint_as_float(b[i] << 16), s);
-        s = fmaf(__uint_as_float(a[i] & 0xFFFF0000u), __uint_as_float(b[i] & 0xFFFF0000u), s);
+        acc = fmaf(__uint_as_float(a[i] << 16), __uint_as_float(b[i] << 16), acc);
+        acc = fmaf(__uint_as_float(a[i] & 0xFFFF0000u), __uint_as_float(b[i] & 0xFFFF0000u), acc);
     }
-    acc[tt] = s;
+    return acc;
 }
 
+// One block reduces R rows of V against T tokens (R x T accumulators per thread, threads stride over K).  Few tokens:
+// R = 2, T = 16 (many blocks).  Many tokens: R = T = 8, which reads each operand four times less often from L2.
+template <int R, int T>
 __device__ void lowrank_role(const PrologueParams& p, int b) {
-    const int jblocks = p.lr_cols / kLrRows;
+    const int jblocks = p.lr_cols / R;
     const int jb = b % jblocks;
-    const int64_t t0 = (int64_t)(b / jblocks) * kLrTokens;
+    const int64_t t0 = (int64_t)(b / jblocks) * T;
     if (t0 >= p.M) return;
-    const int j0 = jb * kLrRows;
-    const int nt = (int)min((int64_t)kLrTokens, p.M - t0);
-    float acc[kLrRows][kLrTokens];
+    const int j0 = jb * R;
+    const int nt = (int)min((int64_t)T, p.M - t0);
+    float acc[R][T];
 #pragma unroll
-    for (int j = 0; j < kLrRows; ++j)
+    for (int j = 0; j < R; ++j)
 #pragma unroll
-        for (int i = 0; i < kLrTokens; ++i) acc[j][i] = 0.f;
+        for (int i = 0; i < T; ++i) acc[j][i] = 0.f;
     griddep_launch_dependents();
     if (j0 < p.r) {
         const int K = p.K;
-        const bool two = j0 + 1 < p.r;
-        const __nv_bfloat16* v0 = p.V + (int64_t)j0 * K;
-        const __nv_bfloat16* v1 = p.V + (int64_t)(two ? j0 + 1 : j0) * K;
+        const int nr = min(R, p.r - j0);                      // rows of V this block really has
+        const __nv_bfloat16* vrow[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) vrow[j] = p.V + (int64_t)(j0 + min(j, nr - 1)) * K;
         const __nv_bfloat16* xt = p.x + t0 * p.ldx;
         const bool vec = ((reinterpret_cast<uintptr_t>(p.V) | reinterpret_cast<uintptr_t>(p.x)) & 15) == 0 && (p.ldx & 7) == 0;
         if (vec) {
             for (int kc = threadIdx.x; kc < (K >> 3); kc += blockDim.x) {
-                const uint4 a0 = __ldg(reinterpret_cast<const uint4*>(v0) + kc);
-                const uint4 a1 = __ldg(reinterpret_cast<const uint4*>(v1) + kc);
+                uint4 a[R];
 #pragma unroll
-                for (int tt = 0; tt < kLrTokens; ++tt) {
+                for (int j = 0; j < R; ++j) a[j] = __ldg(reinterpret_cast<const uint4*>(vrow[j]) + kc);
+#pragma unroll
+                for (int tt = 0; tt < T; ++tt) {
                     if (tt < nt) {
                         const uint4 xv = __ldg(reinterpret_cast<const uint4*>(xt + tt * p.ldx) + kc);
-                        fma8(acc[0], tt, a0, xv);
-                        fma8(acc[1], tt, a1, xv);
+#pragma unroll
+                        for (int j = 0; j < R; ++j) acc[j][tt] = dot8(acc[j][tt], a[j], xv);
                     }
                 }
             }
         } else {
             for (int k = threadIdx.x; k < K; k += blockDim.x) {
-                const float a0 = __bfloat162float(v0[k]), a1 = __bfloat162float(v1[k]);
+                float a[R];
 #pragma unroll
-                for (int tt = 0; tt < kLrTokens; ++tt) {
+                for (int j = 0; j < R; ++j) a[j] = __bfloat162float(vrow[j][k]);
+#pragma unroll
+                for (int tt = 0; tt < T; ++tt) {
                     if (tt < nt) {
                         const float xv = __bfloat162float(xt[tt * p.ldx + k]);
-                        acc[0][tt] = fmaf(a0, xv, acc[0][tt]);
-                        acc[1][tt] = fmaf(a1, xv, acc[1][tt]);
+#pragma unroll
+                        for (int j = 0; j < R; ++j) acc[j][tt] = fmaf(a[j], xv, acc[j][tt]);
                     }
                 }
             }
         }
-        if (!two) {
 #pragma unroll
-            for (int i = 0; i < kLrTokens; ++i) acc[1][i] = 0.f;
-        }
+        for (int j = 0; j < R; ++j)
+            if (j >= nr) {
+#pragma unroll
+                for (int i = 0; i < T; ++i) acc[j][i] = 0.f;
+            }
     }
-    __shared__ float red[kLrMaxWarps][kLrRows * kLrTokens];
+    __shared__ float red[kLrMaxWarps][R * T];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-    for (int j = 0; j < kLrRows; ++j)
+    for (int j = 0; j < R; ++j)
 #pragma unroll
-        for (int i = 0; i < kLrTokens; ++i) {
+        for (int i = 0; i < T; ++i) {
             float v = acc[j][i];
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-            if (lane == 0) red[warp][j * kLrTokens + i] = v;
+            if (lane == 0) red[warp][j * T + i] = v;
         }
     __syncthreads();
     griddep_wait();
-    if (threadIdx.x < kLrRows * kLrTokens) {
-        const int j = threadIdx.x / kLrTokens, i = threadIdx.x % kLrTokens;
+    for (int o = threadIdx.x; o < R * T; o += blockDim.x) {
+        const int j = o / T, i = o % T;
         if (i < nt) {
             float s = 0.f;
-#pragma unroll
-            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w][threadIdx.x];
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w][o];
             // three bf16 terms carry all 24 bits of the fp32 sum
             const __nv_bfloat16 hi = __float2bfloat16_rn(s);
             const float r1 = s - __bfloat162float(hi);
             const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
             const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-            const int64_t o = (t0 + i) * p.lr_cols + j0 + j;
-            p.Thl[o] = hi;
-            p.Thl[p.M * p.lr_cols + o] = mid;
-            p.Thl[2 * p.M * p.lr_cols + o] = lo;
+            const int64_t at = (t0 + i) * p.lr_cols + j0 + j;
+            p.Thl[at] = hi;
+            p.Thl[p.M * p.lr_cols + at] = mid;
+            p.Thl[2 * p.M * p.lr_cols + at] = lo;
         }
     }
 }
@@ -481,7 +488,8 @@ __device__ void lowrank_role(const PrologueParams& p, int b) {
 __global__ void prologue_kernel(PrologueParams p) {
     extern __shared__ __align__(16) float smem[];
     if ((int)blockIdx.x < p.rot_blocks) rotate_role(p, smem);
-    else lowrank_role(p, (int)blockIdx.x - p.rot_blocks);
+    else if (p.lr_wide) lowrank_role<8, 8>(p, (int)blockIdx.x - p.rot_blocks);
+    else lowrank_role<2, 16>(p, (int)blockIdx.x - p.rot_blocks);
 }
 
 // How many clusters of `c` prologue blocks (threads, dynamic shared memory) the device holds at once; cached.
@@ -596,7 +604,8 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     }
     int lr_blocks = 0;
     if (r > 0 && Thl) {
-        lr_blocks = (p.lr_cols / kLrRows) * (int)((M + kLrTokens - 1) / kLrTokens);
+        p.lr_wide = (M >= 64 && p.lr_cols % 8 == 0) ? 1 : 0;
+        lr_blocks = p.lr_wide ? (p.lr_cols / 8) * (int)((M + 7) / 8) : (p.lr_cols / 2) * (int)((M + 15) / 16);
     }
     int grid = p.rot_blocks + lr_blocks;
     grid = (grid + C - 1) / C * C;
