@@ -132,14 +132,10 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
     return ok != 0;
 }
 
-// One output value from its two accumulators.
-__device__ __forceinline__ float finish_value(const UmmaParams& p, int64_t t, int n, int32_t d, float l, float sc,
-                                              int32_t qs, float alpha_n, float mu_n) {
+// One output value from its two accumulators (mu_sc is zero when the layer has no row shift).
+__device__ __forceinline__ float finish_value(int32_t d, float l, float alpha_sc, float mu_sc, int32_t qs) {
     const int32_t acc = -(d >> 6) - qs;
-    if (p.acc_debug) p.acc_debug[t * p.N + n] = acc;
-    float y = __fmul_rn(__fmul_rn(alpha_n, sc), (float)acc) + l;
-    if (p.mu) y = fmaf(__fmul_rn(mu_n, sc), (float)qs, y);
-    return y;
+    return fmaf(mu_sc, (float)qs, __fmul_rn(alpha_sc, (float)acc) + l);
 }
 
 template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS, int EW>
@@ -324,8 +320,10 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         const int e = threadIdx.x - kFirstExpander;   // 0..255 among the expander threads
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         // this row's weight scale and shift do not depend on the preceding kernel: fetched now, used in the epilogue
-        const float alpha_row = n0 + row < p.N ? __ldg(p.alpha + n0 + row) : 0.f;
-        const float mu_row = (p.mu && n0 + row < p.N) ? __ldg(p.mu + n0 + row) : 0.f;
+        float alpha_row = n0 + row < p.N ? __ldg(p.alpha + n0 + row) : 0.f;
+        float mu_row = (p.mu && n0 + row < p.N) ? __ldg(p.mu + n0 + row) : 0.f;
+        // pinned in registers: left alone, the compiler re-issues the global loads where the values are used
+        asm volatile("" : "+f"(alpha_row), "+f"(mu_row));
         if (lowrank_here) {
             // 128 rows x 8 chunks of 16 bytes, 128B-swizzled K-major; rows beyond N and columns beyond r are zero
             const bool vec = (p.r % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.U) & 15) == 0);
@@ -414,6 +412,9 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             const int nacc = min(NISS, my_blocks);             // accumulators that hold something
             const bool single = p.splits == 1;
             const float alpha_n = alpha_row, mu_n = mu_row;
+            int32_t* const dbg = p.acc_debug;
+            const int M_ = p.M, N_ = p.N;
+            const bool valid_row = n < N_;
             // the warps of a quarter take chunks of 16 tokens in turn
 #pragma unroll 1
             for (int c = part; c < N_TOK / 16; c += EW) {
@@ -422,6 +423,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
                 if (lowrank_here) tmem_ld_32x16(tmem_base + lane_addr + L::D2_COL + 16 * c, l);
                 tc_wait_ld();
+                if (e == 64 && c == part) BWLA_STAMP(10);
 #pragma unroll
                 for (int a = 1; a < NISS; ++a) {
                     if (a < nacc) {
@@ -432,25 +434,40 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         for (int j = 0; j < 16; ++j) v[j] += v2[j];
                     }
                 }
+                if (e == 64 && c == part) BWLA_STAMP(13);
+                // the chunk's scales and code sums go to registers first: the tile stores below may alias them as far as
+                // the compiler knows, and a load behind every store would serialise the loop
+                float sc[16]; int32_t qs[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int tt = 16 * c + j;
-                    const int32_t d = (int32_t)v[j];
-                    const float lr = lowrank_here ? __uint_as_float(l[j]) : 0.f;
-                    if (single) {
-                        // finished value -> bf16 tile in shared memory, [token][row]
-                        float y = 0.f;
-                        if (n < p.N && t0 + tt < p.M) y = finish_value(p, t0 + tt, n, d, lr, scale_s[tt], qsum_s[tt], alpha_n, mu_n);
-                        otile[tt * kRowsPerCta + row] = __float2bfloat16_rn(y);
-                    } else if (L::can_split) {
-                        red_i[tt * kRowsPerCta + row] = d;
-                        if (lowrank_here) red_f[tt * kRowsPerCta + row] = lr;
+                for (int j = 0; j < 16; ++j) { sc[j] = scale_s[16 * c + j]; qs[j] = qsum_s[16 * c + j]; }
+                if (e == 64 && c == part) BWLA_STAMP(14);
+                // branch-free per element (rows beyond N and tokens beyond M produce values nobody stores):
+                // a branch per element costs more than the arithmetic it would skip
+                if (dbg && valid_row) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (t0 + 16 * c + j < M_) dbg[(int64_t)(t0 + 16 * c + j) * N_ + n] = -((int32_t)v[j] >> 6) - qs[j];
+                }
+                if (single) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const float lr = lowrank_here ? __uint_as_float(l[j]) : 0.f;
+                        const float y = finish_value((int32_t)v[j], lr, __fmul_rn(alpha_n, sc[j]), __fmul_rn(mu_n, sc[j]), qs[j]);
+                        otile[(16 * c + j) * kRowsPerCta + row] = __float2bfloat16_rn(y);      // [token][row]
+                    }
+                } else if (L::can_split) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        red_i[(16 * c + j) * kRowsPerCta + row] = (int32_t)v[j];
+                        if (lowrank_here) red_f[(16 * c + j) * kRowsPerCta + row] = __uint_as_float(l[j]);
                     }
                 }
             }
         }
+        if (e == 64) BWLA_STAMP(11);
         if (p.splits == 1) {
             asm volatile("bar.sync 1, %0;" ::"r"(kExpanders) : "memory");   // the output tile is complete (all expander warps, always)
+            if (e == 64) BWLA_STAMP(12);
             if (ok && p.out) {
                 // 16 threads move one token's 128 outputs (256 bytes) with 128-bit stores
                 const bool vec = ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) && (p.ldo % 8 == 0) && (n0 + kRowsPerCta <= p.N);
@@ -501,8 +518,11 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     float y = 0.f;
-                    if (n + j < p.N)
-                        y = finish_value(p, t0 + tt, n + j, d[j], l4[j], scale_s[tt], qsum_s[tt], p.alpha[n + j], p.mu ? p.mu[n + j] : 0.f);
+                    if (n + j < p.N) {
+                        y = finish_value(d[j], l4[j], __fmul_rn(p.alpha[n + j], scale_s[tt]),
+                                         p.mu ? __fmul_rn(p.mu[n + j], scale_s[tt]) : 0.f, qsum_s[tt]);
+                        if (p.acc_debug) p.acc_debug[(int64_t)(t0 + tt) * p.N + n + j] = -(d[j] >> 6) - qsum_s[tt];
+                    }
                     y4[j] = __float2bfloat16_rn(y);
                 }
                 if (p.out) {
