@@ -580,7 +580,8 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                 const int tiles = std::max(((cap + p.tr1 - 1) / p.tr1) * (ch1 / 4), ((ch2 + p.tr2 - 1) / p.tr2) * (n2 / 4));
                 const int rounds = (tiles + 511) / 512;
                 threads = ((tiles + rounds - 1) / rounds + 31) / 32 * 32;
-                threads = threads < 128 ? 128 : (threads > 512 ? 512 : threads);
+                // never fewer than 256: the low-rank blocks of the same launch stride over K with this many threads
+                threads = threads < 256 ? 256 : (threads > 512 ? 512 : threads);
             } else {
                 p.ps_cap = 0; p.ch1 = p.ch2 = 4; p.tr1 = p.tr2 = 1;
                 threads = 256;
