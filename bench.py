@@ -30,6 +30,14 @@ if ROOT not in sys.path:
 
 from paper_2605_00422_b200 import inputs as gen  # noqa: E402
 
+# DRAM bytes of one contraction launch from an ncu capture (profiles/), with the algorithmic bytes of that same launch and
+# the hash of the kernel source the capture was taken from.  The ratio scales the average launch of the step; when the
+# kernel source has changed since, the figure is dropped (null).
+NCU_TRAFFIC = {
+    "decode": {"dram_bytes": 19941376, "algorithmic_bytes": 20670592,          # gate_proj launch, M = 16
+               "kernel_sha256": "101e33b2e90acea934b63088c5380c277701efb3a64c3ab54c5a48dd02199c0b"},
+}
+
 METRIC = "W1A6 linear: decode HBM GB/s & prefill INT8 TOPS vs B200 roofline, Qwen3-32B"
 BITS = 6
 
@@ -48,6 +56,19 @@ def contraction_kernel_bytes(sh: gen.LinearShape, M: int) -> int:
     """Algorithmic bytes of one launch of the contraction kernel (fused epilogue): sign bits, int8 codes, U, the three
     bf16 terms of T, alpha, per-token scale and code sum in; bf16 outputs out."""
     return sh.N * sh.K // 8 + M * sh.K + 2 * sh.r * sh.N + 6 * M * 64 + 4 * sh.N + 8 * M + 2 * M * sh.N
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    with open(os.path.join(ROOT, "paper_2605_00422_b200", "csrc", "gemm_umma.cu"), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()
+
+
+def measured_traffic(which: str, algorithmic_bytes_per_launch: float):
+    t = NCU_TRAFFIC.get(which)
+    if not t or not t["dram_bytes"] or t["kernel_sha256"] != kernel_source_hash():
+        return None
+    return t["dram_bytes"] / t["algorithmic_bytes"] * algorithmic_bytes_per_launch
 
 
 def call_ops(sh: gen.LinearShape, M: int) -> int:
@@ -159,7 +180,7 @@ def run_reference(args):
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64/int64", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"qwen3-32b linear stack, decode M={M}, bounded sample: {sample}", "bits": BITS},
         "cpu_baseline": {"value": val, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -322,10 +343,25 @@ def run_ours(args):
     achieved = k_bytes / (k_ms * 1e-3) / 1e9 if k_ms > 0 else None
     roofline = {"bound": "hbm", "kernel": "umma_w1a_kernel (tcgen05 kind::i8 contraction), decode stack",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
-                "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "traffic": None,
+                "frac": (achieved / peaks["hbm_gbs"]) if achieved else None,
+                "traffic": measured_traffic("decode", k_bytes / k_n) if k_n else None,
                 "launches_per_step": k_n, "avg_launch_us": (k_ms / k_n * 1e3) if k_n else None,
+                "algorithmic_bytes_per_launch": (k_bytes / k_n) if k_n else None,
                 "algorithmic_bytes_per_step": k_bytes}
     del graph
+
+    # the other decode batch sizes of the workload, whole-step only
+    decode_other = {}
+    for Mo in args.decode_also:
+        if Mo == M:
+            continue
+        xs_o, outs_o, ws_o = make_io(Mo)
+        graph_o, _ = capture(xs_o, outs_o, ws_o)
+        ms_o = timed(graph_o.replay, max(3, args.steps // 2), 3) / max(3, args.steps // 2)
+        bytes_o = args.layers * sum(call_bytes(sh, Mo) for sh in shapes)
+        decode_other[f"M{Mo}"] = {"value": world * bytes_o / (ms_o * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms_o,
+                                  "status": bwla.bwla_check_status(ws_o)}
+        del graph_o
 
     # ------------------------------ prefill ------------------------------
     prefill = None
@@ -378,7 +414,7 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "int8 x int1 -> int32 (fp32 rotation, bf16 out)", "data": "synthetic",
+            "vs_baseline": None, "dtype": "int8", "dtype_detail": "int8 codes x 1-bit signs -> int32 (fp32 rotation, bf16 in/out)", "data": "synthetic",
             "config": {"workload": f"qwen3-32b linear stack (config 4): {args.layers} layers x 7 W1A6 linears, decode M={M}, "
                                    f"rank 64, all weights resident ({step_bytes / 1e9:.2f} GB algorithmic bytes per step)",
                        "bits": BITS, "l2": "inputs larger than L2 (weights of all layers are streamed every step)",
@@ -387,7 +423,7 @@ def run_ours(args):
                                       "ms_per_step": e2e_ms / args.steps},
             "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
             "kernel_ms_per_step": {k: round(v[0], 4) for k, v in prof.items()},
-            "cpu_baseline": cpu, "prefill": prefill, "device_status": status,
+            "cpu_baseline": cpu, "decode_other_batches": decode_other, "prefill": prefill, "device_status": status,
         }
         print(json.dumps(line))
     if world > 1:
@@ -402,6 +438,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=gen.QWEN3_32B_LAYERS)
     ap.add_argument("--decode-m", type=int, default=16)
+    ap.add_argument("--decode-also", type=int, nargs="*", default=[1, 64], help="further decode batch sizes (whole-step time only)")
     ap.add_argument("--prefill-m", type=int, default=2048)
     ap.add_argument("--prefill-layers", type=int, default=0, help="layers in the prefill step (0 = all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
