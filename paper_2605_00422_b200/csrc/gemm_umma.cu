@@ -42,7 +42,8 @@ constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
 constexpr int kBlockK = 128;             // K per code sub-block / per tensor-memory A stage
 constexpr int kFirstExpander = 192;      // warps 0, 1: TMA; warps 2..5: MMA issue; warps 6..13: expand + epilogue
-constexpr uint32_t kWaitLimit = 1u << 20;   // polls per wait before giving up (tens of milliseconds)
+constexpr uint32_t kParkNs = 4000;          // longest a single poll of a barrier may park its thread
+constexpr uint32_t kWaitLimit = 1u << 15;   // polls per wait before giving up (about a tenth of a second when nothing arrives)
 
 struct UmmaParams {
     int M, N, K;
@@ -99,8 +100,27 @@ struct UmmaCfg {
 #ifdef BWLA_TRACE
 #define BWLA_STAMP(i) do { if (p.status && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
         reinterpret_cast<long long*>(p.status + 16)[i] = clock64(); } while (0)
+// and start / first weights / K loop done / accumulators ready / exit of every CTA on the GPU-wide nanosecond timer
+__device__ unsigned long long g_cta_times[4096 * 8];
+__device__ __forceinline__ unsigned long long global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define BWLA_CTA_STAMP(i) do { const unsigned lb = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); \
+        if (lb < 4096) g_cta_times[lb * 8 + (i)] = global_ns(); } while (0)
+// clock stamps of the ring of CTA (0,0,0): [w][i][.] for w < 8 expander warp w's i-th own k-block (0 before the wait
+// for weights, 1 words loaded, 2 before the wait for the stage, 3 stage free, 4 stored, 5 handed over); for w = 8, 9
+// the issuing threads' i-th own k-block (0 before the wait for codes, 1 codes there, 2 operand there, 3 issued)
+__device__ long long g_ring_trace[10 * 32 * 8];
+#define BWLA_RING(who, i, j) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (i) < 32) \
+        g_ring_trace[((who) * 32 + (i)) * 8 + (j)] = clock64(); } while (0)
+extern "C" int bwla_trace_ring(long long* host) {
+    return cudaMemcpyFromSymbol(host, g_ring_trace, sizeof(g_ring_trace)) == cudaSuccess ? 0 : -4;
+}
+extern "C" int bwla_trace_ctas(unsigned long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, g_cta_times, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -4;
+}
 #else
 #define BWLA_STAMP(i) do { } while (0)
+#define BWLA_CTA_STAMP(i) do { } while (0)
+#define BWLA_RING(who, i, j) do { } while (0)
 #endif
 
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
@@ -113,10 +133,11 @@ __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_fl
 }
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    // Each poll may park the thread for up to kParkNs while the phase is open: a warp that spun on the barrier would
+    // take issue slots from the expander warps that share its scheduler.
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
         if (*abort_flag) return false;
-        if (i > 8192) __nanosleep(64);             // a sleeping warp wakes up late: only back off on long waits
     }
     return false;
 }
@@ -180,7 +201,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     const int unit_end = (int)(((int64_t)(split + 1) * p.total_units) / p.splits);
     const bool lowrank = p.r > 0;
     const bool lowrank_here = lowrank && split == 0;   // the low-rank accumulator lives in the first CTA of a cluster
-    if (threadIdx.x == 0) BWLA_STAMP(0);
+    if (threadIdx.x == 0) { BWLA_STAMP(0); BWLA_CTA_STAMP(0); }
 
     auto sub_count = [&](int u) { return min(kUnitK / kBlockK, (p.K - u * kUnitK) / kBlockK); };
     // k-blocks this CTA contracts; every unit but the last of the matrix has eight
@@ -288,12 +309,15 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     const int sb = s % SUBS;
                     // every issuing thread sees each code stage filled before it releases it, whether or not one of
                     // the stage's k-blocks is its own: its release can then never run a whole ring ahead
+                    if (kb % NISS == iss) BWLA_RING(8 + iss, kb / NISS, 0);
                     if (sb == 0 && !wait_or_abort(&b_full[bs], bph, abort_flag)) { give_up(p.status, abort_flag, 0x30); ok = false; break; }
                     if (kb % NISS == iss) {
+                        BWLA_RING(8 + iss, kb / NISS, 1);
                         const int as = kb % AS;
                         const uint32_t aph = (uint32_t)(kb / AS) & 1u;
                         if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
                         if (kb == 0) BWLA_STAMP(8);
+                        BWLA_RING(8 + iss, kb / NISS, 2);
                         tc_fence_after();
                         const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
                         const uint32_t a_addr = tmem_base + L::A_COL + 32 * as;
@@ -301,6 +325,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         for (int i = 0; i < 4; ++i)
                             mma_i8_ts(d_addr, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, (kb < NISS && i == 0) ? 0u : 1u);
                         tc_commit(&a_empty[as]);
+                        BWLA_RING(8 + iss, kb / NISS, 3);
                     }
                     if (sb == SUBS - 1 || s == ns - 1) {
                         // this thread is done with the code stage once its MMAs so far have completed
@@ -357,8 +382,9 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         bool ok = true;
         int kb0 = 0;                                   // k-block index of sub-block 0 of the current unit
         for (int u = unit_begin; u < unit_end && ok; ++u) {
+            if (lane == 0) BWLA_RING(warp - 6, (kb0 + ((part - kb0) % EW + EW) % EW) / EW, 0);
             if (!warp_wait(&w_full[ws], wph, abort_flag, lane)) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
-            if (e == 64 && u == unit_begin) BWLA_STAMP(3);
+            if (e == 64 && u == unit_begin) { BWLA_STAMP(3); BWLA_CTA_STAMP(1); }
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
             const int s_first = ((part - kb0) % EW + EW) % EW;      // kb0 + s_first = part (mod EW)
@@ -377,18 +403,23 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 const int as = kb % AS;
                 const uint32_t aph = (uint32_t)(kb / AS) & 1u;
                 uint32_t v[32];
+                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 1);
                 const uint32_t w[4] = {w4[i].x, w4[i].y, w4[i].z, w4[i].w};
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
+                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 2);
                 if (!warp_wait(&a_empty[as], aph ^ 1, abort_flag, lane)) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
+                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 3);
                 tc_fence_after();
                 tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
                 tc_wait_st();
+                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 4);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&a_full[as]);
+                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 5);
             }
             // The stage is released only here, after every word loaded from it has gone through the expansion: an
             // arrive placed right behind the loads let the copy of a later unit overwrite words not yet read.
@@ -397,7 +428,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (++ws == WS) { ws = 0; wph ^= 1; }
             kb0 += ns;
         }
-        if (e == 64) BWLA_STAMP(4);
+        if (e == 64) { BWLA_STAMP(4); BWLA_CTA_STAMP(2); }
         // the stores of the epilogue come after the preceding kernel; the per-token scales and code sums it wrote were
         // staged in shared memory by warp 1 while the K loop ran
         griddep_wait();
@@ -405,7 +436,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         if (ok) {
             if (!warp_wait(d_full, 0, abort_flag, lane)) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
-        if (e == 64) BWLA_STAMP(5);
+        if (e == 64) { BWLA_STAMP(5); BWLA_CTA_STAMP(3); }
         if (ok) {
             tc_fence_after();
             const int n = n0 + row;
@@ -486,7 +517,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
         }
     }
-    if (threadIdx.x == kFirstExpander) BWLA_STAMP(6);
+    if (threadIdx.x == kFirstExpander) { BWLA_STAMP(6); BWLA_CTA_STAMP(4); }
     tc_fence_before();
     __syncthreads();
     if (p.splits > 1) {
@@ -544,7 +575,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
-        if (lane == 0) BWLA_STAMP(7);
+        if (lane == 0) { BWLA_STAMP(7); BWLA_CTA_STAMP(5); }
     }
 }
 

@@ -7,18 +7,20 @@
 // (Sec. 3.1: R = R1 (x) R2 evaluated as two small contractions on the reshaped vector; Sec. 4.1: per-token
 // activation quantisation; Sec. 3.2: W x = (W - M) x + A (B x).)
 //
-// Rotation blocks: a thread-block cluster of C CTAs owns one token.  CTA c owns a slab of rows of X: it computes
-// that slab of Z and stores it into the full-size Z buffer of every CTA of the cluster (distributed shared memory),
-// then computes the same slab of rows of Y from the full Z, exchanges its absmax and its code sum the same way and
-// quantises its slab.  With few tokens this spreads one token's 2*K*(n1+n2) flops over C SMs; with many tokens C = 1.
-// X, Z and Y never touch HBM.  Both contractions are register-tiled 4x4 fp32 FMA loops; codes leave as 128-bit stores.
+// Rotation blocks: a thread-block cluster of C CTAs owns one token.  With many tokens C = 1 and the CTA evaluates
+// Z = X * P2, Y = P1^T * Z in chunks.  With few tokens C > 1 spreads one token's 2*K*(n1+n2) flops over C SMs: CTA c
+// owns a slab of rows of Y and evaluates the product in the other order, Z' = (P1^T X)[slab], Y[slab] = Z' * P2,
+// which needs all of x (a few KB) but nothing from the other CTAs; only the absmax and the code sums cross the
+// cluster (distributed shared memory).  X, Z and Y never touch HBM.  Both contractions are register-tiled fp32 FMA
+// loops; codes leave as 128-bit stores.
 //
 // Low-rank blocks (after the rotation blocks in the same grid): each reduces two rows of V against a tile of 16
 // tokens with 128-bit loads and writes T split into three bf16 terms (T = hi + mid + lo, all 24 bits of the fp32 sum), the form
 // the tensor-core epilogue of the contraction consumes.
 //
-// The kernel is launched with programmatic stream serialisation: everything up to the first global store may
-// overlap the preceding kernel of the stream; every block waits for that kernel before it stores anything.
+// The kernel is launched with programmatic stream serialisation.  The activations may be the output of the
+// preceding kernel of the stream, so only the layer's own constants (P1, P2, rows of V) are fetched before that
+// kernel has finished; x is read, and everything is stored, after it.
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -31,7 +33,7 @@ namespace bwla {
 using namespace ptx;
 
 constexpr int kLrMaxWarps = 16;   // blocks have at most 512 threads
-constexpr int kPrologueSmemFloats = 55 * 1024;   // dynamic shared memory of a prologue block, in floats (220 KB; about 6 KB are static)
+constexpr int kPrologueSmemFloats = 57728;   // dynamic shared memory of a prologue block, in floats (225.5 KB; static use is under 1 KB)
 
 // Optional phase timeline of rotation block 0 for tuning (compiled out by default).
 #ifdef BWLA_TRACE
@@ -40,8 +42,15 @@ __device__ long long g_prologue_trace[32];
 extern "C" int bwla_trace_prologue(long long* host32) {
     return cudaMemcpyFromSymbol(host32, g_prologue_trace, sizeof(long long) * 32) == cudaSuccess ? 0 : -4;
 }
+__device__ unsigned long long g_prologue_block_times[1024 * 4];
+__device__ __forceinline__ unsigned long long prologue_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define BWLA_PBLOCK(i) do { if (threadIdx.x == 0 && blockIdx.x < 1024) g_prologue_block_times[blockIdx.x * 4 + (i)] = prologue_ns(); } while (0)
+extern "C" int bwla_trace_prologue_blocks(unsigned long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, g_prologue_block_times, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -4;
+}
 #else
 #define BWLA_PSTAMP(i) do { } while (0)
+#define BWLA_PBLOCK(i) do { } while (0)
 #endif
 
 struct PrologueParams {
@@ -58,9 +67,13 @@ struct PrologueParams {
     int prefetch;       // 1: all of P2 and this CTA's columns of P1 are fetched at the start, with x
     int p1_cap;         // floats reserved for the prefetched columns of P1
     int tr1, tr2;       // rows per thread in the two contractions
+    int split_y;        // 1 (C > 1): each CTA evaluates its rows of Y from all of x, nothing but absmax is exchanged
+    int sp_tr, sp_rp;   // split_y: rows per thread tile (4 or 8); slab rows rounded up to it (row stride of P1s and Zt)
+    int sp_s;           // split_y: slices the contraction depth is cut into (partial sums are added afterwards)
     // low-rank
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
-    int lr_wide;        // 1: blocks of 8 rows of V x 8 tokens (many tokens), 0: 2 rows x 16 tokens
+    int lr_wide;        // rows of V x tokens per low-rank block: 0: 2 x 16, 1: 8 x 8 (many tokens), 2: 2 x 8 (few tokens)
+    int lr_stage;       // 1: a low-rank block copies its rows of V into shared memory before it waits for x
 };
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -75,9 +88,6 @@ __device__ __forceinline__ int warp_sum(int v) {
     return v;
 }
 
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float4 v) {
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
 __device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -87,11 +97,11 @@ __device__ __forceinline__ int slab_begin(int c, int C, int n1, int gran) {
     return (int)(((int64_t)n1 * c / C) / gran * gran);
 }
 
-// Z[rows of this slab][dc .. dc+cw) = X slab * P2[:, dc .. dc+cw).  Ps holds that chunk of P2 (row stride cw).
-// Each thread owns TR rows x 4 columns; the sum runs over b in increasing order.
+// Z[0 .. rows)[dc .. dc+cw) = X * P2[:, dc .. dc+cw) for the `rows` rows of X at Xs.  Ps holds that chunk of P2 (row
+// stride cw).  Each thread owns TR rows x 4 columns; the sum runs over b in increasing order.
 template <int TR>
 __device__ __forceinline__ void stage1_chunk(const float* __restrict__ Xs, int rows, int n2, const float* __restrict__ Ps,
-                                             int dc, int cw, float* Zf, int a_lo, int C) {
+                                             int dc, int cw, float* Zf, float* amax = nullptr) {
     const int ct = cw >> 2;
     const int tiles = ((rows + TR - 1) / TR) * ct;
     for (int tile = threadIdx.x; tile < tiles; tile += blockDim.x) {
@@ -127,14 +137,9 @@ __device__ __forceinline__ void stage1_chunk(const float* __restrict__ Xs, int r
 #pragma unroll
         for (int i = 0; i < TR; ++i)
             if (r0 + i < rows) {
-                float* dst = Zf + (a_lo + r0 + i) * n2 + dc + dl;
                 const float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                if (C == 1) {
-                    *reinterpret_cast<float4*>(dst) = v;
-                } else {
-                    const uint32_t local = smem_u32(dst);
-                    for (int c = 0; c < C; ++c) st_cluster_v4(map_shared_rank(local, c), v);
-                }
+                if (amax) *amax = fmaxf(*amax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+                *reinterpret_cast<float4*>(Zf + (r0 + i) * n2 + dc + dl) = v;
             }
     }
 }
@@ -190,6 +195,111 @@ __device__ __forceinline__ void stage2_chunk(const float* __restrict__ Zf, int n
 // ---------------------------------------------------------------------------------------------
 // rotation + quantiser
 // ---------------------------------------------------------------------------------------------
+// Partial sums of C[r][d] = sum_k A[k][r] * B[k][d] for a slab of rp rows (A: [depth][rp], zero beyond the real
+// rows) and n2 columns.  A work item is a tile of TR rows x 4 columns over one of S slices of the depth; items are
+// dealt to threads with the column index fastest, so a warp reads one run of B and broadcasts A.  The sums over k run
+// in increasing order inside a slice.  part: [S][rp][n2].  B is fp32, or bf16 when B_BF16 (the activations).
+template <int TR, bool B_BF16>
+__device__ __forceinline__ void slab_partial(const float* __restrict__ A, int rp, const void* __restrict__ B, int depth,
+                                             int n2, int S, float* __restrict__ part) {
+    const int cq = n2 >> 2;
+    const int tiles = (rp / TR) * cq;
+    const int items = tiles * S;
+    for (int item = threadIdx.x; item < items; item += blockDim.x) {
+        const int sl = item / tiles, tile = item - sl * tiles;
+        const int mt = tile / cq, d0 = (tile - mt * cq) << 2;
+        const int k0 = (int)((int64_t)depth * sl / S), k1 = (int)((int64_t)depth * (sl + 1) / S);
+        float acc[TR][4];
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        const float* ap = A + mt * TR;
+#pragma unroll 4
+        for (int k = k0; k < k1; ++k) {
+            float4 bv;
+            if (B_BF16) {
+                const uint2 w = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(B) + (size_t)k * n2 + d0);
+                bv = make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u),
+                                 __uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+            } else {
+                bv = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(B) + (size_t)k * n2 + d0);
+            }
+            float a[TR];
+#pragma unroll
+            for (int i = 0; i < TR; i += 4) {
+                const float4 v = *reinterpret_cast<const float4*>(ap + (size_t)k * rp + i);
+                a[i] = v.x; a[i + 1] = v.y; a[i + 2] = v.z; a[i + 3] = v.w;
+            }
+#pragma unroll
+            for (int i = 0; i < TR; ++i) {
+                acc[i][0] = fmaf(a[i], bv.x, acc[i][0]);
+                acc[i][1] = fmaf(a[i], bv.y, acc[i][1]);
+                acc[i][2] = fmaf(a[i], bv.z, acc[i][2]);
+                acc[i][3] = fmaf(a[i], bv.w, acc[i][3]);
+            }
+        }
+        float* dst = part + ((size_t)sl * rp + mt * TR) * n2 + d0;
+#pragma unroll
+        for (int i = 0; i < TR; ++i)
+            *reinterpret_cast<float4*>(dst + (size_t)i * n2) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    }
+}
+
+// Adds the S partial sums.  TRANSPOSED: the result goes to out[d][r] (row stride rp), the A operand of the next
+// contraction; otherwise to out[r][d] (row stride n2), only for the real rows, and the largest magnitude is returned.
+template <bool TRANSPOSED>
+__device__ __forceinline__ float slab_reduce(const float* __restrict__ part, int rp, int rows, int n2, int S, float* out) {
+    float amax = 0.f;
+    const int cq = n2 >> 2;
+    const int quads = (TRANSPOSED ? rp : rows) * cq;
+    for (int o = threadIdx.x; o < quads; o += blockDim.x) {
+        const int r = o / cq, d0 = (o - r * cq) << 2;
+        float4 v = *reinterpret_cast<const float4*>(part + (size_t)r * n2 + d0);
+        for (int sl = 1; sl < S; ++sl) {
+            const float4 w = *reinterpret_cast<const float4*>(part + ((size_t)sl * rp + r) * n2 + d0);
+            v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+        }
+        if (TRANSPOSED) {
+            out[(size_t)(d0 + 0) * rp + r] = v.x; out[(size_t)(d0 + 1) * rp + r] = v.y;
+            out[(size_t)(d0 + 2) * rp + r] = v.z; out[(size_t)(d0 + 3) * rp + r] = v.w;
+        } else {
+            *reinterpret_cast<float4*>(out + (size_t)r * n2 + d0) = v;
+            amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+        }
+    }
+    return amax;
+}
+
+// x_t[first .. first+len) -> fp32 in shared memory
+__device__ __forceinline__ void load_x(const __nv_bfloat16* __restrict__ xt, int len, float* Xs) {
+    if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0 && (len & 7) == 0) {
+        const uint4* xv = reinterpret_cast<const uint4*>(xt);
+        for (int i = threadIdx.x; i < (len >> 3); i += blockDim.x) {
+            const uint4 v = __ldg(xv + i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            float f[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                f[2 * j] = __uint_as_float(w[j] << 16);
+                f[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+            }
+            *reinterpret_cast<float4*>(Xs + 8 * i) = make_float4(f[0], f[1], f[2], f[3]);
+            *reinterpret_cast<float4*>(Xs + 8 * i + 4) = make_float4(f[4], f[5], f[6], f[7]);
+        }
+    } else {
+        for (int k = threadIdx.x; k < len; k += blockDim.x) Xs[k] = __bfloat162float(xt[k]);
+    }
+}
+
+// columns [a_lo, a_lo+rows) of P1 -> shared memory, row stride cwp (padding zero)
+__device__ __forceinline__ void load_p1_columns(const float* __restrict__ P1, int n1, int a_lo, int rows, int cwp, float* dst) {
+    for (int i = threadIdx.x; i < n1 * cwp; i += blockDim.x) {
+        const int a = i / cwp, j = i - a * cwp;
+        dst[i] = j < rows ? __ldg(P1 + (size_t)a * n1 + a_lo + j) : 0.f;
+    }
+}
+
 __device__ void rotate_role(const PrologueParams& p, float* smem) {
     const int C = p.C;
     const int rank = C > 1 ? (int)cluster_ctarank() : 0;
@@ -197,59 +307,82 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     const int n1 = p.n1, n2 = p.n2, K = p.K;
     const int a_lo = slab_begin(rank, C, n1, p.row_gran), a_hi = slab_begin(rank + 1, C, n1, p.row_gran);
     const int rows = a_hi - a_lo;
-    float* Xs = smem;                          // this CTA's slab of X, later of Y
-    float* Zf = smem + p.slab_cap;             // all of Z
-    float* P1s = Zf + K + p.ps_cap;            // this CTA's columns of P1 when they are prefetched
-    float* slots = P1s + p.p1_cap;             // [0..7] absmax per rank, [8..15] code sum per rank (int)
+    float* Xs = smem;                          // this CTA's rows of Y end up here in every mode
+    float* slots;                              // [0..7] absmax per rank, [8..15] code sum per rank (int)
     __shared__ float red_max[32];
     __shared__ int red_sum;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int qmax = (1 << (p.bits - 1)) - 1;
+    float amax = 0.f;
+    if (threadIdx.x == 0) red_sum = 0;
 
     BWLA_PSTAMP(0);
-    // ---- this slab of x_t -> fp32 in shared memory
-    {
-        const __nv_bfloat16* xt = p.x + t * p.ldx + (int64_t)a_lo * n2;
-        const int len = rows * n2;
-        if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0 && (len & 7) == 0) {
-            const uint4* xv = reinterpret_cast<const uint4*>(xt);
-            for (int i = threadIdx.x; i < (len >> 3); i += blockDim.x) {
-                const uint4 v = __ldg(xv + i);
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                float f[8];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    f[2 * j] = __uint_as_float(w[j] << 16);
-                    f[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-                }
-                *reinterpret_cast<float4*>(Xs + 8 * i) = make_float4(f[0], f[1], f[2], f[3]);
-                *reinterpret_cast<float4*>(Xs + 8 * i + 4) = make_float4(f[4], f[5], f[6], f[7]);
-            }
-        } else {
-            for (int k = threadIdx.x; k < len; k += blockDim.x) Xs[k] = __bfloat162float(xt[k]);
-        }
-    }
-    if (p.prefetch) {
-        // one round trip for everything this block reads: P2 and the needed columns of P1 are requested with x
-        float* Ps = Zf + K;
+    if (p.split_y) {
+        // ---- few tokens: this CTA's rows of Y from all of x; nothing but absmax and code sums is exchanged
+        const int rp = p.sp_rp, S = p.sp_s;
+        __nv_bfloat16* Xh = reinterpret_cast<__nv_bfloat16*>(smem);   // all of x_t as it comes; later this CTA's rows of Y (fp32)
+        float* Zt = smem + (K >> 1);           // Z'^T: [n2][rp], Z' = rows [a_lo, a_hi) of P1^T X
+        float* P2s = Zt + n2 * rp;             // all of P2
+        float* P1s = P2s + p.ps_cap;           // columns [a_lo, a_hi) of P1: [n1][rp]
+        float* part = P1s + p.p1_cap;          // [S][rp][n2] partial sums
+        slots = part + S * rp * n2;
+        // the layer's constants do not depend on the preceding kernel
         for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x)
-            *reinterpret_cast<float4*>(Ps + 4 * i) = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
-        const int cwp = (rows + 3) & ~3;
-        for (int i = threadIdx.x; i < n1 * cwp; i += blockDim.x) {
-            const int a = i / cwp, j = i - a * cwp;
-            P1s[i] = j < rows ? __ldg(p.P1 + (size_t)a * n1 + a_lo + j) : 0.f;
+            *reinterpret_cast<float4*>(P2s + 4 * i) = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
+        load_p1_columns(p.P1, n1, a_lo, rows, rp, P1s);
+        cluster_arrive_release();              // "this CTA is running": waited for before the first remote store
+        griddep_launch_dependents();
+        griddep_wait();                        // x may be the output of the preceding kernel
+        BWLA_PSTAMP(1); BWLA_PBLOCK(2);
+        {
+            const __nv_bfloat16* xt = p.x + t * p.ldx;
+            if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0) {
+                for (int i = threadIdx.x; i < (K >> 3); i += blockDim.x)
+                    reinterpret_cast<uint4*>(Xh)[i] = __ldg(reinterpret_cast<const uint4*>(xt) + i);
+            } else {
+                for (int k = threadIdx.x; k < K; k += blockDim.x) Xh[k] = xt[k];
+            }
         }
-    }
-    if (threadIdx.x == 0) red_sum = 0;
-    // every CTA of the cluster must be running before its shared memory is written from outside
-    if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else __syncthreads();
-    griddep_launch_dependents();
-    BWLA_PSTAMP(1);
-
-    float amax = 0.f;
-    if ((n2 & 3) == 0) {
+        __syncthreads();
+        BWLA_PSTAMP(2);
+        if (p.sp_tr == 8) slab_partial<8, true>(P1s, rp, Xh, n1, n2, S, part);
+        else slab_partial<4, true>(P1s, rp, Xh, n1, n2, S, part);
+        __syncthreads();
+        slab_reduce<true>(part, rp, rows, n2, S, Zt);
+        __syncthreads();
+        BWLA_PSTAMP(3);
+#ifdef BWLA_TRACE_REPEAT
+        BWLA_PSTAMP(11);
+        if (p.sp_tr == 8) slab_partial<8, true>(P1s, rp, Xh, n1, n2, S, part);
+        else slab_partial<4, true>(P1s, rp, Xh, n1, n2, S, part);
+        __syncthreads();
+        BWLA_PSTAMP(12);
+        slab_reduce<true>(part, rp, rows, n2, S, Zt);
+        __syncthreads();
+        BWLA_PSTAMP(13);
+#endif
+        if (p.sp_tr == 8) slab_partial<8, false>(Zt, rp, P2s, n2, n2, S, part);
+        else slab_partial<4, false>(Zt, rp, P2s, n2, n2, S, part);
+        __syncthreads();
+        amax = slab_reduce<false>(part, rp, rows, n2, S, Xs);
+        BWLA_PSTAMP(4);
+        cluster_wait_acquire();
+        BWLA_PSTAMP(5);
+    } else if ((n2 & 3) == 0) {
+        // ---- one CTA per token: Z = X * P2, Y = P1^T * Z, the factors staged chunk by chunk
+        float* Zf = smem + p.slab_cap;         // all of Z
         float* Ps = Zf + K;                    // staged chunk of P2, later of P1
-        // ---- Z slab = X slab * P2, one chunk of columns of P2 at a time, stored into every CTA's full Z
+        float* P1s = Ps + p.ps_cap;            // all of P1 when it is prefetched
+        slots = P1s + p.p1_cap;
+        if (p.prefetch) {
+            for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x)
+                *reinterpret_cast<float4*>(Ps + 4 * i) = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
+            load_p1_columns(p.P1, n1, 0, n1, (n1 + 3) & ~3, P1s);
+        }
+        griddep_launch_dependents();
+        griddep_wait();                        // x may be the output of the preceding kernel
+        load_x(p.x + t * p.ldx, K, Xs);
+        BWLA_PSTAMP(1);
         for (int dc = 0; dc < n2; dc += p.ch1) {
             const int cw = min(p.ch1, n2 - dc);
             if (!p.prefetch) for (int i = threadIdx.x; i < n2 * (cw >> 2); i += blockDim.x) {
@@ -259,25 +392,19 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             __syncthreads();
             BWLA_PSTAMP(2);
             switch (p.tr1) {
-                case 8: stage1_chunk<8>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
-                case 4: stage1_chunk<4>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
-                case 2: stage1_chunk<2>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
-                default: stage1_chunk<1>(Xs, rows, n2, Ps, dc, cw, Zf, a_lo, C); break;
+                case 8: stage1_chunk<8>(Xs, n1, n2, Ps, dc, cw, Zf); break;
+                case 4: stage1_chunk<4>(Xs, n1, n2, Ps, dc, cw, Zf); break;
+                case 2: stage1_chunk<2>(Xs, n1, n2, Ps, dc, cw, Zf); break;
+                default: stage1_chunk<1>(Xs, n1, n2, Ps, dc, cw, Zf); break;
             }
             __syncthreads();
         }
         BWLA_PSTAMP(3);
-        if (C > 1) { cluster_arrive_release(); cluster_wait_acquire(); }
-        BWLA_PSTAMP(4);
-        // ---- Y slab = (P1^T * Z) rows [a_lo, a_hi), one chunk of output rows (columns of P1) at a time;
-        //      Y overwrites the X slab, which is dead now
-        for (int c0 = 0; c0 < rows; c0 += p.ch2) {
-            const int cw = min(p.ch2, rows - c0), cwp = (cw + 3) & ~3;
+        // Y overwrites X, which is dead now; one chunk of output rows (columns of P1) at a time
+        for (int c0 = 0; c0 < n1; c0 += p.ch2) {
+            const int cw = min(p.ch2, n1 - c0), cwp = (cw + 3) & ~3;
             const float* Pc = p.prefetch ? P1s : Ps;
-            if (!p.prefetch) for (int i = threadIdx.x; i < n1 * cwp; i += blockDim.x) {
-                const int a = i / cwp, j = i - a * cwp;
-                Ps[i] = j < cw ? __ldg(p.P1 + (size_t)a * n1 + a_lo + c0 + j) : 0.f;
-            }
+            if (!p.prefetch) load_p1_columns(p.P1, n1, c0, cw, cwp, Ps);
             __syncthreads();
             BWLA_PSTAMP(5);
             switch (p.tr2) {
@@ -289,7 +416,13 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             __syncthreads();
         }
     } else {
-        // generic shapes (n2 not a multiple of 4; C == 1): one output per thread step
+        // generic shapes (n2 not a multiple of 4; one CTA per token): one output per thread step
+        float* Zf = smem + p.slab_cap;
+        slots = Zf + K;
+        griddep_launch_dependents();
+        griddep_wait();
+        load_x(p.x + t * p.ldx, K, Xs);
+        __syncthreads();
         for (int o = threadIdx.x; o < K; o += blockDim.x) {
             const int a = o / n2, d = o - a * n2;
             float s = 0.f;
@@ -397,32 +530,45 @@ __device__ __forceinline__ float dot8(float acc, const uint4& v, const uint4& xv
 // One block reduces R rows of V against T tokens (R x T accumulators per thread, threads stride over K).  Few tokens:
 // R = 2, T = 16 (many blocks).  Many tokens: R = T = 8, which reads each operand four times less often from L2.
 template <int R, int T>
-__device__ void lowrank_role(const PrologueParams& p, int b) {
+__device__ void lowrank_role(const PrologueParams& p, int b, float* smem) {
     const int jblocks = p.lr_cols / R;
     const int jb = b % jblocks;
     const int64_t t0 = (int64_t)(b / jblocks) * T;
     if (t0 >= p.M) return;
     const int j0 = jb * R;
     const int nt = (int)min((int64_t)T, p.M - t0);
+    float (*red)[R * T] = reinterpret_cast<float (*)[R * T]>(smem);            // [kLrMaxWarps][R * T]
+    const uint4* vs = reinterpret_cast<const uint4*>(smem + kLrMaxWarps * R * T);   // staged rows of V, [R][K / 8]
     float acc[R][T];
 #pragma unroll
     for (int j = 0; j < R; ++j)
 #pragma unroll
         for (int i = 0; i < T; ++i) acc[j][i] = 0.f;
+    const int K = p.K;
+    const int nr = min(R, p.r - j0);                          // rows of V this block really has (<= 0: padding only)
+    const bool vec = ((reinterpret_cast<uintptr_t>(p.V) | reinterpret_cast<uintptr_t>(p.x)) & 15) == 0 && (p.ldx & 7) == 0 && (K & 7) == 0;
+    const bool staged = p.lr_stage && vec && nr > 0;
+    if (staged) {
+        // V is a constant of the layer: in shared memory before the activations exist
+        uint4* dst = reinterpret_cast<uint4*>(smem + kLrMaxWarps * R * T);
+        for (int j = 0; j < R; ++j) {
+            const uint4* src = reinterpret_cast<const uint4*>(p.V + (int64_t)(j0 + min(j, nr - 1)) * K);
+            for (int kc = threadIdx.x; kc < (K >> 3); kc += blockDim.x) dst[j * (K >> 3) + kc] = __ldg(src + kc);
+        }
+    }
     griddep_launch_dependents();
-    if (j0 < p.r) {
-        const int K = p.K;
-        const int nr = min(R, p.r - j0);                      // rows of V this block really has
+    griddep_wait();                                           // x may be the output of the preceding kernel
+    BWLA_PBLOCK(2);
+    if (nr > 0) {
         const __nv_bfloat16* vrow[R];
 #pragma unroll
         for (int j = 0; j < R; ++j) vrow[j] = p.V + (int64_t)(j0 + min(j, nr - 1)) * K;
         const __nv_bfloat16* xt = p.x + t0 * p.ldx;
-        const bool vec = ((reinterpret_cast<uintptr_t>(p.V) | reinterpret_cast<uintptr_t>(p.x)) & 15) == 0 && (p.ldx & 7) == 0;
         if (vec) {
             for (int kc = threadIdx.x; kc < (K >> 3); kc += blockDim.x) {
                 uint4 a[R];
 #pragma unroll
-                for (int j = 0; j < R; ++j) a[j] = __ldg(reinterpret_cast<const uint4*>(vrow[j]) + kc);
+                for (int j = 0; j < R; ++j) a[j] = staged ? vs[j * (K >> 3) + kc] : __ldg(reinterpret_cast<const uint4*>(vrow[j]) + kc);
 #pragma unroll
                 for (int tt = 0; tt < T; ++tt) {
                     if (tt < nt) {
@@ -454,7 +600,6 @@ __device__ void lowrank_role(const PrologueParams& p, int b) {
                 for (int i = 0; i < T; ++i) acc[j][i] = 0.f;
             }
     }
-    __shared__ float red[kLrMaxWarps][R * T];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int j = 0; j < R; ++j)
@@ -466,7 +611,6 @@ __device__ void lowrank_role(const PrologueParams& p, int b) {
             if (lane == 0) red[warp][j * T + i] = v;
         }
     __syncthreads();
-    griddep_wait();
     for (int o = threadIdx.x; o < R * T; o += blockDim.x) {
         const int j = o / T, i = o % T;
         if (i < nt) {
@@ -487,9 +631,12 @@ __device__ void lowrank_role(const PrologueParams& p, int b) {
 
 __global__ void prologue_kernel(PrologueParams p) {
     extern __shared__ __align__(16) float smem[];
+    BWLA_PBLOCK(0);
     if ((int)blockIdx.x < p.rot_blocks) rotate_role(p, smem);
-    else if (p.lr_wide) lowrank_role<8, 8>(p, (int)blockIdx.x - p.rot_blocks);
-    else lowrank_role<2, 16>(p, (int)blockIdx.x - p.rot_blocks);
+    else if (p.lr_wide == 1) lowrank_role<8, 8>(p, (int)blockIdx.x - p.rot_blocks, smem);
+    else if (p.lr_wide == 2) lowrank_role<2, 8>(p, (int)blockIdx.x - p.rot_blocks, smem);
+    else lowrank_role<2, 16>(p, (int)blockIdx.x - p.rot_blocks, smem);
+    BWLA_PBLOCK(1);
 }
 
 // How many clusters of `c` prologue blocks (threads, dynamic shared memory) the device holds at once; cached.
@@ -548,7 +695,37 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                 cap = cap > (hi - lo) ? cap : (hi - lo);
             }
             p.C = c; p.rot_blocks = (int)(M * c); p.row_gran = gran; p.slab_cap = (cap * n2 + 3) / 4 * 4;
-            p.prefetch = 0; p.p1_cap = 0;
+            p.prefetch = 0; p.p1_cap = 0; p.split_y = 0;
+            auto pick = [](int rows, int cols4, int want_tiles) {
+                for (int tr = 8; tr > 1; tr >>= 1)
+                    if (((rows + tr - 1) / tr) * cols4 >= want_tiles) return tr;
+                return 1;
+            };
+            if (c > 1) {
+                // all of x (bf16), this CTA's rows of Z' (transposed), all of P2, this CTA's columns of P1, partial sums
+                if ((K & 7) != 0) return false;
+                p.split_y = 1;
+                // thread tiles of 8 rows unless padding the slab to a multiple of 8 wastes more than 15 %
+                p.sp_tr = ((cap + 7) / 8 * 8) * 100 <= cap * 115 ? 8 : 4;
+                p.sp_rp = (cap + p.sp_tr - 1) / p.sp_tr * p.sp_tr;
+                p.ps_cap = n2 * n2 + 8;
+                p.p1_cap = n1 * p.sp_rp + 8;
+                p.ch1 = n2; p.ch2 = cap; p.tr1 = p.tr2 = p.sp_tr;
+                const int tiles = (p.sp_rp / p.sp_tr) * (n2 / 4);
+                const int64_t fixed = K / 2 + (int64_t)n2 * p.sp_rp + p.ps_cap + p.p1_cap + 16;
+                // cut the depth until there are about 512 work items, at least four steps per slice, while it fits
+                int S = 1;
+                while (S < 8 && tiles * S < 512 && std::min(n1, n2) / (S * 2) >= 4 &&
+                       fixed + (int64_t)(S * 2) * p.sp_rp * n2 <= kPrologueSmemFloats) S *= 2;
+                p.sp_s = S;
+                const int64_t need = fixed + (int64_t)S * p.sp_rp * n2;
+                if (need > kPrologueSmemFloats) return false;
+                const int items = tiles * S;
+                threads = (items + 31) / 32 * 32;
+                threads = threads < 256 ? 256 : (threads > 512 ? 512 : threads);
+                smem = (size_t)need * 4;
+                return true;
+            }
             if ((n2 & 3) == 0) {
                 // chunks of P2 (ch1 columns) and of P1 (ch2 columns) that fit beside the X slab and Z
                 const int64_t avail = kPrologueSmemFloats - p.slab_cap - K - 16 - 8;
@@ -566,17 +743,9 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                 if (nch1 == 1 && nch2 == 1 && (int64_t)n2 * n2 + 8 + p1_need <= avail) {
                     p.prefetch = 1; p.ps_cap = n2 * n2 + 8; p.p1_cap = (int)p1_need;
                 }
-                // rows per thread: as many as still leave a hundred-odd tiles
-                // (a block that shares a token wants its short chain done soon; a block that owns a whole token
-                // wants enough threads to hide latency)
-                const int want_tiles = c > 1 ? 128 : 256;
-                auto pick = [want_tiles](int rows, int cols4) {
-                    for (int tr = 8; tr > 1; tr >>= 1)
-                        if (((rows + tr - 1) / tr) * cols4 >= want_tiles) return tr;
-                    return 1;
-                };
-                p.tr1 = pick(cap, ch1 / 4);
-                p.tr2 = pick(ch2, n2 / 4);
+                // rows per thread: as many as still leave enough tiles to hide latency
+                p.tr1 = pick(cap, ch1 / 4, 256);
+                p.tr2 = pick(ch2, n2 / 4, 256);
                 const int tiles = std::max(((cap + p.tr1 - 1) / p.tr1) * (ch1 / 4), ((ch2 + p.tr2 - 1) / p.tr2) * (n2 / 4));
                 const int rounds = (tiles + 511) / 512;
                 threads = ((tiles + rounds - 1) / rounds + 31) / 32 * 32;
@@ -593,7 +762,7 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
             // spread one token over several SMs while there are few tokens and the token is worth splitting, as long as
             // every token's cluster is resident at once (a second wave of clusters would double the latency)
             const double flops = 2.0 * (double)K * (n1 + n2);
-            while (C < 8 && M * (C * 2) <= 160 && flops / (C * 2) >= 2.5e5 && n1 / (C * 2) >= gran) C *= 2;
+            while (C < 8 && M * (C * 2) <= 148 && flops / (C * 2) >= 1.5e5 && n1 / (C * 2) >= gran) C *= 2;
             for (; C > 1; C >>= 1) {
                 if (!plan(C)) continue;
                 if (clusters_resident(C, threads, smem) >= M) break;
@@ -605,8 +774,15 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     }
     int lr_blocks = 0;
     if (r > 0 && Thl) {
-        p.lr_wide = (M >= 64 && p.lr_cols % 8 == 0) ? 1 : 0;
-        lr_blocks = p.lr_wide ? (p.lr_cols / 8) * (int)((M + 7) / 8) : (p.lr_cols / 2) * (int)((M + 15) / 16);
+        // few tokens: small tiles, so that the handful of blocks is done sooner; many: tiles that re-read less
+        p.lr_wide = (M >= 64 && p.lr_cols % 8 == 0) ? 1 : (M <= 16 ? 2 : 0);
+        lr_blocks = p.lr_wide == 1 ? (p.lr_cols / 8) * (int)((M + 7) / 8)
+                  : p.lr_wide == 2 ? (p.lr_cols / 2) * (int)((M + 7) / 8) : (p.lr_cols / 2) * (int)((M + 15) / 16);
+        // shared memory of a low-rank block: per-warp partial sums, and its rows of V when those are staged (few tokens)
+        const size_t red_bytes = (size_t)kLrMaxWarps * 64 * 4;
+        const size_t stage_bytes = (size_t)2 * (size_t)K * 2;
+        p.lr_stage = (p.lr_wide != 1 && red_bytes + stage_bytes <= (size_t)kPrologueSmemFloats * 4) ? 1 : 0;
+        smem = std::max(smem, red_bytes + (p.lr_stage ? stage_bytes : 0));
     }
     int grid = p.rot_blocks + lr_blocks;
     grid = (grid + C - 1) / C * C;

@@ -139,6 +139,37 @@ def _run_layer_case(bwla, cfg, shape, M, bits, with_mu=False, direct_words=False
     return rep
 
 
+@pytest.mark.parametrize("M", [3, 16, 130])
+def test_output_of_one_layer_feeds_the_next_without_synchronisation(bwla, M):
+    """Two calls on one stream, the second reading what the first writes: stream order must hold although the kernels
+    are launched with programmatic overlap (a prologue that read x before the preceding kernel had finished would see
+    the poison written here, or the previous round's activations)."""
+    bits = 6
+    shA = gen.small_shape(2048, 1024, 32, 64, 16, shape_id=71)
+    shB = gen.small_shape(1024, 384, 32, 32, 16, shape_id=72)
+    layA, layB = gen.make_layer(0, shA, bits), gen.make_layer(0, shB, bits)
+    dA, dB = H.DeviceLayer(layA, bwla), H.DeviceLayer(layB, bwla)
+    wsA = bwla.new_workspace(M, shA.K, shA.N, shA.r, bits)
+    wsB = bwla.new_workspace(M, shB.K, shB.N, shB.r, bits)
+    y1 = torch.empty((M, shA.N), dtype=torch.bfloat16, device="cuda")
+    y2 = torch.empty((M, shB.N), dtype=torch.bfloat16, device="cuda")
+    for rnd in range(3):
+        xb = gen.make_activations(0, shA, M, layer=rnd)
+        xd = H.bf16_to_dev(xb)
+        y1.view(torch.int16).fill_(0x7FC0)          # NaN: a premature read cannot go unnoticed
+        torch.cuda.synchronize()
+        bwla.bwla_w1ax_linear(xd, dA.P1, dA.P2, bits, dA.packed, dA.alpha, dA.U, dA.V, dA.mu, out=y1, workspace=wsA)
+        bwla.bwla_w1ax_linear(y1, dB.P1, dB.P2, bits, dB.packed, dB.alpha, dB.U, dB.V, dB.mu, out=y2, workspace=wsB)
+        torch.cuda.synchronize()
+        assert bwla.bwla_check_status(wsA) == 0 and bwla.bwla_check_status(wsB) == 0
+        y1_bits = H.bf16_to_host(y1)
+        refA = oracle.linear(xb, layA.P1, layA.P2, bits, dA.packed_host, layA.alpha, layA.U, layA.V, layA.mu)
+        H.check_output(y1_bits, refA["y"])
+        # the second layer is judged on the activations it was really given
+        refB = oracle.linear(y1_bits, layB.P1, layB.P2, bits, dB.packed_host, layB.alpha, layB.U, layB.V, layB.mu)
+        H.check_output(H.bf16_to_host(y2), refB["y"])
+
+
 def test_config0_single_w1a6_linear(bwla):
     rep = _run_layer_case(bwla, 0, gen.CONFIG_SHAPES[0][0], 16, 6)
     assert rep["rel_l2"] <= 2e-3
