@@ -524,6 +524,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         // every thread of every CTA of the cluster takes part, whether or not its CTA gave up
         cluster_arrive_release();
         cluster_wait_acquire();
+        if (threadIdx.x == kFirstExpander) BWLA_CTA_STAMP(6);
         if (L::can_split && warp >= 6 && !*abort_flag) {
             // the tokens of the tile are dealt round-robin to the CTAs of the cluster; a thread sums four consecutive
             // rows of one token over all CTAs with 128-bit distributed-shared-memory loads
@@ -567,6 +568,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 }
             }
         }
+        if (threadIdx.x == kFirstExpander) BWLA_CTA_STAMP(7);
         // nobody leaves while a neighbour may still read its shared memory
         cluster_arrive_release();
         cluster_wait_acquire();

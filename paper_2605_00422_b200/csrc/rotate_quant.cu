@@ -72,7 +72,7 @@ struct PrologueParams {
     int sp_s;           // split_y: slices the contraction depth is cut into (partial sums are added afterwards)
     // low-rank
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
-    int lr_wide;        // rows of V x tokens per low-rank block: 0: 2 x 16, 1: 8 x 8 (many tokens), 2: 2 x 8 (few tokens)
+    int lr_wide;        // low-rank blocks: 0: 2 rows of V x 16 tokens (FMA), 1: 8 x 8 (FMA, many tokens), 2: 8 x 16 on the warp-level tensor-core path (few tokens)
     int lr_stage;       // 1: a low-rank block copies its rows of V into shared memory before it waits for x
 };
 
@@ -629,12 +629,78 @@ __device__ void lowrank_role(const PrologueParams& p, int b, float* smem) {
     }
 }
 
+// Few tokens: T for a tile of 16 tokens x 8 columns per block on the warp-level tensor-core path
+// (mma.sync m16n8k16, bf16 in, fp32 accumulate): far fewer instructions than the FMA version, so these blocks do not
+// take issue slots from the rotation blocks they share SMs with.  The warps of the block split K in chunks of 32; a
+// lane reads 16 bytes of two token rows and of one row of V per chunk, and the chunk is contracted by two MMAs whose
+// k order is permuted the same way for both operands (a sum over k does not care).  Partial tiles are added across
+// the warps in shared memory in warp order.
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ void lowrank_mma_role(const PrologueParams& p, int b, float* smem) {
+    const int jtiles = p.lr_cols / 8;
+    const int j0 = (b % jtiles) * 8;
+    const int64_t t0 = (int64_t)(b / jtiles) * 16;
+    if (t0 >= p.M) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int g = lane >> 2, tg = lane & 3;
+    const int K = p.K;
+    griddep_launch_dependents();
+    griddep_wait();                                           // x may be the output of the preceding kernel
+    BWLA_PBLOCK(2);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    if (j0 < p.r) {
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        const bool row_lo = t0 + g < p.M, row_hi = t0 + g + 8 < p.M, col = j0 + g < p.r;
+        const uint4* xlo = reinterpret_cast<const uint4*>(p.x + (t0 + (row_lo ? g : 0)) * p.ldx) + tg;
+        const uint4* xhi = reinterpret_cast<const uint4*>(p.x + (t0 + (row_hi ? g + 8 : 0)) * p.ldx) + tg;
+        const uint4* vj = reinterpret_cast<const uint4*>(p.V + (int64_t)(j0 + (col ? g : 0)) * K) + tg;
+        const int chunks = K >> 5;
+#pragma unroll 4
+        for (int c = warp; c < chunks; c += nwarps) {
+            const uint4 a = row_lo ? __ldg(xlo + 4 * c) : zero;
+            const uint4 h = row_hi ? __ldg(xhi + 4 * c) : zero;
+            const uint4 v = col ? __ldg(vj + 4 * c) : zero;
+            mma_bf16_16x8x16(acc, a.x, h.x, a.y, h.y, v.x, v.y);
+            mma_bf16_16x8x16(acc, a.z, h.z, a.w, h.w, v.z, v.w);
+        }
+    }
+    // acc: (token g, columns 2tg, 2tg+1), (token g+8, same columns)
+    float* red = smem;                                        // [nwarps][16 * 8]
+    red[warp * 128 + g * 8 + 2 * tg] = acc[0];
+    red[warp * 128 + g * 8 + 2 * tg + 1] = acc[1];
+    red[warp * 128 + (g + 8) * 8 + 2 * tg] = acc[2];
+    red[warp * 128 + (g + 8) * 8 + 2 * tg + 1] = acc[3];
+    __syncthreads();
+    for (int o = threadIdx.x; o < 128; o += blockDim.x) {
+        const int i = o >> 3, j = o & 7;
+        if (t0 + i < p.M) {
+            float s = 0.f;
+            for (int w = 0; w < nwarps; ++w) s += red[w * 128 + o];
+            // three bf16 terms carry all 24 bits of the fp32 sum
+            const __nv_bfloat16 hi = __float2bfloat16_rn(s);
+            const float r1 = s - __bfloat162float(hi);
+            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+            const int64_t at = (t0 + i) * p.lr_cols + j0 + j;
+            p.Thl[at] = hi;
+            p.Thl[p.M * p.lr_cols + at] = mid;
+            p.Thl[2 * p.M * p.lr_cols + at] = lo;
+        }
+    }
+}
+
 __global__ void prologue_kernel(PrologueParams p) {
     extern __shared__ __align__(16) float smem[];
     BWLA_PBLOCK(0);
     if ((int)blockIdx.x < p.rot_blocks) rotate_role(p, smem);
     else if (p.lr_wide == 1) lowrank_role<8, 8>(p, (int)blockIdx.x - p.rot_blocks, smem);
-    else if (p.lr_wide == 2) lowrank_role<2, 8>(p, (int)blockIdx.x - p.rot_blocks, smem);
+    else if (p.lr_wide == 2) lowrank_mma_role(p, (int)blockIdx.x - p.rot_blocks, smem);
     else lowrank_role<2, 16>(p, (int)blockIdx.x - p.rot_blocks, smem);
     BWLA_PBLOCK(1);
 }
@@ -774,14 +840,16 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     }
     int lr_blocks = 0;
     if (r > 0 && Thl) {
-        // few tokens: small tiles, so that the handful of blocks is done sooner; many: tiles that re-read less
-        p.lr_wide = (M >= 64 && p.lr_cols % 8 == 0) ? 1 : (M <= 16 ? 2 : 0);
+        // few tokens: the tensor-core version (needs 16-byte rows); many tokens: FMA tiles that re-read little
+        const bool rows16 = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(V)) & 15) == 0 && ldx % 8 == 0 &&
+                            K % 32 == 0 && p.lr_cols % 8 == 0;
+        p.lr_wide = (M >= 64 && p.lr_cols % 8 == 0) ? 1 : (rows16 ? 2 : 0);
         lr_blocks = p.lr_wide == 1 ? (p.lr_cols / 8) * (int)((M + 7) / 8)
-                  : p.lr_wide == 2 ? (p.lr_cols / 2) * (int)((M + 7) / 8) : (p.lr_cols / 2) * (int)((M + 15) / 16);
+                  : p.lr_wide == 2 ? (p.lr_cols / 8) * (int)((M + 15) / 16) : (p.lr_cols / 2) * (int)((M + 15) / 16);
         // shared memory of a low-rank block: per-warp partial sums, and its rows of V when those are staged (few tokens)
         const size_t red_bytes = (size_t)kLrMaxWarps * 64 * 4;
         const size_t stage_bytes = (size_t)2 * (size_t)K * 2;
-        p.lr_stage = (p.lr_wide != 1 && red_bytes + stage_bytes <= (size_t)kPrologueSmemFloats * 4) ? 1 : 0;
+        p.lr_stage = (p.lr_wide == 0 && red_bytes + stage_bytes <= (size_t)kPrologueSmemFloats * 4) ? 1 : 0;
         smem = std::max(smem, red_bytes + (p.lr_stage ? stage_bytes : 0));
     }
     int grid = p.rot_blocks + lr_blocks;
