@@ -105,22 +105,12 @@ __device__ unsigned long long g_cta_times[4096 * 8];
 __device__ __forceinline__ unsigned long long global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define BWLA_CTA_STAMP(i) do { const unsigned lb = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); \
         if (lb < 4096) g_cta_times[lb * 8 + (i)] = global_ns(); } while (0)
-// clock stamps of the ring of CTA (0,0,0): [w][i][.] for w < 8 expander warp w's i-th own k-block (0 before the wait
-// for weights, 1 words loaded, 2 before the wait for the stage, 3 stage free, 4 stored, 5 handed over); for w = 8, 9
-// the issuing threads' i-th own k-block (0 before the wait for codes, 1 codes there, 2 operand there, 3 issued)
-__device__ long long g_ring_trace[10 * 32 * 8];
-#define BWLA_RING(who, i, j) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (i) < 32) \
-        g_ring_trace[((who) * 32 + (i)) * 8 + (j)] = clock64(); } while (0)
-extern "C" int bwla_trace_ring(long long* host) {
-    return cudaMemcpyFromSymbol(host, g_ring_trace, sizeof(g_ring_trace)) == cudaSuccess ? 0 : -4;
-}
 extern "C" int bwla_trace_ctas(unsigned long long* host, int n) {
     return cudaMemcpyFromSymbol(host, g_cta_times, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -4;
 }
 #else
 #define BWLA_STAMP(i) do { } while (0)
 #define BWLA_CTA_STAMP(i) do { } while (0)
-#define BWLA_RING(who, i, j) do { } while (0)
 #endif
 
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
@@ -142,15 +132,17 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
     return false;
 }
 
-// A whole warp waits on a barrier: lane 0 polls, the result is broadcast and the warp leaves the call converged, as the
-// .sync.aligned tcgen05 instructions that follow such a wait require (lanes that each ran their own polling loop may
-// come out of it at different times, and a warp-wide tensor-memory store issued by part of a warp lands late).
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
-    int ok = 1;
-    if (lane == 0) ok = wait_or_abort(bar, parity, abort_flag) ? 1 : 0;
-    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
-    __syncwarp();
-    return ok != 0;
+// A whole warp waits on a barrier and leaves the call converged, as the .sync.aligned tcgen05 instructions that follow
+// such a wait require (lanes that each ran their own polling loop may come out of it at different times, and a
+// warp-wide tensor-memory store issued by part of a warp lands late): every lane polls, the warp goes on when all saw
+// the phase complete.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        const bool done = mbar_try_wait_parked(bar, parity, kParkNs);
+        if (__all_sync(0xFFFFFFFFu, done)) return true;
+        if (*abort_flag) return false;
+    }
+    return false;
 }
 
 // One output value from its two accumulators (mu_sc is zero when the layer has no row shift).
@@ -301,38 +293,48 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     }
                 }
             }
+            // This thread runs a long chain of dependent scalar instructions beside warps that keep the schedulers busy, so
+            // every instruction here costs several cycles: indices advance by addition (no division), descriptors are
+            // built by adding to one precomputed word, and only this thread's own k-blocks are visited.
+            // k-block kb of the CTA sits in code stage (kb / SUBS) % BS at sub-block kb % SUBS (all units but the last of
+            // the matrix have eight sub-blocks, a multiple of SUBS) and in operand stage kb % AS.
             const uint32_t d_addr = tmem_base + iss * N_TOK;
-            int bs = 0; uint32_t bph = 0; int kb = 0;
-            for (int u = unit_begin; u < unit_end && ok; ++u) {
-                const int ns = sub_count(u);
-                for (int s = 0; s < ns; ++s, ++kb) {
-                    const int sb = s % SUBS;
-                    // every issuing thread sees each code stage filled before it releases it, whether or not one of
-                    // the stage's k-blocks is its own: its release can then never run a whole ring ahead
-                    if (kb % NISS == iss) BWLA_RING(8 + iss, kb / NISS, 0);
-                    if (sb == 0 && !wait_or_abort(&b_full[bs], bph, abort_flag)) { give_up(p.status, abort_flag, 0x30); ok = false; break; }
-                    if (kb % NISS == iss) {
-                        BWLA_RING(8 + iss, kb / NISS, 1);
-                        const int as = kb % AS;
-                        const uint32_t aph = (uint32_t)(kb / AS) & 1u;
-                        if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; break; }
-                        if (kb == 0) BWLA_STAMP(8);
-                        BWLA_RING(8 + iss, kb / NISS, 2);
-                        tc_fence_after();
-                        const uint32_t b_addr = smem_u32(bbuf + bs * L::b_bytes + sb * L::sub_bytes);
-                        const uint32_t a_addr = tmem_base + L::A_COL + 32 * as;
+            const uint32_t a_base = tmem_base + L::A_COL;
+            const uint64_t desc_hi = smem_desc_sw128(0u, 0u);                      // everything but the start address
+            const uint32_t b_lo0 = (smem_u32(bbuf) & 0x3FFFFu) >> 4;               // start-address field of stage 0, sub-block 0
+            int as = iss; uint32_t aph = 0;                                        // NISS <= AS
+            uint32_t acc = 0;
+            int bs = 0; uint32_t bph = 0;
+            for (int kb0 = 0; kb0 < my_blocks && ok; kb0 += SUBS) {
+                // every issuing thread sees each code stage filled before it releases it, whether or not one of the
+                // stage's k-blocks is its own: its release can then never run a whole ring ahead
+                if (!wait_or_abort(&b_full[bs], bph, abort_flag)) { give_up(p.status, abort_flag, 0x30); ok = false; break; }
+                const int cnt = min(SUBS, my_blocks - kb0);
+                const uint32_t stage_lo = b_lo0 + (uint32_t)bs * (L::b_bytes >> 4);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            mma_i8_ts(d_addr, a_addr + 8 * i, smem_desc_sw128(b_addr, 32 * i), idesc, (kb < NISS && i == 0) ? 0u : 1u);
-                        tc_commit(&a_empty[as]);
-                        BWLA_RING(8 + iss, kb / NISS, 3);
-                    }
-                    if (sb == SUBS - 1 || s == ns - 1) {
-                        // this thread is done with the code stage once its MMAs so far have completed
-                        tc_commit(&b_empty[bs]);
-                        if (++bs == BS) { bs = 0; bph ^= 1; }
+                for (int sb = 0; sb < SUBS; ++sb) {
+                    const bool own = (SUBS % NISS == 0) ? (sb % NISS == iss) : ((kb0 + sb) % NISS == iss);
+                    if (ok && sb < cnt && own) {
+                        if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; }
+                        if (ok) {
+                            if (kb0 + sb == 0) BWLA_STAMP(8);
+                            tc_fence_after();
+                            const uint64_t desc = desc_hi | (uint64_t)(stage_lo + (uint32_t)sb * (L::sub_bytes >> 4));
+                            const uint32_t a_addr = a_base + 32 * as;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                mma_i8_ts(d_addr, a_addr + 8 * i, desc + 2 * i, idesc, acc);   // 32 bytes along K = 2 address units
+                                acc = 1u;
+                            }
+                            tc_commit(&a_empty[as]);
+                            as += NISS;
+                            if (as >= AS) { as -= AS; aph ^= 1u; }
+                        }
                     }
                 }
+                // this thread is done with the code stage once its MMAs so far have completed
+                tc_commit(&b_empty[bs]);
+                if (++bs == BS) { bs = 0; bph ^= 1u; }
             }
             tc_commit(d_full);
             if (iss == 0) BWLA_STAMP(9);
@@ -375,66 +377,60 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(u_full);
         }
-        // This warp expands k-blocks kb = part, part + EW, ... of the CTA (stage kb % AS; AS is a multiple of EW).  Its
-        // registers are left alone until tcgen05.wait::st has returned; the other warps of the quarter fill the
-        // store's latency.
+        // This warp expands k-blocks kb = part, part + EW, ... of the CTA (operand stage kb % AS; AS is a multiple of EW and
+        // every unit but the last of the matrix has eight k-blocks, also a multiple of EW, so inside each unit the warp
+        // takes sub-blocks part, part + EW, ...).  Its registers are left alone until tcgen05.wait::st has returned; the
+        // other warps of the quarter fill the store's latency.
         int ws = 0; uint32_t wph = 0;
+        int as = part; uint32_t aph = 0;
         bool ok = true;
-        int kb0 = 0;                                   // k-block index of sub-block 0 of the current unit
         for (int u = unit_begin; u < unit_end && ok; ++u) {
-            if (lane == 0) BWLA_RING(warp - 6, (kb0 + ((part - kb0) % EW + EW) % EW) / EW, 0);
-            if (!warp_wait(&w_full[ws], wph, abort_flag, lane)) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
+            if (!warp_wait(&w_full[ws], wph, abort_flag)) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
             if (e == 64 && u == unit_begin) { BWLA_STAMP(3); BWLA_CTA_STAMP(1); }
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
-            const int s_first = ((part - kb0) % EW + EW) % EW;      // kb0 + s_first = part (mod EW)
             // the sign words of this warp's k-blocks of the unit, loaded together
             uint4 w4[8 / EW];
 #pragma unroll
             for (int i = 0; i < 8 / EW; ++i) {
-                const int s = EW * i + s_first;
+                const int s = EW * i + part;
                 if (s < ns) w4[i] = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
             }
 #pragma unroll
             for (int i = 0; i < 8 / EW; ++i) {
-                const int s = EW * i + s_first;
-                if (s >= ns) break;
-                const int kb = kb0 + s;
-                const int as = kb % AS;
-                const uint32_t aph = (uint32_t)(kb / AS) & 1u;
-                uint32_t v[32];
-                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 1);
-                const uint32_t w[4] = {w4[i].x, w4[i].y, w4[i].z, w4[i].w};
+                if (ok && EW * i + part < ns) {
+                    uint32_t v[32];
+                    const uint32_t w[4] = {w4[i].x, w4[i].y, w4[i].z, w4[i].w};
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                    for (int c = 0; c < 4; ++c)
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
-                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 2);
-                if (!warp_wait(&a_empty[as], aph ^ 1, abort_flag, lane)) { give_up(p.status, abort_flag, 0x41); ok = false; break; }
-                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 3);
-                tc_fence_after();
-                tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
-                tc_wait_st();
-                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 4);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&a_full[as]);
-                if (lane == 0) BWLA_RING(warp - 6, kb / EW, 5);
+                        for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
+                    if (!warp_wait(&a_empty[as], aph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x41); ok = false; }
+                    if (ok) {
+                        tc_fence_after();
+                        tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&a_full[as]);
+                        as += EW;
+                        if (as >= AS) { as = part; aph ^= 1u; }
+                    }
+                }
             }
             // The stage is released only here, after every word loaded from it has gone through the expansion: an
             // arrive placed right behind the loads let the copy of a later unit overwrite words not yet read.
             __syncwarp();
             if (lane == 0) mbar_arrive(&w_empty[ws]);
-            if (++ws == WS) { ws = 0; wph ^= 1; }
-            kb0 += ns;
+            if (++ws == WS) { ws = 0; wph ^= 1u; }
         }
         if (e == 64) { BWLA_STAMP(4); BWLA_CTA_STAMP(2); }
         // the stores of the epilogue come after the preceding kernel; the per-token scales and code sums it wrote were
         // staged in shared memory by warp 1 while the K loop ran
         griddep_wait();
-        if (!warp_wait(s_full, 0, abort_flag, lane)) { give_up(p.status, abort_flag, 0x51); ok = false; }
+        if (!warp_wait(s_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x51); ok = false; }
         if (ok) {
-            if (!warp_wait(d_full, 0, abort_flag, lane)) { give_up(p.status, abort_flag, 0x50); ok = false; }
+            if (!warp_wait(d_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
         if (e == 64) { BWLA_STAMP(5); BWLA_CTA_STAMP(3); }
         if (ok) {

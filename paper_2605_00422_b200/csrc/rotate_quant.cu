@@ -74,6 +74,7 @@ struct PrologueParams {
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
     int lr_wide;        // low-rank blocks: 0: 2 rows of V x 16 tokens (FMA), 1: 8 x 8 (FMA, many tokens), 2: 8 x 16 on the warp-level tensor-core path (few tokens)
     int lr_stage;       // 1: a low-rank block copies its rows of V into shared memory before it waits for x
+    int late_trigger;   // 1: the next kernel of the stream is let in only when this one is nearly done (see launch_prologue)
 };
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -331,7 +332,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             *reinterpret_cast<float4*>(P2s + 4 * i) = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
         load_p1_columns(p.P1, n1, a_lo, rows, rp, P1s);
         cluster_arrive_release();              // "this CTA is running": waited for before the first remote store
-        griddep_launch_dependents();
+        if (!p.late_trigger) griddep_launch_dependents();
         griddep_wait();                        // x may be the output of the preceding kernel
         BWLA_PSTAMP(1); BWLA_PBLOCK(2);
         {
@@ -379,7 +380,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
                 *reinterpret_cast<float4*>(Ps + 4 * i) = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
             load_p1_columns(p.P1, n1, 0, n1, (n1 + 3) & ~3, P1s);
         }
-        griddep_launch_dependents();
+        if (!p.late_trigger) griddep_launch_dependents();
         griddep_wait();                        // x may be the output of the preceding kernel
         load_x(p.x + t * p.ldx, K, Xs);
         BWLA_PSTAMP(1);
@@ -419,7 +420,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         // generic shapes (n2 not a multiple of 4; one CTA per token): one output per thread step
         float* Zf = smem + p.slab_cap;
         slots = Zf + K;
-        griddep_launch_dependents();
+        if (!p.late_trigger) griddep_launch_dependents();
         griddep_wait();
         load_x(p.x + t * p.ldx, K, Xs);
         __syncthreads();
@@ -458,6 +459,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
 
     BWLA_PSTAMP(7);
+    if (p.late_trigger) griddep_launch_dependents();
     // nothing is stored to global memory before the preceding kernel of the stream has completed
     griddep_wait();
     BWLA_PSTAMP(8);
@@ -852,6 +854,10 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
         p.lr_stage = (p.lr_wide == 0 && red_bytes + stage_bytes <= (size_t)kPrologueSmemFloats * 4) ? 1 : 0;
         smem = std::max(smem, red_bytes + (p.lr_stage ? stage_bytes : 0));
     }
+    // A block with this much shared memory leaves no room on its SM for a block of the next kernel of the stream.  Let
+    // in early, that kernel would crowd onto the SMs this one leaves free and stay there; so it is let in late, when
+    // the blocks of this one are about to leave.
+    p.late_trigger = smem > 110 * 1024 ? 1 : 0;
     int grid = p.rot_blocks + lr_blocks;
     grid = (grid + C - 1) / C * C;
     if (grid == 0) return BWLA_OK;
