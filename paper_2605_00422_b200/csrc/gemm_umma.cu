@@ -645,13 +645,29 @@ bool umma_supports(int64_t M, int64_t K, int64_t N, int r) {
            encode_tiled_fn() != nullptr;
 }
 
-// How many CTAs share a tile and split K.  Enough to put about one CTA on every SM, never more than the units there
-// are, never more than the portable cluster size, and only powers of two.
+// How many CTAs share a tile and split K, for the configuration with two CTAs per SM.  Enough to put about one CTA on
+// every SM, never more than the units there are, never more than the portable cluster size; powers of two.
 static int choose_splits(int tiles, int units, bool can_split) {
     if (!can_split) return 1;
     int s = 1;
     while (s * 2 <= 8 && s * 2 <= units && tiles * s * 2 <= 148 + 148 / 4) s *= 2;
     return s;
+}
+
+// Few tokens: a CTA's K loop is a chain of latencies, not of throughput, so one CTA per SM with twice the expander warps
+// and a twice as deep operand ring (all 512 tensor-memory columns) gets through its k-blocks about 1.7 times as fast
+// as one of two CTAs that share an SM.  It is worth it when a K split puts the whole grid on the SMs at once.
+// Returns the split for that configuration, or 0 when two CTAs per SM are expected to finish sooner.
+static int choose_wide_splits(int tiles, int units, int narrow_splits) {
+    if (tiles > 148) return 0;
+    int s = 148 / tiles;
+    if (s > 8) s = 8;
+    if (s > units) s = units;
+    if (s < 1) return 0;
+    const int blocks = units * (kUnitK / kBlockK);
+    const double wide = (double)((blocks + s - 1) / s) / 1.7;
+    const double narrow = (double)((blocks + narrow_splits - 1) / narrow_splits) * (tiles * narrow_splits > 148 ? 1.2 : 1.0);
+    return wide < narrow ? s : 0;
 }
 
 // codes_interleaved: int8 [M][K] in the interleaved order.  a.Thl: bf16 [3][M][64], T = hi + mid + lo.
@@ -661,7 +677,9 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
     const int row_tiles = (N + kRowsPerCta - 1) / kRowsPerCta;
     const int tok_tiles = (M + n_tok - 1) / n_tok;
     const int units = (K + kUnitK - 1) / kUnitK;
-    const int split = choose_splits(row_tiles * tok_tiles, units, n_tok <= 64);
+    int split = choose_splits(row_tiles * tok_tiles, units, n_tok <= 64);
+    const int wide_split = n_tok <= 32 ? choose_wide_splits(row_tiles * tok_tiles, units, split) : 0;
+    if (wide_split) split = wide_split;
 
     CUtensorMap wm, bm, tm;
     {
@@ -698,8 +716,10 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
 
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     switch (n_tok) {
-                case 16: return launch_umma_t<16, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
-        case 32: return launch_umma_t<32, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
+                case 16: return wide_split ? launch_umma_t<16, 3, 2, 512, 2, 4>(wm, bm, tm, p, grid, stream)
+                                   : launch_umma_t<16, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
+        case 32: return wide_split ? launch_umma_t<32, 3, 2, 512, 2, 4>(wm, bm, tm, p, grid, stream)
+                                   : launch_umma_t<32, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
         case 64: return launch_umma_t<64, 4, 3, 512, 2, 2>(wm, bm, tm, p, grid, stream);
         default: return launch_umma_t<128, 2, 6, 512, 2, 2>(wm, bm, tm, p, grid, stream);
     }

@@ -170,6 +170,14 @@ def test_output_of_one_layer_feeds_the_next_without_synchronisation(bwla, M):
         H.check_output(H.bf16_to_host(y2), refB["y"])
 
 
+@pytest.mark.parametrize("N,K,n1,n2", [(5120, 8192, 64, 128), (3328, 5120, 64, 80), (2944, 6144, 64, 96), (2560, 7168, 64, 112)])
+def test_few_tokens_odd_k_splits(bwla, N, K, n1, n2):
+    """Row-tile counts for which the contraction splits K three, five, six and seven ways (clusters of that size)."""
+    shape = gen.small_shape(K, N, n1, n2, 16, shape_id=N + K)
+    _run_layer_case(bwla, 0, shape, 16, 6, direct_words=True)
+    _run_layer_case(bwla, 0, shape, 5, 8, direct_words=True, with_mu=True)
+
+
 def test_config0_single_w1a6_linear(bwla):
     rep = _run_layer_case(bwla, 0, gen.CONFIG_SHAPES[0][0], 16, 6)
     assert rep["rel_l2"] <= 2e-3
