@@ -70,6 +70,8 @@ struct PrologueParams {
     int split_y;        // 1 (C > 1): each CTA evaluates its rows of Y from all of x, nothing but absmax is exchanged
     int sp_tr, sp_rp;   // split_y: rows per thread tile (4 or 8); slab rows rounded up to it (row stride of P1s and Zt)
     int sp_s;           // split_y: slices the contraction depth is cut into (partial sums are added afterwards)
+    int sp_zt_off;      // split_y: where Z'^T lives, in floats from the start of shared memory (0: over x, dead by then)
+    int sp_rest_off;    // split_y: where P2 starts
     // low-rank
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
     int lr_wide;        // low-rank blocks: 0: 2 rows of V x 16 tokens (FMA), 1: 8 x 8 (FMA, many tokens), 2: 8 x 16 on the warp-level tensor-core path (few tokens)
@@ -322,8 +324,8 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         // ---- few tokens: this CTA's rows of Y from all of x; nothing but absmax and code sums is exchanged
         const int rp = p.sp_rp, S = p.sp_s;
         __nv_bfloat16* Xh = reinterpret_cast<__nv_bfloat16*>(smem);   // all of x_t as it comes; later this CTA's rows of Y (fp32)
-        float* Zt = smem + (K >> 1);           // Z'^T: [n2][rp], Z' = rows [a_lo, a_hi) of P1^T X
-        float* P2s = Zt + n2 * rp;             // all of P2
+        float* Zt = smem + p.sp_zt_off;        // Z'^T: [n2][rp], Z' = rows [a_lo, a_hi) of P1^T X (written once x is dead)
+        float* P2s = smem + p.sp_rest_off;     // all of P2
         float* P1s = P2s + p.ps_cap;           // columns [a_lo, a_hi) of P1: [n1][rp]
         float* part = P1s + p.p1_cap;          // [S][rp][n2] partial sums
         slots = part + S * rp * n2;
@@ -780,7 +782,11 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                 p.p1_cap = n1 * p.sp_rp + 8;
                 p.ch1 = n2; p.ch2 = cap; p.tr1 = p.tr2 = p.sp_tr;
                 const int tiles = (p.sp_rp / p.sp_tr) * (n2 / 4);
-                const int64_t fixed = K / 2 + (int64_t)n2 * p.sp_rp + p.ps_cap + p.p1_cap + 16;
+                // Z'^T is written when x is dead and may take its place; Y is written when Z'^T is dead
+                const int64_t zt = (int64_t)n2 * p.sp_rp;
+                p.sp_zt_off = zt <= K / 2 ? 0 : (int)(K / 2);
+                p.sp_rest_off = (int)(K / 2 + (zt <= K / 2 ? 0 : zt));
+                const int64_t fixed = p.sp_rest_off + p.ps_cap + p.p1_cap + 16;
                 // cut the depth until there are about 512 work items, at least four steps per slice, while it fits
                 int S = 1;
                 while (S < 8 && tiles * S < 512 && std::min(n1, n2) / (S * 2) >= 4 &&
@@ -830,8 +836,9 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
             // spread one token over several SMs while there are few tokens and the token is worth splitting, as long as
             // every token's cluster is resident at once (a second wave of clusters would double the latency)
             const double flops = 2.0 * (double)K * (n1 + n2);
-            while (C < 8 && M * (C * 2) <= 148 && flops / (C * 2) >= 1.5e5 && n1 / (C * 2) >= gran) C *= 2;
-            for (; C > 1; C >>= 1) {
+            C = 8;
+            while (C > 1 && (M * C > 148 || flops / C < 1.5e5 || n1 / C < gran)) --C;
+            for (; C > 1; --C) {
                 if (!plan(C)) continue;
                 if (clusters_resident(C, threads, smem) >= M) break;
             }
