@@ -105,12 +105,27 @@ __device__ unsigned long long g_cta_times[4096 * 8];
 __device__ __forceinline__ unsigned long long global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define BWLA_CTA_STAMP(i) do { const unsigned lb = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); \
         if (lb < 4096) g_cta_times[lb * 8 + (i)] = global_ns(); } while (0)
+// clock stamps of the ring of CTA (0,0,0), kept in shared memory while the loop runs (a global store per stamp would
+// disturb what it measures): [w][i][.] for w < 8 the first eight expander warps' i-th own k-block (0 before the wait for
+// the stage, 1 stage free, 2 stored, 3 handed over), for w = 8, 9 the issuing threads' (0 before the wait for the
+// operand, 1 operand there, 2 issued and committed)
+__device__ unsigned int g_ring_log[10 * 32 * 4];
+#define BWLA_RING_DECL __shared__ unsigned int ring_log[10 * 32 * 4];
+#define BWLA_RING(who, i, j) do { if ((who) < 10 && (i) < 32) ring_log[((who) * 32 + (i)) * 4 + (j)] = (unsigned int)clock(); } while (0)
+#define BWLA_RING_DUMP do { __syncthreads(); if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
+        for (int i_ = threadIdx.x; i_ < 10 * 32 * 4; i_ += blockDim.x) g_ring_log[i_] = ring_log[i_]; } while (0)
+extern "C" int bwla_trace_ring(unsigned int* host) {
+    return cudaMemcpyFromSymbol(host, g_ring_log, sizeof(g_ring_log)) == cudaSuccess ? 0 : -4;
+}
 extern "C" int bwla_trace_ctas(unsigned long long* host, int n) {
     return cudaMemcpyFromSymbol(host, g_cta_times, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -4;
 }
 #else
 #define BWLA_STAMP(i) do { } while (0)
 #define BWLA_CTA_STAMP(i) do { } while (0)
+#define BWLA_RING_DECL
+#define BWLA_RING(who, i, j) do { } while (0)
+#define BWLA_RING_DUMP do { } while (0)
 #endif
 
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
@@ -125,6 +140,8 @@ __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_fl
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     // Each poll may park the thread for up to kParkNs while the phase is open: a warp that spun on the barrier would
     // take issue slots from the expander warps that share its scheduler.
+    // a phase that is already complete is seen by the non-blocking probe in a fraction of the time try_wait takes
+    if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
         if (*abort_flag) return false;
@@ -137,6 +154,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
 // warp-wide tensor-memory store issued by part of a warp lands late): every lane polls, the warp goes on when all saw
 // the phase complete.
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (__all_sync(0xFFFFFFFFu, mbar_test_wait(bar, parity))) return true;
     for (uint32_t i = 0; i < kWaitLimit; ++i) {
         const bool done = mbar_try_wait_parked(bar, parity, kParkNs);
         if (__all_sync(0xFFFFFFFFu, done)) return true;
@@ -156,6 +174,7 @@ __global__ void __launch_bounds__(kFirstExpander + 128 * EW, TMEM_COLS == 256 ? 
 umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map,
                 const __grid_constant__ CUtensorMap t_map, UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
+    BWLA_RING_DECL
     using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS, EW>;
     constexpr int AS = L::AS;
     constexpr int SUBS = L::SUBS;
@@ -315,7 +334,9 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 for (int sb = 0; sb < SUBS; ++sb) {
                     const bool own = (SUBS % NISS == 0) ? (sb % NISS == iss) : ((kb0 + sb) % NISS == iss);
                     if (ok && sb < cnt && own) {
+                        BWLA_RING(8 + iss, (kb0 + sb) / NISS, 0);
                         if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; }
+                        BWLA_RING(8 + iss, (kb0 + sb) / NISS, 1);
                         if (ok) {
                             if (kb0 + sb == 0) BWLA_STAMP(8);
                             tc_fence_after();
@@ -327,6 +348,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                                 acc = 1u;
                             }
                             tc_commit(&a_empty[as]);
+                            BWLA_RING(8 + iss, (kb0 + sb) / NISS, 2);
                             as += NISS;
                             if (as >= AS) { as -= AS; aph ^= 1u; }
                         }
@@ -384,8 +406,11 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         int ws = 0; uint32_t wph = 0;
         int as = part; uint32_t aph = 0;
         bool ok = true;
+        int nown = 0;   // own k-blocks so far (tuning stamps only)
         for (int u = unit_begin; u < unit_end && ok; ++u) {
+            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 0);
             if (!warp_wait(&w_full[ws], wph, abort_flag)) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
+            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 1);
             if (e == 64 && u == unit_begin) { BWLA_STAMP(3); BWLA_CTA_STAMP(1); }
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
@@ -396,6 +421,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 const int s = EW * i + part;
                 if (s < ns) w4[i] = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
             }
+            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 2);
 #pragma unroll
             for (int i = 0; i < 8 / EW; ++i) {
                 if (ok && EW * i + part < ns) {
@@ -405,14 +431,19 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     for (int c = 0; c < 4; ++c)
 #pragma unroll
                         for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
+                    if (lane == 0) BWLA_RING(warp - 6, nown, 0);
                     if (!warp_wait(&a_empty[as], aph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x41); ok = false; }
+                    if (lane == 0) BWLA_RING(warp - 6, nown, 1);
                     if (ok) {
                         tc_fence_after();
                         tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
                         tc_wait_st();
+                        if (lane == 0) BWLA_RING(warp - 6, nown, 2);
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&a_full[as]);
+                        if (lane == 0) BWLA_RING(warp - 6, nown, 3);
+                        ++nown;
                         as += EW;
                         if (as >= AS) { as = part; aph ^= 1u; }
                     }
@@ -422,6 +453,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             // arrive placed right behind the loads let the copy of a later unit overwrite words not yet read.
             __syncwarp();
             if (lane == 0) mbar_arrive(&w_empty[ws]);
+            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 3);
             if (++ws == WS) { ws = 0; wph ^= 1u; }
         }
         if (e == 64) { BWLA_STAMP(4); BWLA_CTA_STAMP(2); }
@@ -514,6 +546,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         }
     }
     if (threadIdx.x == kFirstExpander) { BWLA_STAMP(6); BWLA_CTA_STAMP(4); }
+    BWLA_RING_DUMP;
     tc_fence_before();
     __syncthreads();
     if (p.splits > 1) {
