@@ -74,7 +74,8 @@ struct PrologueParams {
     int sp_rest_off;    // split_y: where P2 starts
     // low-rank
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
-    int lr_wide;        // low-rank blocks: 0: 2 rows of V x 16 tokens (FMA), 1: 8 x 8 (FMA, many tokens), 2: 8 x 16 on the warp-level tensor-core path (few tokens)
+    int lr_wide;        // low-rank blocks: 0: 2 rows of V x 16 tokens (FMA), 1: 8 x 8 (FMA, many tokens), 2: 8 columns x 16 tokens on the
+                        // warp-level tensor-core path (few tokens), 3: all 64 columns x 16 tokens on that path (many tokens)
     int lr_stage;       // 1: a low-rank block copies its rows of V into shared memory before it waits for x
     int late_trigger;   // 1: the next kernel of the stream is let in only when this one is nearly done (see launch_prologue)
 };
@@ -699,12 +700,81 @@ __device__ void lowrank_mma_role(const PrologueParams& p, int b, float* smem) {
     }
 }
 
+// Many tokens: the same on tiles of 16 tokens x all 64 columns, so that x is read once; a lane keeps the eight
+// column tiles' accumulators (32 registers) and reads one row of V per column tile and chunk.
+__device__ void lowrank_mma_wide_role(const PrologueParams& p, int b, float* smem) {
+    const int64_t t0 = (int64_t)b * 16;
+    if (t0 >= p.M) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int g = lane >> 2, tg = lane & 3;
+    const int K = p.K;
+    const int ntiles = p.lr_cols / 8;                         // <= 8
+    griddep_launch_dependents();
+    griddep_wait();                                           // x may be the output of the preceding kernel
+    BWLA_PBLOCK(2);
+    float acc[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+    {
+        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+        const bool row_lo = t0 + g < p.M, row_hi = t0 + g + 8 < p.M;
+        const uint4* xlo = reinterpret_cast<const uint4*>(p.x + (t0 + (row_lo ? g : 0)) * p.ldx) + tg;
+        const uint4* xhi = reinterpret_cast<const uint4*>(p.x + (t0 + (row_hi ? g + 8 : 0)) * p.ldx) + tg;
+        const uint4* vbase = reinterpret_cast<const uint4*>(p.V) + tg;
+        const int chunks = K >> 5;
+#pragma unroll 2
+        for (int c = warp; c < chunks; c += nwarps) {
+            const uint4 a = row_lo ? __ldg(xlo + 4 * c) : zero;
+            const uint4 h = row_hi ? __ldg(xhi + 4 * c) : zero;
+            uint4 v[8];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                const int j = 8 * nt + g;
+                v[nt] = (nt < ntiles && j < p.r) ? __ldg(vbase + (size_t)j * (K >> 3) + 4 * c) : zero;
+            }
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                mma_bf16_16x8x16(acc[nt], a.x, h.x, a.y, h.y, v[nt].x, v[nt].y);
+                mma_bf16_16x8x16(acc[nt], a.z, h.z, a.w, h.w, v[nt].z, v[nt].w);
+            }
+        }
+    }
+    // partial tiles of the warps, [warp][token 0..15][column 0..63], added in warp order
+    float* red = smem;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        float* r = red + warp * 1024 + 8 * nt + 2 * tg;
+        r[g * 64] = acc[nt][0]; r[g * 64 + 1] = acc[nt][1];
+        r[(g + 8) * 64] = acc[nt][2]; r[(g + 8) * 64 + 1] = acc[nt][3];
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < 1024; o += blockDim.x) {
+        const int i = o >> 6, j = o & 63;
+        if (t0 + i < p.M && j < p.lr_cols) {
+            float s = 0.f;
+            for (int w = 0; w < nwarps; ++w) s += red[w * 1024 + o];
+            // three bf16 terms carry all 24 bits of the fp32 sum
+            const __nv_bfloat16 hi = __float2bfloat16_rn(s);
+            const float r1 = s - __bfloat162float(hi);
+            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+            const int64_t at = (t0 + i) * p.lr_cols + j;
+            p.Thl[at] = hi;
+            p.Thl[p.M * p.lr_cols + at] = mid;
+            p.Thl[2 * p.M * p.lr_cols + at] = lo;
+        }
+    }
+}
+
 __global__ void prologue_kernel(PrologueParams p) {
     extern __shared__ __align__(16) float smem[];
     BWLA_PBLOCK(0);
     if ((int)blockIdx.x < p.rot_blocks) rotate_role(p, smem);
     else if (p.lr_wide == 1) lowrank_role<8, 8>(p, (int)blockIdx.x - p.rot_blocks, smem);
     else if (p.lr_wide == 2) lowrank_mma_role(p, (int)blockIdx.x - p.rot_blocks, smem);
+    else if (p.lr_wide == 3) lowrank_mma_wide_role(p, (int)blockIdx.x - p.rot_blocks, smem);
     else lowrank_role<2, 16>(p, (int)blockIdx.x - p.rot_blocks, smem);
     BWLA_PBLOCK(1);
 }
@@ -852,11 +922,12 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
         // few tokens: the tensor-core version (needs 16-byte rows); many tokens: FMA tiles that re-read little
         const bool rows16 = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(V)) & 15) == 0 && ldx % 8 == 0 &&
                             K % 32 == 0 && p.lr_cols % 8 == 0;
-        p.lr_wide = (M >= 64 && p.lr_cols % 8 == 0) ? 1 : (rows16 ? 2 : 0);
+        p.lr_wide = rows16 ? ((M > 32 && p.lr_cols == 64) ? 3 : 2) : ((M >= 64 && p.lr_cols % 8 == 0) ? 1 : 0);
         lr_blocks = p.lr_wide == 1 ? (p.lr_cols / 8) * (int)((M + 7) / 8)
-                  : p.lr_wide == 2 ? (p.lr_cols / 8) * (int)((M + 15) / 16) : (p.lr_cols / 2) * (int)((M + 15) / 16);
+                  : p.lr_wide == 2 ? (p.lr_cols / 8) * (int)((M + 15) / 16)
+                  : p.lr_wide == 3 ? (int)((M + 15) / 16) : (p.lr_cols / 2) * (int)((M + 15) / 16);
         // shared memory of a low-rank block: per-warp partial sums, and its rows of V when those are staged (few tokens)
-        const size_t red_bytes = (size_t)kLrMaxWarps * 64 * 4;
+        const size_t red_bytes = (size_t)kLrMaxWarps * 4 * (p.lr_wide == 3 ? 1024 : p.lr_wide == 2 ? 128 : 64);
         const size_t stage_bytes = (size_t)2 * (size_t)K * 2;
         p.lr_stage = (p.lr_wide == 0 && red_bytes + stage_bytes <= (size_t)kPrologueSmemFloats * 4) ? 1 : 0;
         smem = std::max(smem, red_bytes + (p.lr_stage ? stage_bytes : 0));
