@@ -218,23 +218,29 @@ __device__ __forceinline__ void slab_partial(const float* __restrict__ A, int rp
         for (int i = 0; i < TR; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-        const float* ap = A + mt * TR;
+        // operand pointers advance by addition: index arithmetic inside this loop cost as many issue slots as the FMAs
+        const float* ap = A + (size_t)k0 * rp + mt * TR;
+        const float* bf = reinterpret_cast<const float*>(B) + (size_t)k0 * n2 + d0;
+        const __nv_bfloat16* bh = reinterpret_cast<const __nv_bfloat16*>(B) + (size_t)k0 * n2 + d0;
 #pragma unroll 4
         for (int k = k0; k < k1; ++k) {
             float4 bv;
             if (B_BF16) {
-                const uint2 w = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(B) + (size_t)k * n2 + d0);
+                const uint2 w = *reinterpret_cast<const uint2*>(bh);
                 bv = make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u),
                                  __uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+                bh += n2;
             } else {
-                bv = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(B) + (size_t)k * n2 + d0);
+                bv = *reinterpret_cast<const float4*>(bf);
+                bf += n2;
             }
             float a[TR];
 #pragma unroll
             for (int i = 0; i < TR; i += 4) {
-                const float4 v = *reinterpret_cast<const float4*>(ap + (size_t)k * rp + i);
+                const float4 v = *reinterpret_cast<const float4*>(ap + i);
                 a[i] = v.x; a[i + 1] = v.y; a[i + 2] = v.z; a[i + 3] = v.w;
             }
+            ap += rp;
 #pragma unroll
             for (int i = 0; i < TR; ++i) {
                 acc[i][0] = fmaf(a[i], bv.x, acc[i][0]);
