@@ -60,6 +60,8 @@ ROT_CASES = [
     (160, 160, 1, 8),
     (86, 128, 2, 6),      # uneven row slabs
     (24, 8, 1, 6),        # slab boundaries must stay on 32-element groups
+    (160, 160, 150, 6),   # many tokens of the largest K: clusters that stay and take several tokens each
+    (160, 160, 41, 8),
 ]
 
 
