@@ -70,6 +70,7 @@ struct PrologueParams {
     int split_y;        // 1 (C > 1): each CTA evaluates its rows of Y from all of x, nothing but absmax is exchanged
     int sp_tr, sp_rp;   // split_y: rows per thread tile (4 or 8); slab rows rounded up to it (row stride of P1s and Zt)
     int sp_s;           // split_y: slices the contraction depth is cut into (partial sums are added afterwards)
+    int sp_tc;          // split_y: 1: both contractions on the warp-level tensor-core path (split-bf16 operands)
     int sp_zt_off;      // split_y: where Z'^T lives, in floats from the start of shared memory (0: over x, dead by then)
     int sp_rest_off;    // split_y: where P2 starts
     // low-rank
@@ -281,6 +282,175 @@ __device__ __forceinline__ float slab_reduce(const float* __restrict__ part, int
     return amax;
 }
 
+// ---------------------------------------------------------------------------------------------
+// The two slab contractions on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 out).
+//
+// An fp32 factor is split into three bf16 terms (hi + mid + lo carry all 24 bits); x is bf16 already.  Every k-step of
+// 16 starts from a zero accumulator, takes the products of the terms that matter (smallest first) and is then added to
+// the running fp32 sum with an ordinary rounded addition: the tensor core only ever sums 16 exact products (48 or 96
+// with the terms), so what its internal accumulation does to long sums does not enter.  The error stays at the level
+// of the fp32 FMA chain (a CPU model of this scheme with the partial sums rounded toward zero is within 3.4e-7 of the
+// token's full scale for K = 25600, the fp32 chain within 5.9e-7; the code window is 1e-6).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void split3(float v, __nv_bfloat16& h, __nv_bfloat16& m, __nv_bfloat16& l) {
+    h = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(h);
+    m = __float2bfloat16_rn(r1);
+    l = __float2bfloat16_rn(r1 - __bfloat162float(m));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
+    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+}
+
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// A fragment of a row-major [row][k] bf16 tile (row stride `ld` elements): rows r0 + g, r0 + g + 8; k0 + 2tg, + 8
+__device__ __forceinline__ void load_a_frag(uint32_t (&a)[4], const __nv_bfloat16* base, int ld, int r0, int k0, int g, int tg) {
+    const __nv_bfloat16* p0 = base + (size_t)(r0 + g) * ld + k0 + 2 * tg;
+    a[0] = *reinterpret_cast<const uint32_t*>(p0);
+    a[1] = *reinterpret_cast<const uint32_t*>(p0 + 8 * ld);
+    a[2] = *reinterpret_cast<const uint32_t*>(p0 + 8);
+    a[3] = *reinterpret_cast<const uint32_t*>(p0 + 8 * ld + 8);
+}
+
+// Geometry of the tensor-core slab contractions in shared memory (element counts, bf16 unless noted)
+struct TcLayout {
+    int n1p;      // n1 rounded up to 16 (contraction depth of the first stage)
+    int mt;       // 16-row tiles of the slab
+    int xs;       // row stride of x [n1p][n2 + 8]
+    int ps;       // row stride of the P1^T terms [3][16 mt][n1p + 8]
+    int zs;       // row stride of the Z' terms [3][16 mt][n2 + 8] and of the P2 terms [3][n2][n2 + 8]
+};
+
+__host__ __device__ inline TcLayout tc_layout(int n1, int n2, int slab_rows) {
+    TcLayout L;
+    L.n1p = (n1 + 15) / 16 * 16;
+    L.mt = (slab_rows + 15) / 16;
+    L.xs = n2 + 8;
+    L.ps = L.n1p + 8;
+    L.zs = n2 + 8;
+    return L;
+}
+// bytes of x, the P1^T terms, the Z' terms and the P2 terms, in this order; each a multiple of 16
+__host__ __device__ inline size_t tc_x_bytes(const TcLayout& L) { return (size_t)L.n1p * L.xs * 2; }
+__host__ __device__ inline size_t tc_p1_bytes(const TcLayout& L) { return (size_t)3 * 16 * L.mt * L.ps * 2; }
+__host__ __device__ inline size_t tc_z_bytes(const TcLayout& L) { return (size_t)3 * 16 * L.mt * L.zs * 2; }
+__host__ __device__ inline size_t tc_p2_bytes(const TcLayout& L, int n2) { return (size_t)3 * n2 * L.zs * 2; }
+
+// Z' = (P1^T X)[slab] as three bf16 terms.  Each warp takes column tiles of 8 in turn.
+__device__ __forceinline__ void tc_stage_a(const TcLayout& L, int n2, const __nv_bfloat16* Xp, const __nv_bfloat16* P1T,
+                                           __nv_bfloat16* ZT) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int g = lane >> 2, tg = lane & 3;
+    const int rows16 = 16 * L.mt;
+    for (int nt = warp; nt < (n2 >> 3); nt += nwarps) {
+        float acc[4][4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[m][i] = 0.f;
+        for (int ks = 0; ks < (L.n1p >> 4); ++ks) {
+            // x is stored [k][n]: the transposing matrix load gives the B fragment (k pairs for column g)
+            uint32_t b0, b1;
+            const uint32_t addr = smem_u32(Xp + (size_t)(ks * 16 + (lane & 15)) * L.xs + nt * 8);
+            asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                if (m < L.mt) {
+                    float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int term = 2; term >= 0; --term) {          // lo, mid, hi
+                        uint32_t a[4];
+                        load_a_frag(a, P1T + (size_t)term * rows16 * L.ps, L.ps, 16 * m, 16 * ks, g, tg);
+                        mma_bf16(c, a, b0, b1);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[m][i] += c[i];
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            if (m < L.mt) {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+                    split3(acc[m][2 * half], h0, m0, l0);
+                    split3(acc[m][2 * half + 1], h1, m1, l1);
+                    __nv_bfloat16* dst = ZT + (size_t)(16 * m + g + 8 * half) * L.zs + nt * 8 + 2 * tg;
+                    *reinterpret_cast<uint32_t*>(dst) = pack_bf16(h0, h1);
+                    *reinterpret_cast<uint32_t*>(dst + (size_t)rows16 * L.zs) = pack_bf16(m0, m1);
+                    *reinterpret_cast<uint32_t*>(dst + (size_t)2 * rows16 * L.zs) = pack_bf16(l0, l1);
+                }
+            }
+        }
+    }
+}
+
+// Y[slab] = Z' P2 from the terms of both; the real rows go to Y (fp32, row stride n2); returns the largest magnitude.
+__device__ __forceinline__ float tc_stage_b(const TcLayout& L, int n2, int rows, const __nv_bfloat16* ZT,
+                                            const __nv_bfloat16* P2T, float* Y) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int g = lane >> 2, tg = lane & 3;
+    const int rows16 = 16 * L.mt;
+    float amax = 0.f;
+    for (int nt = warp; nt < (n2 >> 3); nt += nwarps) {
+        float acc[4][4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[m][i] = 0.f;
+        for (int ks = 0; ks < (n2 >> 4); ++ks) {
+            uint32_t b[3][2];                                         // P2 terms hi, mid, lo, stored [k][column] like x
+#pragma unroll
+            for (int term = 0; term < 3; ++term) {
+                const uint32_t addr = smem_u32(P2T + ((size_t)term * n2 + ks * 16 + (lane & 15)) * L.zs + nt * 8);
+                asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];"
+                             : "=r"(b[term][0]), "=r"(b[term][1]) : "r"(addr));
+            }
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                if (m < L.mt) {
+                    uint32_t a[3][4];
+#pragma unroll
+                    for (int term = 0; term < 3; ++term)
+                        load_a_frag(a[term], ZT + (size_t)term * rows16 * L.zs, L.zs, 16 * m, 16 * ks, g, tg);
+                    float c[4] = {0.f, 0.f, 0.f, 0.f};
+                    // products of terms whose weight is at least 2^-16 of the leading one, smallest first
+                    mma_bf16(c, a[1], b[1][0], b[1][1]);
+                    mma_bf16(c, a[2], b[0][0], b[0][1]);
+                    mma_bf16(c, a[0], b[2][0], b[2][1]);
+                    mma_bf16(c, a[1], b[0][0], b[0][1]);
+                    mma_bf16(c, a[0], b[1][0], b[1][1]);
+                    mma_bf16(c, a[0], b[0][0], b[0][1]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[m][i] += c[i];
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            if (m < L.mt) {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int r = 16 * m + g + 8 * half;
+                    if (r < rows) {
+                        const float v0 = acc[m][2 * half], v1 = acc[m][2 * half + 1];
+                        *reinterpret_cast<float2*>(Y + (size_t)r * n2 + nt * 8 + 2 * tg) = make_float2(v0, v1);
+                        amax = fmaxf(amax, fmaxf(fabsf(v0), fabsf(v1)));
+                    }
+                }
+            }
+        }
+    }
+    return amax;
+}
+
 // x_t[first .. first+len) -> fp32 in shared memory
 __device__ __forceinline__ void load_x(const __nv_bfloat16* __restrict__ xt, int len, float* Xs) {
     if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0 && (len & 7) == 0) {
@@ -327,7 +497,67 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     if (threadIdx.x == 0) red_sum = 0;
 
     BWLA_PSTAMP(0);
-    if (p.split_y) {
+    if (p.split_y && p.sp_tc) {
+        // ---- few tokens, tensor-core contractions: this CTA's rows of Y from all of x
+        const TcLayout L = tc_layout(n1, n2, p.sp_rp);
+        uint8_t* base = reinterpret_cast<uint8_t*>(smem);
+        __nv_bfloat16* Xp = reinterpret_cast<__nv_bfloat16*>(base);                       // x, later this CTA's rows of Y (fp32)
+        __nv_bfloat16* P1T = reinterpret_cast<__nv_bfloat16*>(base + tc_x_bytes(L));
+        __nv_bfloat16* ZT = reinterpret_cast<__nv_bfloat16*>(base + tc_x_bytes(L) + tc_p1_bytes(L));
+        __nv_bfloat16* P2T = reinterpret_cast<__nv_bfloat16*>(base + tc_x_bytes(L) + tc_p1_bytes(L) + tc_z_bytes(L));
+        slots = reinterpret_cast<float*>(base + tc_x_bytes(L) + tc_p1_bytes(L) + tc_z_bytes(L) + tc_p2_bytes(L, n2));
+        // the layer's constants, split into bf16 terms (P2 keeps its [k][column] order: the B fragments come from
+        // transposing matrix loads, as for x)
+        for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x) {
+            const int b = (4 * i) / n2, d = 4 * i - b * n2;
+            const float4 v = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
+            __nv_bfloat16 h[4], m[4], l[4];
+            split3(v.x, h[0], m[0], l[0]); split3(v.y, h[1], m[1], l[1]);
+            split3(v.z, h[2], m[2], l[2]); split3(v.w, h[3], m[3], l[3]);
+            __nv_bfloat16* dst = P2T + (size_t)b * L.zs + d;
+            *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
+            *reinterpret_cast<uint2*>(dst + (size_t)n2 * L.zs) = make_uint2(pack_bf16(m[0], m[1]), pack_bf16(m[2], m[3]));
+            *reinterpret_cast<uint2*>(dst + (size_t)2 * n2 * L.zs) = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
+        }
+        for (int i = threadIdx.x; i < 16 * L.mt * L.n1p; i += blockDim.x) {
+            const int r = i / L.n1p, a = i - r * L.n1p;
+            const float v = (r < rows && a < n1) ? __ldg(p.P1 + (size_t)a * n1 + a_lo + r) : 0.f;
+            __nv_bfloat16 h, m, l;
+            split3(v, h, m, l);
+            __nv_bfloat16* dst = P1T + (size_t)r * L.ps + a;
+            dst[0] = h; dst[(size_t)16 * L.mt * L.ps] = m; dst[(size_t)2 * 16 * L.mt * L.ps] = l;
+        }
+        cluster_arrive_release();              // "this CTA is running": waited for before the first remote store
+        if (!p.late_trigger) griddep_launch_dependents();
+        griddep_wait();                        // x may be the output of the preceding kernel
+        BWLA_PSTAMP(1); BWLA_PBLOCK(2);
+        {
+            const __nv_bfloat16* xt = p.x + t * p.ldx;
+            const int cpr = n2 >> 3;           // 16-byte chunks per row of X
+            if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0) {
+                for (int i = threadIdx.x; i < n1 * cpr; i += blockDim.x) {
+                    const int a = i / cpr, c = i - a * cpr;
+                    *reinterpret_cast<uint4*>(Xp + (size_t)a * L.xs + 8 * c) = __ldg(reinterpret_cast<const uint4*>(xt) + i);
+                }
+            } else {
+                for (int k = threadIdx.x; k < K; k += blockDim.x) Xp[(size_t)(k / n2) * L.xs + k % n2] = xt[k];
+            }
+            // rows of the depth padding must be finite: 0 * garbage could be NaN
+            for (int i = threadIdx.x; i < (L.n1p - n1) * cpr; i += blockDim.x) {
+                const int a = n1 + i / cpr, c = i % cpr;
+                *reinterpret_cast<uint4*>(Xp + (size_t)a * L.xs + 8 * c) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        __syncthreads();
+        BWLA_PSTAMP(2);
+        tc_stage_a(L, n2, Xp, P1T, ZT);
+        __syncthreads();
+        BWLA_PSTAMP(3);
+        amax = tc_stage_b(L, n2, rows, ZT, P2T, Xs);
+        BWLA_PSTAMP(4);
+        cluster_wait_acquire();
+        BWLA_PSTAMP(5);
+    } else if (p.split_y) {
         // ---- few tokens: this CTA's rows of Y from all of x; nothing but absmax and code sums is exchanged
         const int rp = p.sp_rp, S = p.sp_s;
         __nv_bfloat16* Xh = reinterpret_cast<__nv_bfloat16*>(smem);   // all of x_t as it comes; later this CTA's rows of Y (fp32)
@@ -851,6 +1081,20 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                 // all of x (bf16), this CTA's rows of Z' (transposed), all of P2, this CTA's columns of P1, partial sums
                 if ((K & 7) != 0) return false;
                 p.split_y = 1;
+                p.sp_tc = 0;
+                if (n2 % 16 == 0 && (cap + 15) / 16 <= 4) {
+                    // both contractions on the warp-level tensor-core path when the split operands fit
+                    const TcLayout L = tc_layout(n1, n2, cap);
+                    const size_t bytes = tc_x_bytes(L) + tc_p1_bytes(L) + tc_z_bytes(L) + tc_p2_bytes(L, n2) + 64;
+                    if (bytes <= (size_t)kPrologueSmemFloats * 4) {
+                        p.sp_tc = 1; p.sp_rp = cap; p.sp_tr = 0; p.sp_s = 1;
+                        p.ps_cap = 0; p.p1_cap = 0; p.ch1 = n2; p.ch2 = cap; p.tr1 = p.tr2 = 1;
+                        threads = 32 * (n2 / 8);
+                        threads = threads < 256 ? 256 : (threads > 512 ? 512 : threads);
+                        smem = bytes;
+                        return true;
+                    }
+                }
                 // thread tiles of 8 rows unless padding the slab to a multiple of 8 wastes more than 15 %
                 p.sp_tr = ((cap + 7) / 8 * 8) * 100 <= cap * 115 ? 8 : 4;
                 p.sp_rp = (cap + p.sp_tr - 1) / p.sp_tr * p.sp_tr;
