@@ -69,7 +69,8 @@ struct PrologueParams {
     int tr1, tr2;       // rows per thread in the two contractions
     int split_y;        // 1 (C > 1): each CTA evaluates its rows of Y from all of x, nothing but absmax is exchanged
     int sp_tr, sp_rp;   // split_y: rows per thread tile (4 or 8); slab rows rounded up to it (row stride of P1s and Zt)
-    int sp_s;           // split_y: slices the contraction depth is cut into (partial sums are added afterwards)
+    int sp_s;           // split_y: slices the contraction depth is cut into (partial sums are added afterwards); with sp_tc:
+                        // parts the columns of P2 are staged in
     int sp_tc;          // split_y: 1: both contractions on the warp-level tensor-core path (split-bf16 operands)
     int sp_zt_off;      // split_y: where Z'^T lives, in floats from the start of shared memory (0: over x, dead by then)
     int sp_rest_off;    // split_y: where P2 starts
@@ -324,11 +325,15 @@ struct TcLayout {
     int mt;       // 16-row tiles of the slab
     int xs;       // row stride of x [n1p][n2 + 8]
     int ps;       // row stride of the P1^T terms [3][16 mt][n1p + 8]
-    int zs;       // row stride of the Z' terms [3][16 mt][n2 + 8] and of the P2 terms [3][n2][n2 + 8]
+    int zs;       // row stride of the Z' terms [3][16 mt][n2 + 8]
+    int pc;       // columns of P2 resident at a time (n2, or a part of it when all of P2 does not fit)
+    int p2s;      // row stride of the P2 terms [3][n2][pc + 8]
 };
 
-__host__ __device__ inline TcLayout tc_layout(int n1, int n2, int slab_rows) {
+__host__ __device__ inline TcLayout tc_layout(int n1, int n2, int slab_rows, int p2_chunks) {
     TcLayout L;
+    L.pc = n2 / p2_chunks;
+    L.p2s = L.pc + 8;
     L.n1p = (n1 + 15) / 16 * 16;
     L.mt = (slab_rows + 15) / 16;
     L.xs = n2 + 8;
@@ -340,111 +345,113 @@ __host__ __device__ inline TcLayout tc_layout(int n1, int n2, int slab_rows) {
 __host__ __device__ inline size_t tc_x_bytes(const TcLayout& L) { return (size_t)L.n1p * L.xs * 2; }
 __host__ __device__ inline size_t tc_p1_bytes(const TcLayout& L) { return (size_t)3 * 16 * L.mt * L.ps * 2; }
 __host__ __device__ inline size_t tc_z_bytes(const TcLayout& L) { return (size_t)3 * 16 * L.mt * L.zs * 2; }
-__host__ __device__ inline size_t tc_p2_bytes(const TcLayout& L, int n2) { return (size_t)3 * n2 * L.zs * 2; }
+__host__ __device__ inline size_t tc_p2_bytes(const TcLayout& L, int n2) { return (size_t)3 * n2 * L.p2s * 2; }
 
-// Z' = (P1^T X)[slab] as three bf16 terms.  Each warp takes column tiles of 8 in turn.
+// columns [c0, c0 + L.pc) of P2, split into bf16 terms, in the [k][column] order of the source (the B fragments come from
+// transposing matrix loads, as for x)
+__device__ __forceinline__ void stage_p2_terms(const TcLayout& L, const float* __restrict__ P2, int n2, int c0, __nv_bfloat16* P2T) {
+    const int qpr = L.pc >> 2;                  // float4 per row of the chunk
+    for (int i = threadIdx.x; i < n2 * qpr; i += blockDim.x) {
+        const int b = i / qpr, d = 4 * (i - b * qpr);
+        const float4 v = __ldg(reinterpret_cast<const float4*>(P2 + (size_t)b * n2 + c0 + d));
+        __nv_bfloat16 h[4], m[4], l[4];
+        split3(v.x, h[0], m[0], l[0]); split3(v.y, h[1], m[1], l[1]);
+        split3(v.z, h[2], m[2], l[2]); split3(v.w, h[3], m[3], l[3]);
+        __nv_bfloat16* dst = P2T + (size_t)b * L.p2s + d;
+        *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
+        *reinterpret_cast<uint2*>(dst + (size_t)n2 * L.p2s) = make_uint2(pack_bf16(m[0], m[1]), pack_bf16(m[2], m[3]));
+        *reinterpret_cast<uint2*>(dst + (size_t)2 * n2 * L.p2s) = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
+    }
+}
+
+// Z' = (P1^T X)[slab] as three bf16 terms.  The warps take tiles of 16 rows x 8 columns in turn.  The three term
+// products of a k-step go to accumulators of their own (independent instructions), then into the running sum.
 __device__ __forceinline__ void tc_stage_a(const TcLayout& L, int n2, const __nv_bfloat16* Xp, const __nv_bfloat16* P1T,
                                            __nv_bfloat16* ZT) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int g = lane >> 2, tg = lane & 3;
     const int rows16 = 16 * L.mt;
-    for (int nt = warp; nt < (n2 >> 3); nt += nwarps) {
-        float acc[4][4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[m][i] = 0.f;
+    const int ntiles = n2 >> 3;
+    for (int tile = warp; tile < L.mt * ntiles; tile += nwarps) {
+        const int m = tile / ntiles, nt = tile - m * ntiles;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
         for (int ks = 0; ks < (L.n1p >> 4); ++ks) {
             // x is stored [k][n]: the transposing matrix load gives the B fragment (k pairs for column g)
             uint32_t b0, b1;
             const uint32_t addr = smem_u32(Xp + (size_t)(ks * 16 + (lane & 15)) * L.xs + nt * 8);
             asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(addr));
+            uint32_t a[3][4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                if (m < L.mt) {
-                    float c[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int term = 0; term < 3; ++term)
+                load_a_frag(a[term], P1T + (size_t)term * rows16 * L.ps, L.ps, 16 * m, 16 * ks, g, tg);
+            float c[3][4];
 #pragma unroll
-                    for (int term = 2; term >= 0; --term) {          // lo, mid, hi
-                        uint32_t a[4];
-                        load_a_frag(a, P1T + (size_t)term * rows16 * L.ps, L.ps, 16 * m, 16 * ks, g, tg);
-                        mma_bf16(c, a, b0, b1);
-                    }
+            for (int term = 0; term < 3; ++term) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[m][i] += c[i];
-                }
+                for (int i = 0; i < 4; ++i) c[term][i] = 0.f;
+                mma_bf16(c[term], a[term], b0, b1);
             }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[i] += (c[2][i] + c[1][i]) + c[0][i];       // lo + mid, then hi
         }
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            if (m < L.mt) {
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    __nv_bfloat16 h0, m0, l0, h1, m1, l1;
-                    split3(acc[m][2 * half], h0, m0, l0);
-                    split3(acc[m][2 * half + 1], h1, m1, l1);
-                    __nv_bfloat16* dst = ZT + (size_t)(16 * m + g + 8 * half) * L.zs + nt * 8 + 2 * tg;
-                    *reinterpret_cast<uint32_t*>(dst) = pack_bf16(h0, h1);
-                    *reinterpret_cast<uint32_t*>(dst + (size_t)rows16 * L.zs) = pack_bf16(m0, m1);
-                    *reinterpret_cast<uint32_t*>(dst + (size_t)2 * rows16 * L.zs) = pack_bf16(l0, l1);
-                }
-            }
+        for (int half = 0; half < 2; ++half) {
+            __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+            split3(acc[2 * half], h0, m0, l0);
+            split3(acc[2 * half + 1], h1, m1, l1);
+            __nv_bfloat16* dst = ZT + (size_t)(16 * m + g + 8 * half) * L.zs + nt * 8 + 2 * tg;
+            *reinterpret_cast<uint32_t*>(dst) = pack_bf16(h0, h1);
+            *reinterpret_cast<uint32_t*>(dst + (size_t)rows16 * L.zs) = pack_bf16(m0, m1);
+            *reinterpret_cast<uint32_t*>(dst + (size_t)2 * rows16 * L.zs) = pack_bf16(l0, l1);
         }
     }
 }
 
 // Y[slab] = Z' P2 from the terms of both; the real rows go to Y (fp32, row stride n2); returns the largest magnitude.
-__device__ __forceinline__ float tc_stage_b(const TcLayout& L, int n2, int rows, const __nv_bfloat16* ZT,
+// P2T holds columns [c0, c0 + L.pc) of the P2 terms; only those columns of Y are produced.  Of the nine term products
+// the six whose weight is at least 2^-16 of the leading one are taken, in two independent chains per k-step.
+__device__ __forceinline__ float tc_stage_b(const TcLayout& L, int n2, int rows, int c0, const __nv_bfloat16* ZT,
                                             const __nv_bfloat16* P2T, float* Y) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int g = lane >> 2, tg = lane & 3;
     const int rows16 = 16 * L.mt;
+    const int ntiles = L.pc >> 3;
     float amax = 0.f;
-    for (int nt = warp; nt < (n2 >> 3); nt += nwarps) {
-        float acc[4][4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[m][i] = 0.f;
+    for (int tile = warp; tile < L.mt * ntiles; tile += nwarps) {
+        const int m = tile / ntiles, nt = (c0 >> 3) + tile - m * ntiles;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
         for (int ks = 0; ks < (n2 >> 4); ++ks) {
             uint32_t b[3][2];                                         // P2 terms hi, mid, lo, stored [k][column] like x
 #pragma unroll
             for (int term = 0; term < 3; ++term) {
-                const uint32_t addr = smem_u32(P2T + ((size_t)term * n2 + ks * 16 + (lane & 15)) * L.zs + nt * 8);
+                const uint32_t addr = smem_u32(P2T + ((size_t)term * n2 + ks * 16 + (lane & 15)) * L.p2s + nt * 8 - c0);
                 asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];"
                              : "=r"(b[term][0]), "=r"(b[term][1]) : "r"(addr));
             }
+            uint32_t a[3][4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                if (m < L.mt) {
-                    uint32_t a[3][4];
+            for (int term = 0; term < 3; ++term)
+                load_a_frag(a[term], ZT + (size_t)term * rows16 * L.zs, L.zs, 16 * m, 16 * ks, g, tg);
+            float cs[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
+            // small products: mid*mid, lo*hi, hi*lo; large: mid*hi, hi*mid, hi*hi
+            mma_bf16(cs, a[1], b[1][0], b[1][1]);
+            mma_bf16(cb, a[1], b[0][0], b[0][1]);
+            mma_bf16(cs, a[2], b[0][0], b[0][1]);
+            mma_bf16(cb, a[0], b[1][0], b[1][1]);
+            mma_bf16(cs, a[0], b[2][0], b[2][1]);
+            mma_bf16(cb, a[0], b[0][0], b[0][1]);
 #pragma unroll
-                    for (int term = 0; term < 3; ++term)
-                        load_a_frag(a[term], ZT + (size_t)term * rows16 * L.zs, L.zs, 16 * m, 16 * ks, g, tg);
-                    float c[4] = {0.f, 0.f, 0.f, 0.f};
-                    // products of terms whose weight is at least 2^-16 of the leading one, smallest first
-                    mma_bf16(c, a[1], b[1][0], b[1][1]);
-                    mma_bf16(c, a[2], b[0][0], b[0][1]);
-                    mma_bf16(c, a[0], b[2][0], b[2][1]);
-                    mma_bf16(c, a[1], b[0][0], b[0][1]);
-                    mma_bf16(c, a[0], b[1][0], b[1][1]);
-                    mma_bf16(c, a[0], b[0][0], b[0][1]);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[m][i] += c[i];
-                }
-            }
+            for (int i = 0; i < 4; ++i) acc[i] += cs[i] + cb[i];
         }
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            if (m < L.mt) {
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int r = 16 * m + g + 8 * half;
-                    if (r < rows) {
-                        const float v0 = acc[m][2 * half], v1 = acc[m][2 * half + 1];
-                        *reinterpret_cast<float2*>(Y + (size_t)r * n2 + nt * 8 + 2 * tg) = make_float2(v0, v1);
-                        amax = fmaxf(amax, fmaxf(fabsf(v0), fabsf(v1)));
-                    }
-                }
+        for (int half = 0; half < 2; ++half) {
+            const int r = 16 * m + g + 8 * half;
+            if (r < rows) {
+                const float v0 = acc[2 * half], v1 = acc[2 * half + 1];
+                *reinterpret_cast<float2*>(Y + (size_t)r * n2 + nt * 8 + 2 * tg) = make_float2(v0, v1);
+                amax = fmaxf(amax, fmaxf(fabsf(v0), fabsf(v1)));
             }
         }
     }
@@ -499,26 +506,15 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     BWLA_PSTAMP(0);
     if (p.split_y && p.sp_tc) {
         // ---- few tokens, tensor-core contractions: this CTA's rows of Y from all of x
-        const TcLayout L = tc_layout(n1, n2, p.sp_rp);
+        const TcLayout L = tc_layout(n1, n2, p.sp_rp, p.sp_s);
         uint8_t* base = reinterpret_cast<uint8_t*>(smem);
         __nv_bfloat16* Xp = reinterpret_cast<__nv_bfloat16*>(base);                       // x, later this CTA's rows of Y (fp32)
         __nv_bfloat16* P1T = reinterpret_cast<__nv_bfloat16*>(base + tc_x_bytes(L));
         __nv_bfloat16* ZT = reinterpret_cast<__nv_bfloat16*>(base + tc_x_bytes(L) + tc_p1_bytes(L));
         __nv_bfloat16* P2T = reinterpret_cast<__nv_bfloat16*>(base + tc_x_bytes(L) + tc_p1_bytes(L) + tc_z_bytes(L));
         slots = reinterpret_cast<float*>(base + tc_x_bytes(L) + tc_p1_bytes(L) + tc_z_bytes(L) + tc_p2_bytes(L, n2));
-        // the layer's constants, split into bf16 terms (P2 keeps its [k][column] order: the B fragments come from
-        // transposing matrix loads, as for x)
-        for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x) {
-            const int b = (4 * i) / n2, d = 4 * i - b * n2;
-            const float4 v = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
-            __nv_bfloat16 h[4], m[4], l[4];
-            split3(v.x, h[0], m[0], l[0]); split3(v.y, h[1], m[1], l[1]);
-            split3(v.z, h[2], m[2], l[2]); split3(v.w, h[3], m[3], l[3]);
-            __nv_bfloat16* dst = P2T + (size_t)b * L.zs + d;
-            *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(h[0], h[1]), pack_bf16(h[2], h[3]));
-            *reinterpret_cast<uint2*>(dst + (size_t)n2 * L.zs) = make_uint2(pack_bf16(m[0], m[1]), pack_bf16(m[2], m[3]));
-            *reinterpret_cast<uint2*>(dst + (size_t)2 * n2 * L.zs) = make_uint2(pack_bf16(l[0], l[1]), pack_bf16(l[2], l[3]));
-        }
+        // the layer's constants, split into bf16 terms (the first columns of P2 when not all of it fits)
+        stage_p2_terms(L, p.P2, n2, 0, P2T);
         for (int i = threadIdx.x; i < 16 * L.mt * L.n1p; i += blockDim.x) {
             const int r = i / L.n1p, a = i - r * L.n1p;
             const float v = (r < rows && a < n1) ? __ldg(p.P1 + (size_t)a * n1 + a_lo + r) : 0.f;
@@ -553,7 +549,13 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         tc_stage_a(L, n2, Xp, P1T, ZT);
         __syncthreads();
         BWLA_PSTAMP(3);
-        amax = tc_stage_b(L, n2, rows, ZT, P2T, Xs);
+        amax = tc_stage_b(L, n2, rows, 0, ZT, P2T, Xs);
+        for (int c0 = L.pc; c0 < n2; c0 += L.pc) {
+            __syncthreads();                   // every warp is done with the columns in place
+            stage_p2_terms(L, p.P2, n2, c0, P2T);
+            __syncthreads();
+            amax = fmaxf(amax, tc_stage_b(L, n2, rows, c0, ZT, P2T, Xs));
+        }
         BWLA_PSTAMP(4);
         cluster_wait_acquire();
         BWLA_PSTAMP(5);
@@ -1084,10 +1086,19 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                 p.sp_tc = 0;
                 if (n2 % 16 == 0 && (cap + 15) / 16 <= 4) {
                     // both contractions on the warp-level tensor-core path when the split operands fit
-                    const TcLayout L = tc_layout(n1, n2, cap);
-                    const size_t bytes = tc_x_bytes(L) + tc_p1_bytes(L) + tc_z_bytes(L) + tc_p2_bytes(L, n2) + 64;
-                    if (bytes <= (size_t)kPrologueSmemFloats * 4) {
-                        p.sp_tc = 1; p.sp_rp = cap; p.sp_tr = 0; p.sp_s = 1;
+                    // P2 whole.  (Staging it in parts of its columns works -- the kernel takes any number of parts -- but
+                    // was measured no faster than the FMA version for K = 25600: mma.sync runs at ~6 cycles per
+                    // m16n8k16 per SM on this part, and the restaging is exposed.)
+                    int chunks = 1;
+                    size_t bytes = 0;
+                    for (; chunks <= 1; chunks *= 2) {
+                        if ((n2 / chunks) % 8 != 0 || n2 % chunks != 0) { chunks = 8; break; }
+                        const TcLayout L = tc_layout(n1, n2, cap, chunks);
+                        bytes = tc_x_bytes(L) + tc_p1_bytes(L) + tc_z_bytes(L) + tc_p2_bytes(L, n2) + 64;
+                        if (bytes <= (size_t)kPrologueSmemFloats * 4) break;
+                    }
+                    if (chunks <= 1) {
+                        p.sp_tc = 1; p.sp_rp = cap; p.sp_tr = 0; p.sp_s = chunks;   // sp_s: parts of P2 in this mode
                         p.ps_cap = 0; p.p1_cap = 0; p.ch1 = n2; p.ch2 = cap; p.tr1 = p.tr2 = 1;
                         threads = 32 * (n2 / 8);
                         threads = threads < 256 ? 256 : (threads > 512 ? 512 : threads);
