@@ -63,6 +63,10 @@ constexpr int kStatusBytes = 256;        // word 0: status; words 1..: where a b
 #endif
 constexpr int kLowrankPad = 64;          // T is kept as bf16 [3][M][64] (T = hi + mid + lo), zero beyond r <= 64
 
+// The code sum of a token is kept as kQsumParts partial sums (one per CTA of the prologue cluster that quantised a slab
+// of the token; unused parts are zero): the consumer adds them, the producers need no exchange.
+constexpr int kQsumParts = 8;
+
 __host__ __device__ inline int lowrank_cols(int r) { return r > kLowrankPad ? (r + 1) / 2 * 2 : kLowrankPad; }
 
 struct Workspace {
@@ -74,7 +78,7 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     size_t off = 0;
     w.status = off; off += kStatusBytes;
     w.scales = off; off += align_up((size_t)M * 4, 256);
-    w.qsum = off;   off += align_up((size_t)M * 4, 256);
+    w.qsum = off;   off += align_up((size_t)M * 4 * kQsumParts, 256);
     const size_t lr_cols = (size_t)lowrank_cols(r);
     w.T = off;      off += align_up((size_t)M * lr_cols * 6, 256);     // bf16 [3][M][cols]
     w.codes = off;  off += align_up((size_t)M * (size_t)K, 256);
@@ -91,20 +95,20 @@ int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ld
 
 // One launch: fused rotate + absmax + quantise (skipped when codes == NULL) and T = V x (skipped when r == 0 or
 // Thl == NULL).  codes_layout: 0 = natural k order, 1 = interleaved order used by the tensor-core contraction (inside
-// each group of 32, position 4*j + i holds k = j + 8*i).  qsum (int32 [M]) may be NULL.
+// each group of 32, position 4*j + i holds k = j + 8*i).  qsum (int32 [M][kQsumParts], partial sums) may be NULL.
 // Thl: bf16 [3][M][cols], cols = lowrank_cols(r): T as the sum of three bf16 terms (exact for an fp32 T).
 int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2, int n2,
                     int bits, int8_t* codes, int codes_layout, float* scales, int32_t* qsum, const void* V, int r,
                     void* Thl, cudaStream_t stream);
 
-// qsum[t] = sum_k codes[t][k]; optionally rewrites natural-order codes into the interleaved order.
+// qsum[t][0] = sum_k codes[t][k] (the other parts zero); optionally rewrites natural-order codes into the interleaved order.
 int launch_prepare_codes(const int8_t* codes, int64_t M, int64_t K, int8_t* codes_interleaved, int32_t* qsum,
                          cudaStream_t stream);
 
 struct GemmArgs {
     const int8_t* codes;      // [M][K]; natural order for the simple path
     const float* scales;      // [M]
-    const int32_t* qsum;      // [M]
+    const int32_t* qsum;      // [M][kQsumParts] partial sums
     int64_t M, K, N;
     int bits;
     const uint32_t* packed;   // [N][K/32]

@@ -58,7 +58,11 @@ __global__ void __launch_bounds__(128) gemm_simple_kernel(GemmArgs a) {
                     l = fmaf(__bfloat162float(u[j]), (__bfloat162float(hi[j]) + __bfloat162float(mid[j])) + __bfloat162float(lo[j]), l);
                 y += l;
             }
-            if (a.mu) y = fmaf(__fmul_rn(a.mu[n], sc), (float)a.qsum[t], y);
+            if (a.mu) {
+                int32_t qs = 0;
+                for (int c = 0; c < kQsumParts; ++c) qs += a.qsum[t * kQsumParts + c];
+                y = fmaf(__fmul_rn(a.mu[n], sc), (float)qs, y);
+            }
             ((__nv_bfloat16*)a.out)[t * a.ldo + n] = __float2bfloat16_rn(y);
         }
     }

@@ -50,7 +50,7 @@ struct UmmaParams {
     int total_units, splits;
     int r;                       // low-rank width, 0..kLowrankPad
     const float* scales;         // [M]
-    const int32_t* qsum;         // [M]
+    const int32_t* qsum;         // [M][kQsumParts] partial sums
     const float* alpha;          // [N]
     const float* mu;             // [N] or NULL
     const __nv_bfloat16* U;      // [N][r] or NULL
@@ -260,7 +260,13 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         for (int i = lane; i < N_TOK; i += 32) {
             const int t = t0 + i;
             scale_s[i] = t < p.M ? p.scales[t] : 0.f;
-            qsum_s[i] = t < p.M ? p.qsum[t] : 0;
+            int32_t qs = 0;
+            if (t < p.M) {
+                const int4* parts = reinterpret_cast<const int4*>(p.qsum + (size_t)t * kQsumParts);
+                const int4 a = parts[0], b = parts[1];
+                qs = a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w;
+            }
+            qsum_s[i] = qs;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(s_full);

@@ -495,7 +495,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     const int a_lo = slab_begin(rank, C, n1, p.row_gran), a_hi = slab_begin(rank + 1, C, n1, p.row_gran);
     const int rows = a_hi - a_lo;
     float* Xs = smem;                          // this CTA's rows of Y end up here in every mode
-    float* slots;                              // [0..7] absmax per rank, [8..15] code sum per rank (int)
+    float* slots;                              // [0..7] absmax per rank
     __shared__ float red_max[32];
     __shared__ int red_sum;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -742,16 +742,14 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     if (lane == 0 && local_sum != 0) atomicAdd(&red_sum, local_sum);
     __syncthreads();
     BWLA_PSTAMP(9);
-    if (C > 1) {
-        if (threadIdx.x == 0) st_cluster_u32(map_shared_rank(smem_u32(slots + 8 + rank), 0), (uint32_t)red_sum);
-        cluster_arrive_release();
-        cluster_wait_acquire();
-    }
-    if (rank == 0 && threadIdx.x == 0) {
-        int s = red_sum;
-        if (C > 1) { s = 0; for (int c = 0; c < C; ++c) s += (int)__float_as_uint(slots[8 + c]); }
-        p.scales[t] = scale;
-        if (p.qsum) p.qsum[t] = s;
+    // every CTA leaves its own part of the token's code sum; the consumer adds the parts, so no exchange is needed here
+    if (threadIdx.x == 0) {
+        if (p.qsum) {
+            p.qsum[t * kQsumParts + rank] = red_sum;
+            if (rank == 0)
+                for (int c = C; c < kQsumParts; ++c) p.qsum[t * kQsumParts + c] = 0;
+        }
+        if (rank == 0) p.scales[t] = scale;
     }
     BWLA_PSTAMP(10);
 }
@@ -1266,7 +1264,7 @@ __global__ void __launch_bounds__(256) prepare_codes_kernel(const int8_t* __rest
     local = warp_sum(local);
     if ((threadIdx.x & 31) == 0 && local != 0) atomicAdd(&red_sum, local);
     __syncthreads();
-    if (threadIdx.x == 0 && qsum) qsum[t] = red_sum;
+    if (threadIdx.x < kQsumParts && qsum) qsum[t * kQsumParts + threadIdx.x] = threadIdx.x == 0 ? red_sum : 0;
 }
 
 int launch_prepare_codes(const int8_t* codes, int64_t M, int64_t K, int8_t* codes_interleaved, int32_t* qsum,
