@@ -1098,8 +1098,9 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                     if (chunks <= 1) {
                         p.sp_tc = 1; p.sp_rp = cap; p.sp_tr = 0; p.sp_s = chunks;   // sp_s: parts of P2 in this mode
                         p.ps_cap = 0; p.p1_cap = 0; p.ch1 = n2; p.ch2 = cap; p.tr1 = p.tr2 = 1;
-                        threads = 32 * (n2 / 8);
-                        threads = threads < 256 ? 256 : (threads > 512 ? 512 : threads);
+                        // all the warps a block may have: splitting the constants into terms is instruction-bound, and a
+                        // block of this kernel cannot share an SM with the contraction CTAs before it in any case
+                        threads = 512;
                         smem = bytes;
                         return true;
                     }
