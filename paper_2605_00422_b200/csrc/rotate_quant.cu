@@ -458,6 +458,17 @@ __device__ __forceinline__ float tc_stage_b(const TcLayout& L, int n2, int rows,
     return amax;
 }
 
+// asynchronous copies global -> shared (no register in between, so all of a thread's copies are in flight at once)
+__device__ __forceinline__ void cp_async_16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_4(void* dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
 // x_t[first .. first+len) -> fp32 in shared memory
 __device__ __forceinline__ void load_x(const __nv_bfloat16* __restrict__ xt, int len, float* Xs) {
     if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0 && (len & 7) == 0) {
@@ -568,12 +579,17 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         float* P1s = P2s + p.ps_cap;           // columns [a_lo, a_hi) of P1: [n1][rp]
         float* part = P1s + p.p1_cap;          // [S][rp][n2] partial sums
         slots = part + S * rp * n2;
-        // the layer's constants do not depend on the preceding kernel
-        for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x)
-            *reinterpret_cast<float4*>(P2s + 4 * i) = __ldg(reinterpret_cast<const float4*>(p.P2) + i);
-        load_p1_columns(p.P1, n1, a_lo, rows, rp, P1s);
+        // the layer's constants do not depend on the preceding kernel; asynchronous copies, so that one round trip
+        // brings all of them (with a load and a store per loop iteration it was one round trip per iteration)
+        for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x) cp_async_16(P2s + 4 * i, p.P2 + 4 * i);
+        for (int i = threadIdx.x; i < n1 * rp; i += blockDim.x) {
+            const int a = i / rp, j = i - a * rp;
+            if (j < rows) cp_async_4(P1s + i, p.P1 + (size_t)a * n1 + a_lo + j);
+            else P1s[i] = 0.f;
+        }
         cluster_arrive_release();              // "this CTA is running": waited for before the first remote store
         if (!p.late_trigger) griddep_launch_dependents();
+        cp_async_wait_all();                   // made visible to the block by the barrier behind the load of x
         griddep_wait();                        // x may be the output of the preceding kernel
         BWLA_PSTAMP(1); BWLA_PBLOCK(2);
         {
