@@ -366,8 +366,10 @@ __device__ __forceinline__ void stage_p2_terms(const TcLayout& L, const float* _
 
 // Z' = (P1^T X)[slab] as three bf16 terms.  The warps take tiles of 16 rows x 8 columns in turn.  The three term
 // products of a k-step go to accumulators of their own (independent instructions), then into the running sum.
+// With Zf != nullptr the result is written as fp32, transposed ([column][row], row stride 16 mt), for the FMA version
+// of the second contraction, instead of as terms.
 __device__ __forceinline__ void tc_stage_a(const TcLayout& L, int n2, const __nv_bfloat16* Xp, const __nv_bfloat16* P1T,
-                                           __nv_bfloat16* ZT) {
+                                           __nv_bfloat16* ZT, float* Zf = nullptr) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int g = lane >> 2, tg = lane & 3;
     const int rows16 = 16 * L.mt;
@@ -394,6 +396,15 @@ __device__ __forceinline__ void tc_stage_a(const TcLayout& L, int n2, const __nv
             }
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[i] += (c[2][i] + c[1][i]) + c[0][i];       // lo + mid, then hi
+        }
+        if (Zf) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int r = 16 * m + g + 8 * half;
+                Zf[(size_t)(nt * 8 + 2 * tg) * rows16 + r] = acc[2 * half];
+                Zf[(size_t)(nt * 8 + 2 * tg + 1) * rows16 + r] = acc[2 * half + 1];
+            }
+            continue;
         }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -515,7 +526,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     if (threadIdx.x == 0) red_sum = 0;
 
     BWLA_PSTAMP(0);
-    if (p.split_y && p.sp_tc) {
+    if (p.split_y && p.sp_tc == 1) {
         // ---- few tokens, tensor-core contractions: this CTA's rows of Y from all of x
         const TcLayout L = tc_layout(n1, n2, p.sp_rp, p.sp_s);
         uint8_t* base = reinterpret_cast<uint8_t*>(smem);
@@ -567,6 +578,77 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             __syncthreads();
             amax = fmaxf(amax, tc_stage_b(L, n2, rows, c0, ZT, P2T, Xs));
         }
+        BWLA_PSTAMP(4);
+        cluster_wait_acquire();
+        BWLA_PSTAMP(5);
+    } else if (p.split_y && p.sp_tc == 2) {
+        // ---- few tokens, large P2: the first contraction on the tensor-core path (its factor, a slab of P1^T, is small),
+        //      the second as FMA tiles over fp32 P2 (splitting all of P2 into terms costs more than it saves there)
+        const TcLayout L = tc_layout(n1, n2, p.sp_rp, 1);
+        const int rp = 16 * L.mt, S = p.sp_s;
+        uint8_t* base = reinterpret_cast<uint8_t*>(smem);
+        __nv_bfloat16* Xp = reinterpret_cast<__nv_bfloat16*>(base);                       // x | P1^T terms; later the partial
+        __nv_bfloat16* P1T = reinterpret_cast<__nv_bfloat16*>(base + tc_x_bytes(L));      // sums and this CTA's rows of Y
+        float* part = smem;
+        float* Zt = reinterpret_cast<float*>(base + tc_x_bytes(L) + tc_p1_bytes(L));      // Z'^T fp32 [n2][rp]
+        float* P2s = Zt + (size_t)n2 * rp;
+        slots = P2s + n2 * n2 + 8;
+        for (int i = threadIdx.x; i < (n2 * n2) >> 2; i += blockDim.x) cp_async_16(P2s + 4 * i, p.P2 + 4 * i);
+        {
+            // the slab of P1^T: eight loads in flight per thread (consecutive threads read one row of P1), then the terms
+            constexpr int U = 8;
+            const int total = rp * L.n1p;
+            for (int i0 = threadIdx.x; i0 < total; i0 += U * blockDim.x) {
+                float v[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int i = i0 + u * blockDim.x;
+                    const int a = i / rp, r = i - a * rp;
+                    v[u] = (i < total && r < rows && a < n1) ? __ldg(p.P1 + (size_t)a * n1 + a_lo + r) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int i = i0 + u * blockDim.x;
+                    if (i < total) {
+                        const int a = i / rp, r = i - a * rp;
+                        __nv_bfloat16 h, m, l;
+                        split3(v[u], h, m, l);
+                        __nv_bfloat16* dst = P1T + (size_t)r * L.ps + a;
+                        dst[0] = h; dst[(size_t)rp * L.ps] = m; dst[(size_t)2 * rp * L.ps] = l;
+                    }
+                }
+            }
+        }
+        cluster_arrive_release();              // "this CTA is running": waited for before the first remote store
+        if (!p.late_trigger) griddep_launch_dependents();
+        griddep_wait();                        // x may be the output of the preceding kernel
+        BWLA_PSTAMP(1); BWLA_PBLOCK(2);
+        {
+            const __nv_bfloat16* xt = p.x + t * p.ldx;
+            const int cpr = n2 >> 3;           // 16-byte chunks per row of X
+            if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0) {
+                for (int i = threadIdx.x; i < n1 * cpr; i += blockDim.x) {
+                    const int a = i / cpr, c = i - a * cpr;
+                    *reinterpret_cast<uint4*>(Xp + (size_t)a * L.xs + 8 * c) = __ldg(reinterpret_cast<const uint4*>(xt) + i);
+                }
+            } else {
+                for (int k = threadIdx.x; k < K; k += blockDim.x) Xp[(size_t)(k / n2) * L.xs + k % n2] = xt[k];
+            }
+            for (int i = threadIdx.x; i < (L.n1p - n1) * cpr; i += blockDim.x) {
+                const int a = n1 + i / cpr, c = i % cpr;
+                *reinterpret_cast<uint4*>(Xp + (size_t)a * L.xs + 8 * c) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        __syncthreads();
+        BWLA_PSTAMP(2);
+        tc_stage_a(L, n2, Xp, P1T, nullptr, Zt);
+        cp_async_wait_all();                   // P2 has been arriving meanwhile; it is first read below
+        __syncthreads();                       // x and the P1^T terms are dead: their place takes the partial sums
+        BWLA_PSTAMP(3);
+        slab_partial<8, false>(Zt, rp, P2s, n2, n2, S, part);
+        __syncthreads();
+        // Y goes where the first slice of the partial sums is: a thread reads its own elements of every slice first
+        amax = slab_reduce<false>(part, rp, rows, n2, S, Xs);
         BWLA_PSTAMP(4);
         cluster_wait_acquire();
         BWLA_PSTAMP(5);
@@ -1118,6 +1200,24 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                         // block of this kernel cannot share an SM with the contraction CTAs before it in any case
                         threads = 512;
                         smem = bytes;
+                        return true;
+                    }
+                }
+                if (n2 % 8 == 0 && (cap + 15) / 16 <= 4) {
+                    // P2 too large for its terms: first contraction on the tensor-core path, second as FMA tiles
+                    const TcLayout L = tc_layout(n1, n2, cap, 1);
+                    const int rp16 = 16 * L.mt;
+                    const size_t r0 = tc_x_bytes(L) + tc_p1_bytes(L);
+                    const size_t slice = (size_t)rp16 * n2 * 4;
+                    const size_t rest = (size_t)n2 * rp16 * 4 + ((size_t)n2 * n2 + 8) * 4 + 64;
+                    if (slice <= r0 && r0 + rest <= (size_t)kPrologueSmemFloats * 4) {
+                        const int tiles = (rp16 / 8) * (n2 / 4);
+                        int S = 1;
+                        while (S < 8 && tiles * S < 512 && n2 / (S * 2) >= 4 && (size_t)(S * 2) * slice <= r0) S *= 2;
+                        p.sp_tc = 2; p.sp_rp = cap; p.sp_tr = 8; p.sp_s = S;
+                        p.ps_cap = 0; p.p1_cap = 0; p.ch1 = n2; p.ch2 = cap; p.tr1 = p.tr2 = 8;
+                        threads = 512;
+                        smem = r0 + rest;
                         return true;
                     }
                 }
