@@ -94,7 +94,7 @@ int bwla_rotate_quant_act(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
     if (((uintptr_t)codes & 15) || ((uintptr_t)P1 & 15) || ((uintptr_t)P2 & 15)) return BWLA_ERR_INVALID_ARG;
     int st = check_device();
     if (st != BWLA_OK) return st;
-    return launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, 0, scales, nullptr, nullptr, 0, nullptr,
+    return launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, 0, scales, nullptr, nullptr, 0, nullptr, nullptr, nullptr,
                            (cudaStream_t)stream);
 }
 
@@ -140,7 +140,7 @@ int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, cons
     const int path = resolve_path(M, K, N, r, bits);
 
     st = launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum,
-                         V_bf16, r, Thl, s);
+                         V_bf16, r, Thl, r > 0 ? (float*)(base + ws.lr_part) : nullptr, (uint32_t*)(base + ws.status), s);
     if (st != BWLA_OK) return st;
     GemmArgs g{};
     g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
@@ -174,7 +174,8 @@ int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int
     st = launch_prepare_codes(codes, M, K, inter, qsum, s);
     if (st != BWLA_OK) return st;
     if (r > 0) {
-        st = launch_prologue(x_bf16, M, K, ldx, nullptr, 0, nullptr, 0, bits, nullptr, 0, nullptr, nullptr, V_bf16, r, Thl, s);
+        st = launch_prologue(x_bf16, M, K, ldx, nullptr, 0, nullptr, 0, bits, nullptr, 0, nullptr, nullptr, V_bf16, r, Thl,
+                             (float*)(base + ws.lr_part), (uint32_t*)(base + ws.status), s);
         if (st != BWLA_OK) return st;
     }
     GemmArgs g{};

@@ -67,10 +67,15 @@ constexpr int kLowrankPad = 64;          // T is kept as bf16 [3][M][64] (T = hi
 // of the token; unused parts are zero): the consumer adds them, the producers need no exchange.
 constexpr int kQsumParts = 8;
 
+// With few tokens and a large K the rows of V are read by several blocks that each take a part of K; their partial sums
+// of T meet in the workspace and the last block to arrive adds them in a fixed order (counters: status words 4..11).
+constexpr int kLrKSplitMax = 8;
+constexpr int kLrCounterWord = 4;
+
 __host__ __device__ inline int lowrank_cols(int r) { return r > kLowrankPad ? (r + 1) / 2 * 2 : kLowrankPad; }
 
 struct Workspace {
-    size_t status, scales, qsum, T, codes, total;
+    size_t status, scales, qsum, T, lr_part, codes, total;
 };
 
 inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bits) {
@@ -81,6 +86,7 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     w.qsum = off;   off += align_up((size_t)M * 4 * kQsumParts, 256);
     const size_t lr_cols = (size_t)lowrank_cols(r);
     w.T = off;      off += align_up((size_t)M * lr_cols * 6, 256);     // bf16 [3][M][cols]
+    w.lr_part = off; off += r > 0 ? align_up((size_t)kLrKSplitMax * 16 * lr_cols * 4, 256) : 0;   // fp32 [KS][16][cols]
     w.codes = off;  off += align_up((size_t)M * (size_t)K, 256);
     (void)N; (void)bits;
     w.total = off;
@@ -97,9 +103,10 @@ int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ld
 // Thl == NULL).  codes_layout: 0 = natural k order, 1 = interleaved order used by the tensor-core contraction (inside
 // each group of 32, position 4*j + i holds k = j + 8*i).  qsum (int32 [M][kQsumParts], partial sums) may be NULL.
 // Thl: bf16 [3][M][cols], cols = lowrank_cols(r): T as the sum of three bf16 terms (exact for an fp32 T).
+// lr_part / status (both may be NULL): scratch for the partial sums of T and the workspace status words (see kLrKSplitMax).
 int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2, int n2,
                     int bits, int8_t* codes, int codes_layout, float* scales, int32_t* qsum, const void* V, int r,
-                    void* Thl, cudaStream_t stream);
+                    void* Thl, float* lr_part, uint32_t* status, cudaStream_t stream);
 
 // qsum[t][0] = sum_k codes[t][k] (the other parts zero); optionally rewrites natural-order codes into the interleaved order.
 int launch_prepare_codes(const int8_t* codes, int64_t M, int64_t K, int8_t* codes_interleaved, int32_t* qsum,

@@ -78,6 +78,9 @@ struct PrologueParams {
     const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
     int lr_wide;        // low-rank blocks: 0: 2 rows of V x 16 tokens (FMA), 1: 8 x 8 (FMA, many tokens), 2: 8 columns x 16 tokens on the
                         // warp-level tensor-core path (few tokens), 3: all 64 columns x 16 tokens on that path (many tokens)
+    int lr_ks;          // lr_wide == 2: blocks that share a tile of T and split K (1: no split)
+    float* lr_part;     // [tiles][lr_ks][16 * 8] partial sums of those blocks
+    uint32_t* lr_count; // one arrival counter per tile, zero between calls
     int lr_stage;       // 1: a low-rank block copies its rows of V into shared memory before it waits for x
     int late_trigger;   // 1: the next kernel of the stream is let in only when this one is nearly done (see launch_prologue)
 };
@@ -983,8 +986,10 @@ __device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uin
 
 __device__ void lowrank_mma_role(const PrologueParams& p, int b, float* smem) {
     const int jtiles = p.lr_cols / 8;
+    const int KS = p.lr_ks;
     const int j0 = (b % jtiles) * 8;
-    const int64_t t0 = (int64_t)(b / jtiles) * 16;
+    const int ks = (b / jtiles) % KS;
+    const int64_t t0 = (int64_t)(b / (jtiles * KS)) * 16;
     if (t0 >= p.M) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int g = lane >> 2, tg = lane & 3;
@@ -1000,8 +1005,9 @@ __device__ void lowrank_mma_role(const PrologueParams& p, int b, float* smem) {
         const uint4* xhi = reinterpret_cast<const uint4*>(p.x + (t0 + (row_hi ? g + 8 : 0)) * p.ldx) + tg;
         const uint4* vj = reinterpret_cast<const uint4*>(p.V + (int64_t)(j0 + (col ? g : 0)) * K) + tg;
         const int chunks = K >> 5;
+        const int c_lo = (int)((int64_t)chunks * ks / KS), c_hi = (int)((int64_t)chunks * (ks + 1) / KS);
 #pragma unroll 4
-        for (int c = warp; c < chunks; c += nwarps) {
+        for (int c = c_lo + warp; c < c_hi; c += nwarps) {
             const uint4 a = row_lo ? __ldg(xlo + 4 * c) : zero;
             const uint4 h = row_hi ? __ldg(xhi + 4 * c) : zero;
             const uint4 v = col ? __ldg(vj + 4 * c) : zero;
@@ -1016,6 +1022,41 @@ __device__ void lowrank_mma_role(const PrologueParams& p, int b, float* smem) {
     red[warp * 128 + (g + 8) * 8 + 2 * tg] = acc[2];
     red[warp * 128 + (g + 8) * 8 + 2 * tg + 1] = acc[3];
     __syncthreads();
+    if (KS > 1) {
+        // Several blocks share this tile of T and split K.  Each leaves its partial tile in the workspace; the last one
+        // to arrive adds them in the order of the K parts (so the result does not depend on who came last).
+        const int tile = (int)(b / (jtiles * KS)) * jtiles + (b % jtiles);
+        float* mine = p.lr_part + ((size_t)tile * KS + ks) * 128;
+        for (int o = threadIdx.x; o < 128; o += blockDim.x) {
+            float s = 0.f;
+            for (int w = 0; w < nwarps; ++w) s += red[w * 128 + o];
+            mine[o] = s;
+        }
+        __threadfence();
+        __syncthreads();
+        __shared__ uint32_t arrived;
+        if (threadIdx.x == 0) arrived = atomicAdd(p.lr_count + tile, 1u);
+        __syncthreads();
+        if (arrived != (uint32_t)(KS - 1)) return;
+        __threadfence();
+        for (int o = threadIdx.x; o < 128; o += blockDim.x) {
+            const int i = o >> 3, j = o & 7;
+            float s = 0.f;
+            for (int k = 0; k < KS; ++k) s += __ldcg(p.lr_part + ((size_t)tile * KS + k) * 128 + o);
+            if (t0 + i < p.M) {
+                const __nv_bfloat16 hi = __float2bfloat16_rn(s);
+                const float r1 = s - __bfloat162float(hi);
+                const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                const int64_t at = (t0 + i) * p.lr_cols + j0 + j;
+                p.Thl[at] = hi;
+                p.Thl[p.M * p.lr_cols + at] = mid;
+                p.Thl[2 * p.M * p.lr_cols + at] = lo;
+            }
+        }
+        if (threadIdx.x == 0) p.lr_count[tile] = 0;          // ready for the next call
+        return;
+    }
     for (int o = threadIdx.x; o < 128; o += blockDim.x) {
         const int i = o >> 3, j = o & 7;
         if (t0 + i < p.M) {
@@ -1145,7 +1186,7 @@ static int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } re
 
 int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2, int n2,
                     int bits, int8_t* codes, int codes_layout, float* scales, int32_t* qsum, const void* V, int r,
-                    void* Thl, cudaStream_t stream) {
+                    void* Thl, float* lr_part, uint32_t* status, cudaStream_t stream) {
     if (M == 0) return BWLA_OK;
     const bool rotate = codes != nullptr;
     PrologueParams p{};
@@ -1302,6 +1343,13 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
         lr_blocks = p.lr_wide == 1 ? (p.lr_cols / 8) * (int)((M + 7) / 8)
                   : p.lr_wide == 2 ? (p.lr_cols / 8) * (int)((M + 15) / 16)
                   : p.lr_wide == 3 ? (int)((M + 15) / 16) : (p.lr_cols / 2) * (int)((M + 15) / 16);
+        // One tile of 16 tokens and a large K: eight blocks would stream all of V (cold: from HBM) through eight SMs and
+        // become the longest part of the launch; more blocks take a part of K each.
+        p.lr_ks = 1; p.lr_part = lr_part; p.lr_count = status ? status + kLrCounterWord : nullptr;
+        if (p.lr_wide == 2 && M <= 16 && lr_part && status && p.lr_cols / 8 <= 8) {
+            const int ksplit = (int)std::min<int64_t>(kLrKSplitMax, (K >> 5) / 100);
+            if (ksplit > 1) { p.lr_ks = ksplit; lr_blocks *= ksplit; }
+        }
         // shared memory of a low-rank block: per-warp partial sums, and its rows of V when those are staged (few tokens)
         const size_t red_bytes = (size_t)kLrMaxWarps * 4 * (p.lr_wide == 3 ? 1024 : p.lr_wide == 2 ? 128 : 64);
         const size_t stage_bytes = (size_t)2 * (size_t)K * 2;
