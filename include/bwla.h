@@ -90,11 +90,13 @@ size_t bwla_workspace_bytes(int64_t M, int64_t K, int64_t N, int r, int bits);
  *   workspace device, 256-byte aligned, >= bwla_workspace_bytes(M,K,N,r,bits); contents are scratch, except that
  *     its first 256 bytes must be zero before the first call that uses it.  The first word is a status word that
  *     bounded device-side waits set and that stays set (later calls on this workspace then skip their work) until
- *     bwla_check_status reads and clears it.
+ *     bwla_check_status reads and clears it; a few of the following words are arrival counters that every call
+ *     leaves at zero.
  *   Two calls that share a workspace must be ordered on one stream.
- *   The kernels are launched with programmatic stream serialisation: the part of a call that does not depend on
- *   earlier work (streaming the sign words into shared memory) may overlap the tail of the preceding kernel of
- *   `stream`; every global store waits for that kernel to finish.
+ *   The kernels are launched with programmatic stream serialisation: the part of a call that depends only on the
+ *   layer's constants (streaming the sign words, fetching P1, P2 and V) may overlap the tail of the preceding kernel
+ *   of `stream`; x is read and every global store is made only after that kernel has finished, so a call may consume
+ *   what the preceding call of the stream produced.
  */
 int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx,
                      const float* P1, int n1, const float* P2, int n2, int bits,
