@@ -210,6 +210,27 @@ def test_qwen32b_shapes(bwla, idx, M):
     _run_layer_case(bwla, 2, gen.CONFIG_SHAPES[2][idx], M, 6, direct_words=True)
 
 
+def test_blocks_that_split_k_for_the_low_rank_term_give_the_same_bits_every_time(bwla):
+    """down_proj at 16 tokens: several blocks share a tile of T = V x, each takes a part of K, and whichever arrives
+    last adds the parts in the order of K.  The result must not depend on the order of arrival, and the arrival
+    counters in the workspace must be back at zero for the next call."""
+    shape = gen.CONFIG_SHAPES[2][6]
+    _run_layer_case(bwla, 2, shape, 16, 6, direct_words=True)
+    lay = gen.make_layer(2, shape, 6, direct_words=True)
+    dl = H.DeviceLayer(lay, bwla)
+    xd = H.bf16_to_dev(gen.make_activations(2, shape, 16))
+    ws = bwla.new_workspace(16, shape.K, shape.N, shape.r, 6)
+    first = None
+    for _ in range(8):
+        out = bwla.bwla_w1ax_linear(xd, dl.P1, dl.P2, 6, dl.packed, dl.alpha, dl.U, dl.V, dl.mu, workspace=ws)
+        bits = H.bf16_to_host(out)
+        if first is None:
+            first = bits
+        assert np.array_equal(bits, first)
+    assert bwla.bwla_check_status(ws) == 0
+    assert int(ws[:256].view(torch.int32).abs().sum().item()) == 0      # status words, counters included, are zero again
+
+
 @pytest.mark.parametrize("bits", [4, 6, 8])
 def test_bit_width_sweep_down_proj(bwla, bits):
     _run_layer_case(bwla, 3, gen.CONFIG_SHAPES[3][0], 1, bits, direct_words=True)
