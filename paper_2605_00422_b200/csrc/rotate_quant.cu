@@ -1221,8 +1221,10 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                 if ((K & 7) != 0) return false;
                 p.split_y = 1;
                 p.sp_tc = 0;
-                if (n2 % 16 == 0 && (cap + 15) / 16 <= 4) {
-                    // both contractions on the warp-level tensor-core path when the split operands fit
+                if (n2 % 16 == 0 && (cap + 15) / 16 <= 4 && n2 <= 96) {
+                    // both contractions on the warp-level tensor-core path when the split operands fit and P2 is small
+                    // (splitting all of a larger P2 into terms costs more than the FMA version of the second contraction:
+                    // o_proj, n2 = 128, is 1.6 us faster the mixed way)
                     // P2 whole.  (Staging it in parts of its columns works -- the kernel takes any number of parts -- but
                     // was measured no faster than the FMA version for K = 25600: mma.sync runs at ~6 cycles per
                     // m16n8k16 per SM on this part, and the restaging is exposed.)
