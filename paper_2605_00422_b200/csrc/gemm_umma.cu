@@ -420,43 +420,37 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (e == 64 && u == unit_begin) { BWLA_STAMP(3); BWLA_CTA_STAMP(1); }
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
-            // the sign words of this warp's k-blocks of the unit, loaded together
-            uint4 w4[8 / EW];
-#pragma unroll
-            for (int i = 0; i < 8 / EW; ++i) {
-                const int s = EW * i + part;
-                if (s < ns) w4[i] = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
-            }
             if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 2);
+            // a rolled loop over this warp's k-blocks of the unit; each block's sign words are loaded just before they are
+            // expanded
+#pragma unroll 1
+            for (int s = part; s < ns && ok; s += EW) {
+                const uint4 w4 = *reinterpret_cast<const uint4*>(wrow + ((s ^ (row & 7)) << 4));
+                uint32_t v[32];
+                const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-            for (int i = 0; i < 8 / EW; ++i) {
-                if (ok && EW * i + part < ns) {
-                    uint32_t v[32];
-                    const uint32_t w[4] = {w4[i].x, w4[i].y, w4[i].z, w4[i].w};
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
-                    if (lane == 0) BWLA_RING(warp - 6, nown, 0);
-                    if (!warp_wait(&a_empty[as], aph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x41); ok = false; }
-                    if (lane == 0) BWLA_RING(warp - 6, nown, 1);
-                    if (ok) {
-                        tc_fence_after();
-                        tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
-                        tc_wait_st();
-                        if (lane == 0) BWLA_RING(warp - 6, nown, 2);
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&a_full[as]);
-                        if (lane == 0) BWLA_RING(warp - 6, nown, 3);
-                        ++nown;
-                        as += EW;
-                        if (as >= AS) { as = part; aph ^= 1u; }
-                    }
+                    for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
+                if (lane == 0) BWLA_RING(warp - 6, nown, 0);
+                if (!warp_wait(&a_empty[as], aph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x41); ok = false; }
+                if (lane == 0) BWLA_RING(warp - 6, nown, 1);
+                if (ok) {
+                    tc_fence_after();
+                    tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
+                    tc_wait_st();
+                    if (lane == 0) BWLA_RING(warp - 6, nown, 2);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&a_full[as]);
+                    if (lane == 0) BWLA_RING(warp - 6, nown, 3);
+                    ++nown;
+                    as += EW;
+                    if (as >= AS) { as = part; aph ^= 1u; }
                 }
             }
-            // The stage is released only here, after every word loaded from it has gone through the expansion: an
-            // arrive placed right behind the loads let the copy of a later unit overwrite words not yet read.
+            // The stage is released only here, after every word of it that this warp needs has gone through the expansion:
+            // an arrive placed earlier let the copy of a later unit overwrite words not yet read.
             __syncwarp();
             if (lane == 0) mbar_arrive(&w_empty[ws]);
             if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 3);
