@@ -70,7 +70,7 @@ def summand_magnitude(ref: dict, alpha: np.ndarray) -> np.ndarray:
 
 
 def check_codes(gpu_codes: np.ndarray, gpu_scales: np.ndarray, Y: np.ndarray, bits: int) -> dict:
-    """The benchmark spec rule for the integer codes; returns counts for the report."""
+    """The comparison rule for the integer codes (see the module docstring); returns counts for the report."""
     ref = oracle.quantize(Y, bits, "f64")
     diff = gpu_codes.astype(np.int32) - ref["codes"].astype(np.int32)
     bad = diff != 0
