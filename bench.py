@@ -86,6 +86,23 @@ def measured_peaks():
 
 
 # ----------------------------------------------------------------------------------------------
+# replicas: N processes, one GPU each, no exchange on the data path
+# ----------------------------------------------------------------------------------------------
+def max_over_ranks(ms: float, world: int, device, dist, torch) -> float:
+    """The slowest rank's time: what a job of `world` replicas that start together takes."""
+    if world <= 1:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_rate(world: int, units_per_rank_per_step: float, steps: int, ms: float) -> float:
+    """Whole-job units per second: every rank processes its own copy of the workload (weak scaling)."""
+    return world * units_per_rank_per_step * steps / (ms * 1e-3)
+
+
+# ----------------------------------------------------------------------------------------------
 # clocks
 # ----------------------------------------------------------------------------------------------
 class ClockSampler:
@@ -292,12 +309,7 @@ def run_ours(args):
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), world, device, dist, torch)
 
     def kernel_profile(xs, outs, ws, passes=1, layers=None):
         bwla.bwla_profile_enable(True)
@@ -319,7 +331,7 @@ def run_ours(args):
     clocks = sampler.stop()
     status = bwla.bwla_check_status(ws)
     step_bytes = args.layers * sum(call_bytes(sh, M) for sh in shapes)
-    value = world * step_bytes * args.steps / (ms * 1e-3) / 1e9
+    value = replica_rate(world, step_bytes, args.steps, ms) / 1e9
 
     # end to end: activations arrive from pinned host memory and the last layer's outputs go back, every step
     h_xs = {K: xs[K].cpu().pin_memory() for K in Ks}
@@ -335,7 +347,7 @@ def run_ours(args):
     e2e_ms = timed(e2e_step, args.steps, 3)
     h2d = sum(h_xs[K].numel() * 2 for K in Ks)
     d2h = sum(h_outs[N].numel() * 2 for N in Ns)
-    e2e_value = world * step_bytes * args.steps / (e2e_ms * 1e-3) / 1e9
+    e2e_value = replica_rate(world, step_bytes, args.steps, e2e_ms) / 1e9
 
     prof = kernel_profile(xs, outs, ws)
     k_ms, k_n = prof.get("contraction", (0.0, 0))
