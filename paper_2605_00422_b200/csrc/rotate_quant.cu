@@ -59,7 +59,9 @@ struct PrologueParams {
     const float* P1; int n1; const float* P2; int n2; int bits;
     int8_t* codes; int codes_layout; float* scales; int32_t* qsum;
     int C;              // CTAs per token (cluster size)
-    int rot_blocks;     // M * C
+    int rot_blocks;     // clusters * C
+    int tok_stride;     // number of clusters: a cluster takes tokens t, t + tok_stride, ... (== M unless the clusters stay and loop)
+    int rot_first;      // first rotation block: 0, or (clusters that stay) behind the low-rank blocks, which then start first
     int row_gran;       // slab boundaries are multiples of this many rows of X
     int slab_cap;       // floats reserved for one slab
     int ps_cap;         // floats reserved for a staged chunk of P2 / P1
@@ -512,10 +514,92 @@ __device__ __forceinline__ void load_p1_columns(const float* __restrict__ P1, in
     }
 }
 
+// Second half of a token: absmax over the block and the cluster, quantisation of this CTA's rows of Y (at Xs), code
+// sums, scale.  One cluster barrier per token when C > 1 (every CTA of the cluster calls this for the same tokens).
+__device__ __forceinline__ void finish_token(const PrologueParams& p, int64_t t, int C, int rank, const float* Xs, float* slots,
+                                             float amax, int rows, int a_lo, float* red_max, int* red_sum_p, bool last) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int qmax = (1 << (p.bits - 1)) - 1;
+    const int n2 = p.n2, K = p.K;
+    int& red_sum = *red_sum_p;
+    BWLA_PSTAMP(6);
+    // ---- absmax over the block, then over the cluster
+    amax = warp_max(amax);
+    if (lane == 0) red_max[warp] = amax;
+    __syncthreads();
+    amax = (lane < nwarps) ? red_max[lane] : 0.f;
+    amax = warp_max(amax);
+    if (C > 1) {
+        if (threadIdx.x < C) st_cluster_u32(map_shared_rank(smem_u32(slots + rank), threadIdx.x), __float_as_uint(amax));
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        float m = (lane < C) ? slots[lane] : 0.f;
+        amax = warp_max(m);
+    }
+
+    float inv, scale;
+    if (amax == 0.f) { inv = 0.f; scale = 1.f; }
+    else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
+
+    BWLA_PSTAMP(7);
+    if (p.late_trigger && last) griddep_launch_dependents();
+    // nothing is stored to global memory before the preceding kernel of the stream has completed
+    griddep_wait();
+    BWLA_PSTAMP(8);
+
+    int local_sum = 0;
+    int8_t* ct = p.codes + t * (int64_t)K + (int64_t)a_lo * n2;
+    const int words = (rows * n2) >> 5;
+    for (int g = threadIdx.x; g < words; g += blockDim.x) {
+        const float* y = Xs + 32 * g;
+        int q[32];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 v = *reinterpret_cast<const float4*>(y + 4 * i);
+            const float f[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int c = __float2int_rn(__fmul_rn(f[j], inv));
+                c = max(-qmax, min(qmax, c));
+                q[4 * i + j] = c;
+                local_sum += c;
+            }
+        }
+        uint32_t w[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint32_t v = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int k = p.codes_layout ? (j + 8 * i) : (4 * j + i);
+                v |= (uint32_t)(q[k] & 0xFF) << (8 * i);
+            }
+            w[j] = v;
+        }
+        uint4* dst = reinterpret_cast<uint4*>(ct + 32 * g);
+        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
+    local_sum = warp_sum(local_sum);
+    if (lane == 0 && local_sum != 0) atomicAdd(&red_sum, local_sum);
+    __syncthreads();
+    BWLA_PSTAMP(9);
+    // every CTA leaves its own part of the token's code sum; the consumer adds the parts, so no exchange is needed here
+    if (threadIdx.x == 0) {
+        if (p.qsum) {
+            p.qsum[t * kQsumParts + rank] = red_sum;
+            if (rank == 0)
+                for (int c = C; c < kQsumParts; ++c) p.qsum[t * kQsumParts + c] = 0;
+        }
+        if (rank == 0) p.scales[t] = scale;
+    }
+    BWLA_PSTAMP(10);
+}
+
 __device__ void rotate_role(const PrologueParams& p, float* smem) {
     const int C = p.C;
     const int rank = C > 1 ? (int)cluster_ctarank() : 0;
-    const int64_t t = blockIdx.x / C;
+    const int64_t t = ((int)blockIdx.x - p.rot_first) / C;   // the cluster's first (with few tokens: only) token
     const int n1 = p.n1, n2 = p.n2, K = p.K;
     const int a_lo = slab_begin(rank, C, n1, p.row_gran), a_hi = slab_begin(rank + 1, C, n1, p.row_gran);
     const int rows = a_hi - a_lo;
@@ -626,8 +710,15 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         if (!p.late_trigger) griddep_launch_dependents();
         griddep_wait();                        // x may be the output of the preceding kernel
         BWLA_PSTAMP(1); BWLA_PBLOCK(2);
-        {
-            const __nv_bfloat16* xt = p.x + t * p.ldx;
+        // The cluster takes tokens t, t + tok_stride, ...: with few tokens exactly one; with many tokens of a large K the
+        // clusters stay, and the constants above are fetched and split once per cluster instead of once per token.
+        for (int64_t tt = t; tt < p.M; tt += p.tok_stride) {
+            if (tt != t) {
+                // every thread of the block is past its reads of the previous token's Y (the barriers of finish_token)
+                if (threadIdx.x == 0) red_sum = 0;
+                amax = 0.f;
+            }
+            const __nv_bfloat16* xt = p.x + tt * p.ldx;
             const int cpr = n2 >> 3;           // 16-byte chunks per row of X
             if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0) {
                 for (int i = threadIdx.x; i < n1 * cpr; i += blockDim.x) {
@@ -641,20 +732,22 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
                 const int a = n1 + i / cpr, c = i % cpr;
                 *reinterpret_cast<uint4*>(Xp + (size_t)a * L.xs + 8 * c) = make_uint4(0u, 0u, 0u, 0u);
             }
+            __syncthreads();
+            BWLA_PSTAMP(2);
+            tc_stage_a(L, n2, Xp, P1T, nullptr, Zt);
+            cp_async_wait_all();               // P2 has been arriving meanwhile; it is first read below
+            __syncthreads();                   // x is dead: its place takes the partial sums (and, with one token per
+            BWLA_PSTAMP(3);                    // cluster, that of the P1^T terms too)
+            slab_partial<8, false>(Zt, rp, P2s, n2, n2, S, part);
+            __syncthreads();
+            // Y goes where the first slice of the partial sums is: a thread reads its own elements of every slice first
+            amax = slab_reduce<false>(part, rp, rows, n2, S, Xs);
+            BWLA_PSTAMP(4);
+            if (tt == t) cluster_wait_acquire();
+            BWLA_PSTAMP(5);
+            finish_token(p, tt, C, rank, Xs, slots, amax, rows, a_lo, red_max, &red_sum, tt + p.tok_stride >= p.M);
         }
-        __syncthreads();
-        BWLA_PSTAMP(2);
-        tc_stage_a(L, n2, Xp, P1T, nullptr, Zt);
-        cp_async_wait_all();                   // P2 has been arriving meanwhile; it is first read below
-        __syncthreads();                       // x and the P1^T terms are dead: their place takes the partial sums
-        BWLA_PSTAMP(3);
-        slab_partial<8, false>(Zt, rp, P2s, n2, n2, S, part);
-        __syncthreads();
-        // Y goes where the first slice of the partial sums is: a thread reads its own elements of every slice first
-        amax = slab_reduce<false>(part, rp, rows, n2, S, Xs);
-        BWLA_PSTAMP(4);
-        cluster_wait_acquire();
-        BWLA_PSTAMP(5);
+        return;
     } else if (p.split_y) {
         // ---- few tokens: this CTA's rows of Y from all of x; nothing but absmax and code sums is exchanged
         const int rp = p.sp_rp, S = p.sp_s;
@@ -781,78 +874,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             amax = fmaxf(amax, fabsf(s));
         }
     }
-    BWLA_PSTAMP(6);
-    // ---- absmax over the block, then over the cluster
-    amax = warp_max(amax);
-    if (lane == 0) red_max[warp] = amax;
-    __syncthreads();
-    amax = (lane < nwarps) ? red_max[lane] : 0.f;
-    amax = warp_max(amax);
-    if (C > 1) {
-        if (threadIdx.x < C) st_cluster_u32(map_shared_rank(smem_u32(slots + rank), threadIdx.x), __float_as_uint(amax));
-        cluster_arrive_release();
-        cluster_wait_acquire();
-        float m = (lane < C) ? slots[lane] : 0.f;
-        amax = warp_max(m);
-    }
-
-    float inv, scale;
-    if (amax == 0.f) { inv = 0.f; scale = 1.f; }
-    else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
-
-    BWLA_PSTAMP(7);
-    if (p.late_trigger) griddep_launch_dependents();
-    // nothing is stored to global memory before the preceding kernel of the stream has completed
-    griddep_wait();
-    BWLA_PSTAMP(8);
-
-    int local_sum = 0;
-    int8_t* ct = p.codes + t * (int64_t)K + (int64_t)a_lo * n2;
-    const int words = (rows * n2) >> 5;
-    for (int g = threadIdx.x; g < words; g += blockDim.x) {
-        const float* y = Xs + 32 * g;
-        int q[32];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float4 v = *reinterpret_cast<const float4*>(y + 4 * i);
-            const float f[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                int c = __float2int_rn(__fmul_rn(f[j], inv));
-                c = max(-qmax, min(qmax, c));
-                q[4 * i + j] = c;
-                local_sum += c;
-            }
-        }
-        uint32_t w[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            uint32_t v = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int k = p.codes_layout ? (j + 8 * i) : (4 * j + i);
-                v |= (uint32_t)(q[k] & 0xFF) << (8 * i);
-            }
-            w[j] = v;
-        }
-        uint4* dst = reinterpret_cast<uint4*>(ct + 32 * g);
-        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-    }
-    local_sum = warp_sum(local_sum);
-    if (lane == 0 && local_sum != 0) atomicAdd(&red_sum, local_sum);
-    __syncthreads();
-    BWLA_PSTAMP(9);
-    // every CTA leaves its own part of the token's code sum; the consumer adds the parts, so no exchange is needed here
-    if (threadIdx.x == 0) {
-        if (p.qsum) {
-            p.qsum[t * kQsumParts + rank] = red_sum;
-            if (rank == 0)
-                for (int c = C; c < kQsumParts; ++c) p.qsum[t * kQsumParts + c] = 0;
-        }
-        if (rank == 0) p.scales[t] = scale;
-    }
-    BWLA_PSTAMP(10);
+    finish_token(p, t, C, rank, Xs, slots, amax, rows, a_lo, red_max, &red_sum, true);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1146,11 +1168,13 @@ __device__ void lowrank_mma_wide_role(const PrologueParams& p, int b, float* sme
 __global__ void prologue_kernel(PrologueParams p) {
     extern __shared__ __align__(16) float smem[];
     BWLA_PBLOCK(0);
-    if ((int)blockIdx.x < p.rot_blocks) rotate_role(p, smem);
-    else if (p.lr_wide == 1) lowrank_role<8, 8>(p, (int)blockIdx.x - p.rot_blocks, smem);
-    else if (p.lr_wide == 2) lowrank_mma_role(p, (int)blockIdx.x - p.rot_blocks, smem);
-    else if (p.lr_wide == 3) lowrank_mma_wide_role(p, (int)blockIdx.x - p.rot_blocks, smem);
-    else lowrank_role<2, 16>(p, (int)blockIdx.x - p.rot_blocks, smem);
+    const int b = (int)blockIdx.x;
+    const int lr = p.rot_first ? b : b - p.rot_blocks;        // index among the low-rank blocks (when not a rotation block)
+    if (b >= p.rot_first && b < p.rot_first + p.rot_blocks) rotate_role(p, smem);
+    else if (p.lr_wide == 1) lowrank_role<8, 8>(p, lr, smem);
+    else if (p.lr_wide == 2) lowrank_mma_role(p, lr, smem);
+    else if (p.lr_wide == 3) lowrank_mma_wide_role(p, lr, smem);
+    else lowrank_role<2, 16>(p, lr, smem);
     BWLA_PBLOCK(1);
 }
 
@@ -1201,6 +1225,8 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     size_t smem = 0;
     if (rotate) {
         const int gran = 32 / gcd_int(n2, 32);
+        // clusters that stay and take several tokens must keep the terms of P1^T: the partial sums then take x's place only
+        bool keep_p1t = false;
         // lays the block out for clusters of `c` CTAs per token; false if it does not fit
         auto plan = [&](int c) -> bool {
             int cap = 0;
@@ -1251,12 +1277,13 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
                     const TcLayout L = tc_layout(n1, n2, cap, 1);
                     const int rp16 = 16 * L.mt;
                     const size_t r0 = tc_x_bytes(L) + tc_p1_bytes(L);
+                    const size_t part_room = keep_p1t ? tc_x_bytes(L) : r0;
                     const size_t slice = (size_t)rp16 * n2 * 4;
                     const size_t rest = (size_t)n2 * rp16 * 4 + ((size_t)n2 * n2 + 8) * 4 + 64;
-                    if (slice <= r0 && r0 + rest <= (size_t)kPrologueSmemFloats * 4) {
+                    if (slice <= part_room && r0 + rest <= (size_t)kPrologueSmemFloats * 4) {
                         const int tiles = (rp16 / 8) * (n2 / 4);
                         int S = 1;
-                        while (S < 8 && tiles * S < 512 && n2 / (S * 2) >= 4 && (size_t)(S * 2) * slice <= r0) S *= 2;
+                        while (S < 8 && tiles * S < 512 && n2 / (S * 2) >= 4 && (size_t)(S * 2) * slice <= part_room) S *= 2;
                         p.sp_tc = 2; p.sp_rp = cap; p.sp_tr = 8; p.sp_s = S;
                         p.ps_cap = 0; p.p1_cap = 0; p.ch1 = n2; p.ch2 = cap; p.tr1 = p.tr2 = 8;
                         threads = 512;
@@ -1321,18 +1348,37 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
             smem = ((size_t)p.slab_cap + (size_t)K + (size_t)p.ps_cap + (size_t)p.p1_cap + 16) * 4;
             return true;
         };
+        int64_t clusters = M;                  // clusters of C CTAs; each takes tokens t, t + clusters, ...
         if ((n2 & 3) == 0) {
-            // spread one token over several SMs while there are few tokens and the token is worth splitting, as long as
-            // every token's cluster is resident at once (a second wave of clusters would double the latency)
             const double flops = 2.0 * (double)K * (n1 + n2);
-            C = 8;
-            while (C > 1 && (M * C > 148 || flops / C < 1.5e5 || n1 / C < gran)) --C;
-            for (; C > 1; --C) {
-                if (!plan(C)) continue;
-                if (clusters_resident(C, threads, smem) >= M) break;
+            int cmax = 8;
+            while (cmax > 1 && (flops / cmax < 1.5e5 || n1 / cmax < gran)) --cmax;
+            // Few tokens: spread one token over several SMs, as long as every token's cluster is resident at once (a
+            // second wave of clusters would double the latency).
+            bool chosen = false;
+            for (int c = cmax; c > 1 && !chosen; --c) {
+                if (M * c > 148 || !plan(c)) continue;
+                if (clusters_resident(c, threads, smem) >= M) { C = c; chosen = true; }
             }
+            // Many tokens of a large K: one CTA per token would stage P1 and P2 chunk by chunk for every token.  Clusters
+            // that stay, keep the constants and take tokens in turn do that once per cluster; the cluster size that puts
+            // the most CTAs on the device wins.  (Only the mode whose first contraction runs on the tensor-core path is
+            // fast enough per token to beat one CTA per token.)
+            if (!chosen && plan(1) && !p.prefetch) {
+                keep_p1t = true;
+                int best_ctas = 0;
+                for (int c = cmax; c > 1; --c) {
+                    if (!plan(c) || p.sp_tc != 2) continue;
+                    const int64_t n = std::min<int64_t>(M, clusters_resident(c, threads, smem));
+                    if (n * c > best_ctas) { best_ctas = (int)(n * c); C = c; clusters = n; chosen = true; }
+                }
+                if (!chosen) keep_p1t = false;
+            }
+            if (!chosen) C = 1;
         }
         if (!plan(C)) return BWLA_ERR_INVALID_ARG;
+        p.rot_blocks = (int)(clusters * C);
+        p.tok_stride = (int)clusters;
     } else {
         p.C = 1; p.rot_blocks = 0;
     }
@@ -1362,7 +1408,10 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     // in early, that kernel would crowd onto the SMs this one leaves free and stay there; so it is let in late, when
     // the blocks of this one are about to leave.
     p.late_trigger = smem > 110 * 1024 ? 1 : 0;
-    int grid = p.rot_blocks + lr_blocks;
+    // Clusters that stay hold their SMs until the last token: the low-rank blocks go first in block order then, or they
+    // would only start when the rotation is over.
+    p.rot_first = (rotate && p.tok_stride < M && lr_blocks > 0) ? (lr_blocks + C - 1) / C * C : 0;
+    int grid = p.rot_first ? p.rot_first + p.rot_blocks : p.rot_blocks + lr_blocks;
     grid = (grid + C - 1) / C * C;
     if (grid == 0) return BWLA_OK;
 
