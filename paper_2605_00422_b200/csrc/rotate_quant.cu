@@ -1387,7 +1387,8 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
         // few tokens: the tensor-core version (needs 16-byte rows); many tokens: FMA tiles that re-read little
         const bool rows16 = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(V)) & 15) == 0 && ldx % 8 == 0 &&
                             K % 32 == 0 && p.lr_cols % 8 == 0;
-        p.lr_wide = rows16 ? ((M > 32 && p.lr_cols == 64) ? 3 : 2) : ((M >= 64 && p.lr_cols % 8 == 0) ? 1 : 0);
+        // (the wide tiles read x once but need enough token tiles to fill the device: 16 tokens x 64 columns per block)
+        p.lr_wide = rows16 ? ((M >= 1024 && p.lr_cols == 64) ? 3 : 2) : ((M >= 64 && p.lr_cols % 8 == 0) ? 1 : 0);
         lr_blocks = p.lr_wide == 1 ? (p.lr_cols / 8) * (int)((M + 7) / 8)
                   : p.lr_wide == 2 ? (p.lr_cols / 8) * (int)((M + 15) / 16)
                   : p.lr_wide == 3 ? (int)((M + 15) / 16) : (p.lr_cols / 2) * (int)((M + 15) / 16);
