@@ -753,7 +753,9 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
                                    : launch_umma_t<16, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
         case 32: return wide_split ? launch_umma_t<32, 3, 2, 512, 2, 4>(wm, bm, tm, p, grid, stream)
                                    : launch_umma_t<32, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
-        case 64: return launch_umma_t<64, 4, 3, 512, 2, 4>(wm, bm, tm, p, grid, stream);
+        // a grid larger than the SM count would run in two waves with one CTA per SM: two smaller CTAs per SM instead
+        case 64: return grid.x * grid.y * grid.z > 148 ? launch_umma_t<64, 2, 2, 256, 1, 2>(wm, bm, tm, p, grid, stream)
+                                                       : launch_umma_t<64, 4, 3, 512, 2, 4>(wm, bm, tm, p, grid, stream);
         default: return launch_umma_t<128, 2, 6, 512, 1, 4>(wm, bm, tm, p, grid, stream);
     }
 }
