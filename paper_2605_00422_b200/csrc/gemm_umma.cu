@@ -13,8 +13,8 @@
 //     (programmatic dependent launch);
 //   * warp 1 waits for the preceding kernel, then streams the three bf16 terms of T and the activation codes
 //     (tokens x 128 bytes per k-block, the canonical K-major 128B-swizzled UMMA layout);
-//   * warps 6..13 (two per tensor-memory lane quarter, thread = output row, the two warps of a quarter taking
-//     alternate k-blocks) stage the U tile in shared memory, then turn each 32-bit sign word into eight registers
+//   * warps 6.. (EW = 2 or 4 per tensor-memory lane quarter, thread = output row, the warps of a quarter taking
+//     k-blocks in turn) stage the U tile in shared memory, then turn each 32-bit sign word into eight registers
 //     of four int8 with one shift and one mask per register ((w << (7-j)) & 0x80808080) and write them with
 //     tcgen05.st into tensor memory, where they are the A operand: expanded weights never touch shared memory.
 //   * NISS threads (one each in warps 2..5) issue tcgen05.mma.kind::i8 (M = 128, N = tokens, K = 32; A from tensor
@@ -22,8 +22,11 @@
 //     tensor memory: with few tokens an MMA is short and the issue latency of one thread would be the bottleneck.
 //     The first of them also issues the kind::f16 MMAs of the low-rank term (A = U tile, B = T as three bf16
 //     terms, fp32 accumulator in tensor memory);
-//   * warps 6..13 read the accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
+//   * the same warps read the accumulators back (tcgen05.ld), reduce across the cluster when K is split, apply the
 //     scales, transpose through shared memory and store bf16 with 128-bit stores.
+// Few tokens make the K loop a chain of latencies rather than of throughput; the launch then takes either two CTAs per SM
+// (8 expander warps and 256 tensor-memory columns each) or, when a K split puts the whole grid on the SMs at once, one
+// CTA per SM with 16 expander warps and all 512 columns (a twice as deep operand ring).
 // The shift-and-mask expansion meets the weights of a 32-group in the order k = j + 8*i (register j, byte i), so the
 // codes are stored in that interleaved order by the quantiser.
 //
@@ -41,7 +44,7 @@ using namespace ptx;
 constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
 constexpr int kBlockK = 128;             // K per code sub-block / per tensor-memory A stage
-constexpr int kFirstExpander = 192;      // warps 0, 1: TMA; warps 2..5: MMA issue; warps 6..13: expand + epilogue
+constexpr int kFirstExpander = 192;      // warps 0, 1: TMA; warps 2..5: MMA issue; warps 6..: expand + epilogue
 constexpr uint32_t kParkNs = 4000;          // longest a single poll of a barrier may park its thread
 constexpr uint32_t kWaitLimit = 1u << 15;   // polls per wait before giving up (about a tenth of a second when nothing arrives)
 

@@ -7,16 +7,18 @@
 // (Sec. 3.1: R = R1 (x) R2 evaluated as two small contractions on the reshaped vector; Sec. 4.1: per-token
 // activation quantisation; Sec. 3.2: W x = (W - M) x + A (B x).)
 //
-// Rotation blocks: a thread-block cluster of C CTAs owns one token.  With many tokens C = 1 and the CTA evaluates
-// Z = X * P2, Y = P1^T * Z in chunks.  With few tokens C > 1 spreads one token's 2*K*(n1+n2) flops over C SMs: CTA c
-// owns a slab of rows of Y and evaluates the product in the other order, Z' = (P1^T X)[slab], Y[slab] = Z' * P2,
-// which needs all of x (a few KB) but nothing from the other CTAs; only the absmax and the code sums cross the
-// cluster (distributed shared memory).  X, Z and Y never touch HBM.  Both contractions are register-tiled fp32 FMA
-// loops; codes leave as 128-bit stores.
+// Rotation blocks.  Many tokens whose constants fit beside X and Z: one CTA per token evaluates Z = X * P2, Y = P1^T * Z
+// with register-tiled fp32 FMA loops.  Few tokens: a thread-block cluster of C CTAs owns one token; CTA c owns a slab of
+// rows of Y and evaluates the product in the other order, Z' = (P1^T X)[slab], Y[slab] = Z' * P2, which needs all of x (a
+// few KB) but nothing from the other CTAs; only the absmax crosses the cluster (distributed shared memory).  Where the
+// operands fit, these slab contractions run on the warp-level tensor-core path with fp32 factors split into three bf16
+// terms (see tc_stage_a); a P2 too large for that keeps its fp32 form and only the first contraction does.  Many
+// tokens of a large K: such clusters stay resident, keep the constants and take tokens in turn.  X, Z and Y never
+// touch HBM; codes leave as 128-bit stores; the code sum of a token is left as one partial sum per CTA.
 //
-// Low-rank blocks (after the rotation blocks in the same grid): each reduces two rows of V against a tile of 16
-// tokens with 128-bit loads and writes T split into three bf16 terms (T = hi + mid + lo, all 24 bits of the fp32 sum), the form
-// the tensor-core epilogue of the contraction consumes.
+// Low-rank blocks (in the same grid): T = V x on the warp-level tensor-core path, tiles of 16 tokens x 8 (or 64)
+// columns, written as three bf16 terms (T = hi + mid + lo, all 24 bits of the fp32 sum), the form the tensor-core
+// epilogue of the contraction consumes.  (FMA versions remain for rows that are not 16-byte aligned.)
 //
 // The kernel is launched with programmatic stream serialisation.  The activations may be the output of the
 // preceding kernel of the stream, so only the layer's own constants (P1, P2, rows of V) are fetched before that
