@@ -62,6 +62,9 @@ ROT_CASES = [
     (24, 8, 1, 6),        # slab boundaries must stay on 32-element groups
     (160, 160, 150, 6),   # many tokens of the largest K: clusters that stay and take several tokens each
     (160, 160, 41, 8),
+    (128, 40, 2, 6),      # n2 a multiple of 8 but not of 16: only the first contraction on the tensor-core path
+    (96, 72, 3, 8),
+    (80, 64, 5, 4),       # both contractions on the tensor-core path, slab of 10 rows padded to 16
 ]
 
 
