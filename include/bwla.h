@@ -158,9 +158,22 @@ int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int
  */
 int bwla_check_status(void* workspace, void* stream);
 
-/* Force every later call in this process onto one kernel family (benchmarking the non-chosen path,
- * cross-checks).  Returns BWLA_ERR_INVALID_ARG for an unknown value.  Not thread-safe against
- * concurrent compute calls. */
+/*
+ * Where bwla_w1ax_linear keeps an intermediate inside its workspace, so that tests can compare the quantiser's
+ * output of the fused call itself (Sec. 4.1) and not only that of bwla_rotate_quant_act.  No launch.
+ *   which: BWLA_WS_SCALES  fp32 [M]                        per-token scale s_t
+ *          BWLA_WS_QSUM    int32 [M][8]                    partial code sums; sum_k q_t[k] is the sum of the eight
+ *          BWLA_WS_T       bf16 [3][M][max(64, r)]         T = V x as hi + mid + lo
+ *          BWLA_WS_CODES   int8 [M][K]                     codes; on the tensor-core path inside each group of 32
+ *                                                          consecutive k, byte 4*j + i holds k = j + 8*i
+ *   offset, bytes: host pointers that receive the section's position and size.
+ * Returns BWLA_ERR_INVALID_ARG for invalid dimensions or an unknown section.
+ */
+enum { BWLA_WS_SCALES = 0, BWLA_WS_QSUM = 1, BWLA_WS_T = 2, BWLA_WS_CODES = 3 };
+int bwla_workspace_section(int64_t M, int64_t K, int64_t N, int r, int bits, int which, size_t* offset, size_t* bytes);
+
+/* Force every later call of the calling thread onto one kernel family (benchmarking the non-chosen path,
+ * cross-checks); the setting is per thread.  Returns BWLA_ERR_INVALID_ARG for an unknown value. */
 int bwla_force_path(int path);
 
 /* The family BWLA_PATH_AUTO resolves to for this problem (no launch). */

@@ -33,6 +33,7 @@ EXPORTS = [
     "bwla_pack_signs", "bwla_rotate_quant_act", "bwla_workspace_bytes", "bwla_w1ax_linear", "bwla_w1a_gemm_codes",
     "bwla_check_status", "bwla_force_path", "bwla_chosen_path", "bwla_last_launch_count", "bwla_last_cuda_error",
     "bwla_status_string", "bwla_profile_enable", "bwla_profile_collect", "bwla_w1ax_linear_static",
+    "bwla_workspace_section",
 ]
 
 
@@ -57,6 +58,8 @@ def _load() -> C.CDLL:
     lib.bwla_w1a_gemm_codes.argtypes = [vp, vp, i64, i64, ci, vp, vp, vp, vp, i64, vp, vp, ci, vp, i64, i64, vp,
                                         vp, sz, vp]
     lib.bwla_check_status.argtypes = [vp, vp]
+    lib.bwla_workspace_section.argtypes = [i64, i64, i64, ci, ci, ci, C.POINTER(sz), C.POINTER(sz)]
+    lib.bwla_workspace_section.restype = ci
     lib.bwla_w1ax_linear_static.argtypes = [vp, i64, i64, i64, vp, ci, vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, i64, i64, vp]
     lib.bwla_w1ax_linear_static.restype = ci
     lib.bwla_force_path.argtypes = [ci]
@@ -159,11 +162,8 @@ def bwla_rotate_quant_act(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, b
     return codes, scales
 
 
-def bwla_w1ax_linear(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, bits: int, packed: torch.Tensor,
-                     alpha: torch.Tensor, U: Optional[torch.Tensor] = None, V: Optional[torch.Tensor] = None,
-                     mu: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
-                     workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """The whole layer: bf16 x [M][K] -> bf16 out [M][N]."""
+def _linear_args(x, P1, P2, packed, alpha, U, V, mu, out):
+    """Type and layout checks shared by the two whole-layer entry points; returns (M, K, N, r, out)."""
     _need(x, torch.bfloat16, "x", 2)
     _need(packed, torch.int32, "packed", 2)
     _need(alpha, torch.float32, "alpha", 1)
@@ -183,6 +183,15 @@ def bwla_w1ax_linear(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, bits: 
     if out is None:
         out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
     _need(out, torch.bfloat16, "out", 2)
+    return M, K, N, r, out
+
+
+def bwla_w1ax_linear(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, bits: int, packed: torch.Tensor,
+                     alpha: torch.Tensor, U: Optional[torch.Tensor] = None, V: Optional[torch.Tensor] = None,
+                     mu: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                     workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The whole layer: bf16 x [M][K] -> bf16 out [M][N]."""
+    M, K, N, r, out = _linear_args(x, P1, P2, packed, alpha, U, V, mu, out)
     if workspace is None:
         workspace = new_workspace(M, K, N, r, bits, x.device)
     st = _lib.bwla_w1ax_linear(_ptr(x), M, K, x.stride(0) if M > 0 else K, _ptr(P1), P1.shape[0], _ptr(P2),
@@ -199,25 +208,7 @@ def bwla_w1ax_linear_static(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor,
     """The whole layer through the entry point that owns its scratch memory (see include/bwla.h): for callers that
     cannot allocate a workspace.  `out` should be passed by such a caller; it is created here only for convenience.
     Calls share one built-in scratch array per device and must not overlap on the GPU."""
-    _need(x, torch.bfloat16, "x", 2)
-    _need(packed, torch.int32, "packed", 2)
-    _need(alpha, torch.float32, "alpha", 1)
-    M, K = x.shape
-    N = packed.shape[0]
-    r = 0
-    if U is not None:
-        _need(U, torch.bfloat16, "U", 2)
-        _need(V, torch.bfloat16, "V", 2)
-        r = U.shape[1]
-        if not (U.is_contiguous() and V.is_contiguous()) or tuple(V.shape) != (r, K) or U.shape[0] != N:
-            raise TypeError("U must be contiguous [N][r] and V contiguous [r][K]")
-    if mu is not None:
-        _need(mu, torch.float32, "mu", 1)
-    if not (packed.is_contiguous() and P1.is_contiguous() and P2.is_contiguous()):
-        raise TypeError("packed, P1 and P2 must be contiguous")
-    if out is None:
-        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
-    _need(out, torch.bfloat16, "out", 2)
+    M, K, N, r, out = _linear_args(x, P1, P2, packed, alpha, U, V, mu, out)
     st = _lib.bwla_w1ax_linear_static(_ptr(x), M, K, x.stride(0) if M > 0 else K, _ptr(P1), P1.shape[0], _ptr(P2),
                                       P2.shape[0], bits, _ptr(packed), _ptr(alpha), _ptr(mu), _ptr(U), _ptr(V), r,
                                       _ptr(out), N, out.stride(0) if M > 0 else N, _stream())
@@ -257,6 +248,16 @@ def bwla_w1a_gemm_codes(codes: torch.Tensor, scales: torch.Tensor, bits: int, pa
                                   _ptr(workspace), workspace.numel(), _stream())
     _check(st, "bwla_w1a_gemm_codes")
     return out, acc
+
+
+BWLA_WS_SCALES, BWLA_WS_QSUM, BWLA_WS_T, BWLA_WS_CODES = 0, 1, 2, 3
+
+
+def bwla_workspace_section(M: int, K: int, N: int, r: int, bits: int, which: int):
+    """(offset, bytes) of one intermediate inside the workspace of bwla_w1ax_linear."""
+    off, nb = C.c_size_t(0), C.c_size_t(0)
+    _check(_lib.bwla_workspace_section(M, K, N, r, bits, which, C.byref(off), C.byref(nb)), "bwla_workspace_section")
+    return int(off.value), int(nb.value)
 
 
 def bwla_check_status(workspace: torch.Tensor) -> int:

@@ -7,7 +7,7 @@ namespace bwla {
 
 thread_local int g_last_cuda_error = 0;
 thread_local int g_launch_count = 0;
-static int g_forced_path = BWLA_PATH_AUTO;
+static thread_local int g_forced_path = BWLA_PATH_AUTO;   // per calling thread, like the other bookkeeping
 
 // ---- optional kernel timing -------------------------------------------------------------------
 struct ProfPair { cudaEvent_t a, b; int kind; };
@@ -54,11 +54,10 @@ static bool valid_rotation_dims(int64_t K, int n1, int n2) {
 
 // Which kernel family runs the contraction.  A forced family that cannot take the shape falls back to the simple one.
 static int resolve_path(int64_t M, int64_t K, int64_t N, int r, int bits) {
-    (void)bits;
     int path = g_forced_path;
     if (path == BWLA_PATH_AUTO) path = BWLA_PATH_I8;
     if (path == BWLA_PATH_BITPLANE) path = BWLA_PATH_SIMPLE;   // not built yet
-    if (path == BWLA_PATH_I8 && !umma_supports(M, K, N, r)) path = BWLA_PATH_SIMPLE;
+    if (path == BWLA_PATH_I8 && !umma_supports(M, K, N, r, bits)) path = BWLA_PATH_SIMPLE;
     return path;
 }
 
@@ -116,19 +115,33 @@ static int validate_gemm_tail(int64_t M, int64_t K, int bits, const uint32_t* pa
     return BWLA_OK;
 }
 
-int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2,
-                     int n2, int bits, const uint32_t* packed, const float* alpha, const float* mu, const void* U_bf16,
-                     const void* V_bf16, int r, void* out_bf16, int64_t N, int64_t ldo, void* workspace,
-                     size_t workspace_bytes, void* stream) {
-    g_launch_count = 0;
+}  // extern "C"
+
+// Every check bwla_w1ax_linear makes before it touches the GPU (also used by the entry point with built-in scratch).
+int bwla::validate_linear_call(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1,
+                               const float* P2, int n2, int bits, const uint32_t* packed, const float* alpha,
+                               const void* U_bf16, const void* V_bf16, int r, const void* out_bf16, int64_t N,
+                               int64_t ldo, const void* workspace, size_t workspace_bytes) {
     if (!valid_rotation_dims(K, n1, n2) || ldx < K) return BWLA_ERR_INVALID_ARG;
     int st = validate_gemm_tail(M, K, bits, packed, alpha, U_bf16, V_bf16, r, N, ldo, workspace, workspace_bytes);
     if (st != BWLA_OK) return st;
     if (M == 0 || N == 0) return BWLA_OK;
     if (!x_bf16 || !P1 || !P2 || !out_bf16) return BWLA_ERR_INVALID_ARG;
     if (((uintptr_t)P1 & 15) || ((uintptr_t)P2 & 15)) return BWLA_ERR_INVALID_ARG;
-    st = check_device();
+    return check_device();
+}
+
+extern "C" {
+
+int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2,
+                     int n2, int bits, const uint32_t* packed, const float* alpha, const float* mu, const void* U_bf16,
+                     const void* V_bf16, int r, void* out_bf16, int64_t N, int64_t ldo, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    g_launch_count = 0;
+    int st = validate_linear_call(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, packed, alpha, U_bf16, V_bf16, r, out_bf16, N,
+                                  ldo, workspace, workspace_bytes);
     if (st != BWLA_OK) return st;
+    if (M == 0 || N == 0) return BWLA_OK;
 
     cudaStream_t s = (cudaStream_t)stream;
     const Workspace ws = workspace_layout(M, K, N, r, bits);
@@ -183,6 +196,18 @@ int bwla_w1a_gemm_codes(const int8_t* codes, const float* scales, int64_t M, int
     g.mu = mu; g.Thl = r > 0 ? Thl : nullptr; g.U = U_bf16; g.r = r; g.out = out_bf16; g.ldo = ldo; g.acc_debug = acc_debug;
     g.status = (uint32_t*)(base + ws.status);
     return run_contraction(path, g, inter ? inter : codes, s);
+}
+
+int bwla_workspace_section(int64_t M, int64_t K, int64_t N, int r, int bits, int which, size_t* offset, size_t* bytes) {
+    if (!offset || !bytes || M < 0 || K <= 0 || K % 32 != 0 || N < 0 || r < 0 || !valid_bits(bits)) return BWLA_ERR_INVALID_ARG;
+    const Workspace w = workspace_layout(M, K, N, r, bits);
+    switch (which) {
+        case BWLA_WS_SCALES: *offset = w.scales; *bytes = (size_t)M * 4; return BWLA_OK;
+        case BWLA_WS_QSUM:   *offset = w.qsum;   *bytes = (size_t)M * 4 * kQsumParts; return BWLA_OK;
+        case BWLA_WS_T:      *offset = w.T;      *bytes = (size_t)M * lowrank_cols(r) * 6; return BWLA_OK;
+        case BWLA_WS_CODES:  *offset = w.codes;  *bytes = (size_t)M * (size_t)K; return BWLA_OK;
+        default: return BWLA_ERR_INVALID_ARG;
+    }
 }
 
 int bwla_check_status(void* workspace, void* stream) {

@@ -10,7 +10,7 @@
 namespace bwla {
 
 // ---------------------------------------------------------------------------------------------
-// per-thread bookkeeping (no global mutable state apart from the forced path)
+// per-thread bookkeeping (the library keeps no process-global mutable state)
 // ---------------------------------------------------------------------------------------------
 extern thread_local int g_last_cuda_error;
 extern thread_local int g_launch_count;
@@ -36,6 +36,19 @@ inline int after_launch() {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Number of SMs of the current device (cached per thread and device); 0 if it cannot be queried.
+inline int sm_count() {
+    static thread_local int cached_dev = -1, cached_n = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (dev != cached_dev) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+        cached_dev = dev; cached_n = n;
+    }
+    return cached_n;
+}
+
 // ---------------------------------------------------------------------------------------------
 // optional per-kernel timing (bwla_profile_enable / bwla_profile_collect): CUDA events recorded on the launching
 // stream right around each kernel launch, summed per kernel kind.  Off by default; not usable under stream capture.
@@ -56,11 +69,7 @@ struct ProfScope {
 // ---------------------------------------------------------------------------------------------
 // workspace layout (byte offsets into the caller's scratch buffer; every section 256-byte aligned)
 // ---------------------------------------------------------------------------------------------
-#ifdef BWLA_TRACE
-constexpr int kStatusBytes = 8192;       // tuning builds keep a timeline behind the status words
-#else
 constexpr int kStatusBytes = 256;        // word 0: status; words 1..: where a bounded wait gave up
-#endif
 constexpr int kLowrankPad = 64;          // T is kept as bf16 [3][M][64] (T = hi + mid + lo), zero beyond r <= 64
 
 // The code sum of a token is kept as kQsumParts partial sums (one per CTA of the prologue cluster that quantised a slab
@@ -92,6 +101,13 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     w.total = off;
     return w;
 }
+
+// Argument checks of bwla_w1ax_linear (everything that can be refused without touching the GPU, then the device check).
+// BWLA_OK also for the empty problems M == 0 / N == 0, which the caller turns into a no-op.
+int validate_linear_call(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2,
+                         int n2, int bits, const uint32_t* packed, const float* alpha, const void* U_bf16,
+                         const void* V_bf16, int r, const void* out_bf16, int64_t N, int64_t ldo, const void* workspace,
+                         size_t workspace_bytes);
 
 // ---------------------------------------------------------------------------------------------
 // kernel launchers (each returns a BWLA status; all asynchronous on `stream`)
@@ -133,7 +149,7 @@ struct GemmArgs {
 int launch_gemm_simple(const GemmArgs& a, cudaStream_t stream);
 
 // tcgen05 path with the fused epilogue.  codes_interleaved: int8 [M][K] in the interleaved order.
-bool umma_supports(int64_t M, int64_t K, int64_t N, int r);
+bool umma_supports(int64_t M, int64_t K, int64_t N, int r, int bits);
 int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream);
 
 }  // namespace bwla

@@ -99,38 +99,6 @@ struct UmmaCfg {
     static_assert(N_TOK * kRowsPerCta * 2 <= u_off, "output tile does not fit the stage memory");
 };
 
-// Optional timeline of CTA (0,0,0) for tuning: clock64 stamps behind the status words (compiled out by default).
-#ifdef BWLA_TRACE
-#define BWLA_STAMP(i) do { if (p.status && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
-        reinterpret_cast<long long*>(p.status + 16)[i] = clock64(); } while (0)
-// and start / first weights / K loop done / accumulators ready / exit of every CTA on the GPU-wide nanosecond timer
-__device__ unsigned long long g_cta_times[4096 * 8];
-__device__ __forceinline__ unsigned long long global_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define BWLA_CTA_STAMP(i) do { const unsigned lb = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); \
-        if (lb < 4096) g_cta_times[lb * 8 + (i)] = global_ns(); } while (0)
-// clock stamps of the ring of CTA (0,0,0), kept in shared memory while the loop runs (a global store per stamp would
-// disturb what it measures): [w][i][.] for w < 8 the first eight expander warps' i-th own k-block (0 before the wait for
-// the stage, 1 stage free, 2 stored, 3 handed over), for w = 8, 9 the issuing threads' (0 before the wait for the
-// operand, 1 operand there, 2 issued and committed)
-__device__ unsigned int g_ring_log[10 * 32 * 4];
-#define BWLA_RING_DECL __shared__ unsigned int ring_log[10 * 32 * 4];
-#define BWLA_RING(who, i, j) do { if ((who) < 10 && (i) < 32) ring_log[((who) * 32 + (i)) * 4 + (j)] = (unsigned int)clock(); } while (0)
-#define BWLA_RING_DUMP do { __syncthreads(); if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) \
-        for (int i_ = threadIdx.x; i_ < 10 * 32 * 4; i_ += blockDim.x) g_ring_log[i_] = ring_log[i_]; } while (0)
-extern "C" int bwla_trace_ring(unsigned int* host) {
-    return cudaMemcpyFromSymbol(host, g_ring_log, sizeof(g_ring_log)) == cudaSuccess ? 0 : -4;
-}
-extern "C" int bwla_trace_ctas(unsigned long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, g_cta_times, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -4;
-}
-#else
-#define BWLA_STAMP(i) do { } while (0)
-#define BWLA_CTA_STAMP(i) do { } while (0)
-#define BWLA_RING_DECL
-#define BWLA_RING(who, i, j) do { } while (0)
-#define BWLA_RING_DUMP do { } while (0)
-#endif
-
 __device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
     if (status) {
         atomicExch(status, 1u);
@@ -177,7 +145,6 @@ __global__ void __launch_bounds__(kFirstExpander + 128 * EW, TMEM_COLS == 256 ? 
 umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap b_map,
                 const __grid_constant__ CUtensorMap t_map, UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
-    BWLA_RING_DECL
     using L = UmmaCfg<N_TOK, WS, BS, TMEM_COLS, NISS, EW>;
     constexpr int AS = L::AS;
     constexpr int SUBS = L::SUBS;
@@ -215,7 +182,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     const int unit_end = (int)(((int64_t)(split + 1) * p.total_units) / p.splits);
     const bool lowrank = p.r > 0;
     const bool lowrank_here = lowrank && split == 0;   // the low-rank accumulator lives in the first CTA of a cluster
-    if (threadIdx.x == 0) { BWLA_STAMP(0); BWLA_CTA_STAMP(0); }
 
     auto sub_count = [&](int u) { return min(kUnitK / kBlockK, (p.K - u * kUnitK) / kBlockK); };
     // k-blocks this CTA contracts; every unit but the last of the matrix has eight
@@ -250,7 +216,12 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             tma_prefetch_desc(&w_map);
             int ws = 0; uint32_t wph = 0;
             for (int u = unit_begin; u < unit_end && !*abort_flag; ++u) {
-                if (!wait_or_abort(&w_empty[ws], wph ^ 1, abort_flag)) { give_up(p.status, abort_flag, 0x10); break; }
+                // A stage that is not free yet is released by the expansion, which in the end waits for the preceding
+                // kernel's codes: the bounded wait starts counting once that kernel has finished.
+                if (!mbar_test_wait(&w_empty[ws], wph ^ 1)) {
+                    griddep_wait();
+                    if (!wait_or_abort(&w_empty[ws], wph ^ 1, abort_flag)) { give_up(p.status, abort_flag, 0x10); break; }
+                }
                 mbar_expect_tx(&w_full[ws], L::w_bytes);
                 tma_load_2d(wbuf + ws * L::w_bytes, &w_map, u * (kUnitK / 32), n0, &w_full[ws]);
                 if (++ws == WS) { ws = 0; wph ^= 1; }
@@ -305,6 +276,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc_lr = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
             bool ok = true;
+            griddep_wait();                           // everything this thread waits for follows the preceding kernel
             if (iss == 0 && lowrank_here) {
                 if (!wait_or_abort(u_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x32); ok = false; }
                 if (ok && !wait_or_abort(t_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x33); ok = false; }
@@ -343,11 +315,8 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 for (int sb = 0; sb < SUBS; ++sb) {
                     const bool own = (SUBS % NISS == 0) ? (sb % NISS == iss) : ((kb0 + sb) % NISS == iss);
                     if (ok && sb < cnt && own) {
-                        BWLA_RING(8 + iss, (kb0 + sb) / NISS, 0);
                         if (!wait_or_abort(&a_full[as], aph, abort_flag)) { give_up(p.status, abort_flag, 0x31); ok = false; }
-                        BWLA_RING(8 + iss, (kb0 + sb) / NISS, 1);
                         if (ok) {
-                            if (kb0 + sb == 0) BWLA_STAMP(8);
                             tc_fence_after();
                             const uint64_t desc = desc_hi | (uint64_t)(stage_lo + (uint32_t)sb * (L::sub_bytes >> 4));
                             const uint32_t a_addr = a_base + 32 * as;
@@ -357,7 +326,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                                 acc = 1u;
                             }
                             tc_commit(&a_empty[as]);
-                            BWLA_RING(8 + iss, (kb0 + sb) / NISS, 2);
                             as += NISS;
                             if (as >= AS) { as -= AS; aph ^= 1u; }
                         }
@@ -368,7 +336,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 if (++bs == BS) { bs = 0; bph ^= 1u; }
             }
             tc_commit(d_full);
-            if (iss == 0) BWLA_STAMP(9);
         }
     } else {
         // ---------------- U tile, expansion of sign bits into tensor memory, then the epilogue ----------------
@@ -415,15 +382,10 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         int ws = 0; uint32_t wph = 0;
         int as = part; uint32_t aph = 0;
         bool ok = true;
-        int nown = 0;   // own k-blocks so far (tuning stamps only)
         for (int u = unit_begin; u < unit_end && ok; ++u) {
-            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 0);
             if (!warp_wait(&w_full[ws], wph, abort_flag)) { give_up(p.status, abort_flag, 0x40); ok = false; break; }
-            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 1);
-            if (e == 64 && u == unit_begin) { BWLA_STAMP(3); BWLA_CTA_STAMP(1); }
             const uint8_t* wrow = wbuf + ws * L::w_bytes + row * 128;
             const int ns = sub_count(u);
-            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 2);
             // a rolled loop over this warp's k-blocks of the unit; each block's sign words are loaded just before they are
             // expanded
 #pragma unroll 1
@@ -435,19 +397,19 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[8 * c + j] = (w[c] << (7 - j)) & 0x80808080u;
-                if (lane == 0) BWLA_RING(warp - 6, nown, 0);
-                if (!warp_wait(&a_empty[as], aph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x41); ok = false; }
-                if (lane == 0) BWLA_RING(warp - 6, nown, 1);
+                // An operand stage that is still taken frees up only when MMAs have run, and those need the codes of the
+                // preceding kernel: the bounded wait starts counting once that kernel has finished.
+                if (!__all_sync(0xFFFFFFFFu, mbar_test_wait(&a_empty[as], aph ^ 1u))) {
+                    griddep_wait();
+                    if (!warp_wait(&a_empty[as], aph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x41); ok = false; }
+                }
                 if (ok) {
                     tc_fence_after();
                     tmem_st_32x32(tmem_base + lane_addr + L::A_COL + 32 * as, v);
                     tc_wait_st();
-                    if (lane == 0) BWLA_RING(warp - 6, nown, 2);
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&a_full[as]);
-                    if (lane == 0) BWLA_RING(warp - 6, nown, 3);
-                    ++nown;
                     as += EW;
                     if (as >= AS) { as = part; aph ^= 1u; }
                 }
@@ -456,10 +418,8 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             // an arrive placed earlier let the copy of a later unit overwrite words not yet read.
             __syncwarp();
             if (lane == 0) mbar_arrive(&w_empty[ws]);
-            if (lane == 0) BWLA_RING(warp - 6, 24 + (u - unit_begin), 3);
             if (++ws == WS) { ws = 0; wph ^= 1u; }
         }
-        if (e == 64) { BWLA_STAMP(4); BWLA_CTA_STAMP(2); }
         // the stores of the epilogue come after the preceding kernel; the per-token scales and code sums it wrote were
         // staged in shared memory by warp 1 while the K loop ran
         griddep_wait();
@@ -467,7 +427,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         if (ok) {
             if (!warp_wait(d_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x50); ok = false; }
         }
-        if (e == 64) { BWLA_STAMP(5); BWLA_CTA_STAMP(3); }
         if (ok) {
             tc_fence_after();
             const int n = n0 + row;
@@ -485,7 +444,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 tmem_ld_32x16(tmem_base + lane_addr + 16 * c, v);
                 if (lowrank_here) tmem_ld_32x16(tmem_base + lane_addr + L::D2_COL + 16 * c, l);
                 tc_wait_ld();
-                if (e == 64 && c == part) BWLA_STAMP(10);
 #pragma unroll
                 for (int a = 1; a < NISS; ++a) {
                     if (a < nacc) {
@@ -496,13 +454,11 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                         for (int j = 0; j < 16; ++j) v[j] += v2[j];
                     }
                 }
-                if (e == 64 && c == part) BWLA_STAMP(13);
                 // the chunk's scales and code sums go to registers first: the tile stores below may alias them as far as
                 // the compiler knows, and a load behind every store would serialise the loop
                 float sc[16]; int32_t qs[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) { sc[j] = scale_s[16 * c + j]; qs[j] = qsum_s[16 * c + j]; }
-                if (e == 64 && c == part) BWLA_STAMP(14);
                 // branch-free per element (rows beyond N and tokens beyond M produce values nobody stores):
                 // a branch per element costs more than the arithmetic it would skip
                 if (dbg && valid_row) {
@@ -526,10 +482,8 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 }
             }
         }
-        if (e == 64) BWLA_STAMP(11);
         if (p.splits == 1) {
             asm volatile("bar.sync 1, %0;" ::"r"(kExpanders) : "memory");   // the output tile is complete (all expander warps, always)
-            if (e == 64) BWLA_STAMP(12);
             if (ok && p.out) {
                 // 16 threads move one token's 128 outputs (256 bytes) with 128-bit stores
                 const bool vec = ((reinterpret_cast<uintptr_t>(p.out) & 15) == 0) && (p.ldo % 8 == 0) && (n0 + kRowsPerCta <= p.N);
@@ -548,15 +502,12 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             }
         }
     }
-    if (threadIdx.x == kFirstExpander) { BWLA_STAMP(6); BWLA_CTA_STAMP(4); }
-    BWLA_RING_DUMP;
     tc_fence_before();
     __syncthreads();
     if (p.splits > 1) {
         // every thread of every CTA of the cluster takes part, whether or not its CTA gave up
         cluster_arrive_release();
         cluster_wait_acquire();
-        if (threadIdx.x == kFirstExpander) BWLA_CTA_STAMP(6);
         if (L::can_split && warp >= 6 && !*abort_flag) {
             // the tokens of the tile are dealt round-robin to the CTAs of the cluster; a thread sums four consecutive
             // rows of one token over all CTAs with 128-bit distributed-shared-memory loads
@@ -600,7 +551,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 }
             }
         }
-        if (threadIdx.x == kFirstExpander) BWLA_CTA_STAMP(7);
         // nobody leaves while a neighbour may still read its shared memory
         cluster_arrive_release();
         cluster_wait_acquire();
@@ -609,7 +559,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
-        if (lane == 0) { BWLA_STAMP(7); BWLA_CTA_STAMP(5); }
     }
 }
 
@@ -676,17 +625,19 @@ static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUt
     return after_launch();
 }
 
-bool umma_supports(int64_t M, int64_t K, int64_t N, int r) {
-    return M > 0 && N > 0 && K % 128 == 0 && r <= kLowrankPad && M * N < (int64_t)1 << 31 && M < (int64_t)1 << 30 &&
-           encode_tiled_fn() != nullptr;
+bool umma_supports(int64_t M, int64_t K, int64_t N, int r, int bits) {
+    // the tensor core sums -128 * code over the set sign bits: |D| <= 128 * K * qmax must fit the int32 accumulator
+    const int64_t qmax = ((int64_t)1 << (bits - 1)) - 1;
+    return M > 0 && N > 0 && K % 128 == 0 && 128 * K * qmax < ((int64_t)1 << 31) && r <= kLowrankPad &&
+           M * N < (int64_t)1 << 31 && M < (int64_t)1 << 30 && encode_tiled_fn() != nullptr;
 }
 
 // How many CTAs share a tile and split K, for the configuration with two CTAs per SM.  Enough to put about one CTA on
 // every SM, never more than the units there are, never more than the portable cluster size; powers of two.
-static int choose_splits(int tiles, int units, bool can_split) {
+static int choose_splits(int tiles, int units, bool can_split, int sms) {
     if (!can_split) return 1;
     int s = 1;
-    while (s * 2 <= 8 && s * 2 <= units && tiles * s * 2 <= 148 + 148 / 4) s *= 2;
+    while (s * 2 <= 8 && s * 2 <= units && tiles * s * 2 <= sms + sms / 4) s *= 2;
     return s;
 }
 
@@ -694,15 +645,15 @@ static int choose_splits(int tiles, int units, bool can_split) {
 // and a twice as deep operand ring (all 512 tensor-memory columns) gets through its k-blocks about 1.7 times as fast
 // as one of two CTAs that share an SM.  It is worth it when a K split puts the whole grid on the SMs at once.
 // Returns the split for that configuration, or 0 when two CTAs per SM are expected to finish sooner.
-static int choose_wide_splits(int tiles, int units, int narrow_splits) {
-    if (tiles > 148) return 0;
-    int s = 148 / tiles;
+static int choose_wide_splits(int tiles, int units, int narrow_splits, int sms) {
+    if (tiles > sms) return 0;
+    int s = sms / tiles;
     if (s > 8) s = 8;
     if (s > units) s = units;
     if (s < 1) return 0;
     const int blocks = units * (kUnitK / kBlockK);
     const double wide = (double)((blocks + s - 1) / s) / 1.7;
-    const double narrow = (double)((blocks + narrow_splits - 1) / narrow_splits) * (tiles * narrow_splits > 148 ? 1.2 : 1.0);
+    const double narrow = (double)((blocks + narrow_splits - 1) / narrow_splits) * (tiles * narrow_splits > sms ? 1.2 : 1.0);
     return wide < narrow ? s : 0;
 }
 
@@ -713,8 +664,10 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
     const int row_tiles = (N + kRowsPerCta - 1) / kRowsPerCta;
     const int tok_tiles = (M + n_tok - 1) / n_tok;
     const int units = (K + kUnitK - 1) / kUnitK;
-    int split = choose_splits(row_tiles * tok_tiles, units, n_tok <= 64);
-    const int wide_split = n_tok <= 32 ? choose_wide_splits(row_tiles * tok_tiles, units, split) : 0;
+    const int sms = sm_count();
+    if (sms <= 0) return BWLA_ERR_CUDA;
+    int split = choose_splits(row_tiles * tok_tiles, units, n_tok <= 64, sms);
+    const int wide_split = n_tok <= 32 ? choose_wide_splits(row_tiles * tok_tiles, units, split, sms) : 0;
     if (wide_split) split = wide_split;
 
     CUtensorMap wm, bm, tm;
@@ -757,7 +710,7 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
         case 32: return wide_split ? launch_umma_t<32, 3, 2, 512, 2, 4>(wm, bm, tm, p, grid, stream)
                                    : launch_umma_t<32, 3, 2, 256, 2, 2>(wm, bm, tm, p, grid, stream);
         // a grid larger than the SM count would run in two waves with one CTA per SM: two smaller CTAs per SM instead
-        case 64: return grid.x * grid.y * grid.z > 148 ? launch_umma_t<64, 2, 2, 256, 1, 2>(wm, bm, tm, p, grid, stream)
+        case 64: return grid.x * grid.y * grid.z > (unsigned)sms ? launch_umma_t<64, 2, 2, 256, 1, 2>(wm, bm, tm, p, grid, stream)
                                                        : launch_umma_t<64, 4, 3, 512, 2, 4>(wm, bm, tm, p, grid, stream);
         default: return launch_umma_t<128, 2, 6, 512, 1, 4>(wm, bm, tm, p, grid, stream);
     }

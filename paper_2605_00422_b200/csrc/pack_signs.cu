@@ -36,7 +36,8 @@ int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ld
     if (total == 0) return BWLA_OK;
     const int warps_per_block = 8;
     int64_t blocks = (total + warps_per_block - 1) / warps_per_block;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    const int64_t cap = (int64_t)(sm_count() > 0 ? sm_count() : 128) * 16;   // the kernel strides over the rest
+    if (blocks > cap) blocks = cap;
     ProfScope prof(kProfPack, stream);
     if (dtype == BWLA_DTYPE_F32)
         pack_signs_kernel<float><<<(unsigned)blocks, 256, 0, stream>>>((const float*)w, N, words, ldw, packed);

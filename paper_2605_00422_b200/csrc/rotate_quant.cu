@@ -28,78 +28,13 @@
 #include <algorithm>
 
 #include "bwla_common.cuh"
+#include "prologue_roles.cuh"
 #include "umma_ptx.cuh"
 
 namespace bwla {
 
-using namespace ptx;
-
-constexpr int kLrMaxWarps = 16;   // blocks have at most 512 threads
 constexpr int kPrologueSmemFloats = 57728;   // dynamic shared memory of a prologue block, in floats (225.5 KB; static use is under 1 KB)
 
-// Optional phase timeline of rotation block 0 for tuning (compiled out by default).
-#ifdef BWLA_TRACE
-__device__ long long g_prologue_trace[32];
-#define BWLA_PSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_prologue_trace[i] = clock64(); } while (0)
-extern "C" int bwla_trace_prologue(long long* host32) {
-    return cudaMemcpyFromSymbol(host32, g_prologue_trace, sizeof(long long) * 32) == cudaSuccess ? 0 : -4;
-}
-__device__ unsigned long long g_prologue_block_times[1024 * 4];
-__device__ __forceinline__ unsigned long long prologue_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define BWLA_PBLOCK(i) do { if (threadIdx.x == 0 && blockIdx.x < 1024) g_prologue_block_times[blockIdx.x * 4 + (i)] = prologue_ns(); } while (0)
-extern "C" int bwla_trace_prologue_blocks(unsigned long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, g_prologue_block_times, sizeof(unsigned long long) * (size_t)n) == cudaSuccess ? 0 : -4;
-}
-#else
-#define BWLA_PSTAMP(i) do { } while (0)
-#define BWLA_PBLOCK(i) do { } while (0)
-#endif
-
-struct PrologueParams {
-    const __nv_bfloat16* x; int64_t M; int K; int64_t ldx;
-    // rotation + quantiser (rot_blocks == 0 skips them)
-    const float* P1; int n1; const float* P2; int n2; int bits;
-    int8_t* codes; int codes_layout; float* scales; int32_t* qsum;
-    int C;              // CTAs per token (cluster size)
-    int rot_blocks;     // clusters * C
-    int tok_stride;     // number of clusters: a cluster takes tokens t, t + tok_stride, ... (== M unless the clusters stay and loop)
-    int rot_first;      // first rotation block: 0, or (clusters that stay) behind the low-rank blocks, which then start first
-    int row_gran;       // slab boundaries are multiples of this many rows of X
-    int slab_cap;       // floats reserved for one slab
-    int ps_cap;         // floats reserved for a staged chunk of P2 / P1
-    int ch1, ch2;       // columns of P2 / of P1 staged at a time
-    int prefetch;       // 1: all of P2 and this CTA's columns of P1 are fetched at the start, with x
-    int p1_cap;         // floats reserved for the prefetched columns of P1
-    int tr1, tr2;       // rows per thread in the two contractions
-    int split_y;        // 1 (C > 1): each CTA evaluates its rows of Y from all of x, nothing but absmax is exchanged
-    int sp_tr, sp_rp;   // split_y: rows per thread tile (4 or 8); slab rows rounded up to it (row stride of P1s and Zt)
-    int sp_s;           // split_y: slices the contraction depth is cut into (partial sums are added afterwards); with sp_tc:
-                        // parts the columns of P2 are staged in
-    int sp_tc;          // split_y: 1: both contractions on the warp-level tensor-core path (split-bf16 operands)
-    int sp_zt_off;      // split_y: where Z'^T lives, in floats from the start of shared memory (0: over x, dead by then)
-    int sp_rest_off;    // split_y: where P2 starts
-    // low-rank
-    const __nv_bfloat16* V; int r; int lr_cols; __nv_bfloat16* Thl;   // [3][M][lr_cols]
-    int lr_wide;        // low-rank blocks: 0: 2 rows of V x 16 tokens (FMA), 1: 8 x 8 (FMA, many tokens), 2: 8 columns x 16 tokens on the
-                        // warp-level tensor-core path (few tokens), 3: all 64 columns x 16 tokens on that path (many tokens)
-    int lr_ks;          // lr_wide == 2: blocks that share a tile of T and split K (1: no split)
-    float* lr_part;     // [tiles][lr_ks][16 * 8] partial sums of those blocks
-    uint32_t* lr_count; // one arrival counter per tile, zero between calls
-    int lr_stage;       // 1: a low-rank block copies its rows of V into shared memory before it waits for x
-    int late_trigger;   // 1: the next kernel of the stream is let in only when this one is nearly done (see launch_prologue)
-};
-
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-    return v;
-}
-
-__device__ __forceinline__ int warp_sum(int v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
 
 __device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
@@ -288,27 +223,6 @@ __device__ __forceinline__ float slab_reduce(const float* __restrict__ part, int
         }
     }
     return amax;
-}
-
-// ---------------------------------------------------------------------------------------------
-// The two slab contractions on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 out).
-//
-// An fp32 factor is split into three bf16 terms (hi + mid + lo carry all 24 bits); x is bf16 already.  Every k-step of
-// 16 starts from a zero accumulator, takes the products of the terms that matter (smallest first) and is then added to
-// the running fp32 sum with an ordinary rounded addition: the tensor core only ever sums 16 exact products (48 or 96
-// with the terms), so what its internal accumulation does to long sums does not enter.  The error stays at the level
-// of the fp32 FMA chain (a CPU model of this scheme with the partial sums rounded toward zero is within 3.4e-7 of the
-// token's full scale for K = 25600, the fp32 chain within 5.9e-7; the code window is 1e-6).
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void split3(float v, __nv_bfloat16& h, __nv_bfloat16& m, __nv_bfloat16& l) {
-    h = __float2bfloat16_rn(v);
-    const float r1 = v - __bfloat162float(h);
-    m = __float2bfloat16_rn(r1);
-    l = __float2bfloat16_rn(r1 - __bfloat162float(m));
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
-    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
 }
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -524,7 +438,6 @@ __device__ __forceinline__ void finish_token(const PrologueParams& p, int64_t t,
     const int qmax = (1 << (p.bits - 1)) - 1;
     const int n2 = p.n2, K = p.K;
     int& red_sum = *red_sum_p;
-    BWLA_PSTAMP(6);
     // ---- absmax over the block, then over the cluster
     amax = warp_max(amax);
     if (lane == 0) red_max[warp] = amax;
@@ -537,17 +450,21 @@ __device__ __forceinline__ void finish_token(const PrologueParams& p, int64_t t,
         cluster_wait_acquire();
         float m = (lane < C) ? slots[lane] : 0.f;
         amax = warp_max(m);
+        if (!last) {
+            // a cluster that goes on to another token: nobody may store the next token's absmax into these slots before
+            // every CTA has read this token's
+            cluster_arrive_release();
+            cluster_wait_acquire();
+        }
     }
 
     float inv, scale;
     if (amax == 0.f) { inv = 0.f; scale = 1.f; }
     else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
 
-    BWLA_PSTAMP(7);
     if (p.late_trigger && last) griddep_launch_dependents();
     // nothing is stored to global memory before the preceding kernel of the stream has completed
     griddep_wait();
-    BWLA_PSTAMP(8);
 
     int local_sum = 0;
     int8_t* ct = p.codes + t * (int64_t)K + (int64_t)a_lo * n2;
@@ -585,7 +502,6 @@ __device__ __forceinline__ void finish_token(const PrologueParams& p, int64_t t,
     local_sum = warp_sum(local_sum);
     if (lane == 0 && local_sum != 0) atomicAdd(&red_sum, local_sum);
     __syncthreads();
-    BWLA_PSTAMP(9);
     // every CTA leaves its own part of the token's code sum; the consumer adds the parts, so no exchange is needed here
     if (threadIdx.x == 0) {
         if (p.qsum) {
@@ -595,7 +511,6 @@ __device__ __forceinline__ void finish_token(const PrologueParams& p, int64_t t,
         }
         if (rank == 0) p.scales[t] = scale;
     }
-    BWLA_PSTAMP(10);
 }
 
 __device__ void rotate_role(const PrologueParams& p, float* smem) {
@@ -614,7 +529,6 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     float amax = 0.f;
     if (threadIdx.x == 0) red_sum = 0;
 
-    BWLA_PSTAMP(0);
     if (p.split_y && p.sp_tc == 1) {
         // ---- few tokens, tensor-core contractions: this CTA's rows of Y from all of x
         const TcLayout L = tc_layout(n1, n2, p.sp_rp, p.sp_s);
@@ -637,7 +551,6 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         cluster_arrive_release();              // "this CTA is running": waited for before the first remote store
         if (!p.late_trigger) griddep_launch_dependents();
         griddep_wait();                        // x may be the output of the preceding kernel
-        BWLA_PSTAMP(1); BWLA_PBLOCK(2);
         {
             const __nv_bfloat16* xt = p.x + t * p.ldx;
             const int cpr = n2 >> 3;           // 16-byte chunks per row of X
@@ -656,10 +569,8 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             }
         }
         __syncthreads();
-        BWLA_PSTAMP(2);
         tc_stage_a(L, n2, Xp, P1T, ZT);
         __syncthreads();
-        BWLA_PSTAMP(3);
         amax = tc_stage_b(L, n2, rows, 0, ZT, P2T, Xs);
         for (int c0 = L.pc; c0 < n2; c0 += L.pc) {
             __syncthreads();                   // every warp is done with the columns in place
@@ -667,9 +578,7 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             __syncthreads();
             amax = fmaxf(amax, tc_stage_b(L, n2, rows, c0, ZT, P2T, Xs));
         }
-        BWLA_PSTAMP(4);
         cluster_wait_acquire();
-        BWLA_PSTAMP(5);
     } else if (p.split_y && p.sp_tc == 2) {
         // ---- few tokens, large P2: the first contraction on the tensor-core path (its factor, a slab of P1^T, is small),
         //      the second as FMA tiles over fp32 P2 (splitting all of P2 into terms costs more than it saves there)
@@ -711,7 +620,6 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         cluster_arrive_release();              // "this CTA is running": waited for before the first remote store
         if (!p.late_trigger) griddep_launch_dependents();
         griddep_wait();                        // x may be the output of the preceding kernel
-        BWLA_PSTAMP(1); BWLA_PBLOCK(2);
         // The cluster takes tokens t, t + tok_stride, ...: with few tokens exactly one; with many tokens of a large K the
         // clusters stay, and the constants above are fetched and split once per cluster instead of once per token.
         for (int64_t tt = t; tt < p.M; tt += p.tok_stride) {
@@ -735,18 +643,15 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
                 *reinterpret_cast<uint4*>(Xp + (size_t)a * L.xs + 8 * c) = make_uint4(0u, 0u, 0u, 0u);
             }
             __syncthreads();
-            BWLA_PSTAMP(2);
             tc_stage_a(L, n2, Xp, P1T, nullptr, Zt);
             cp_async_wait_all();               // P2 has been arriving meanwhile; it is first read below
             __syncthreads();                   // x is dead: its place takes the partial sums (and, with one token per
-            BWLA_PSTAMP(3);                    // cluster, that of the P1^T terms too)
+                    // cluster, that of the P1^T terms too)
             slab_partial<8, false>(Zt, rp, P2s, n2, n2, S, part);
             __syncthreads();
             // Y goes where the first slice of the partial sums is: a thread reads its own elements of every slice first
             amax = slab_reduce<false>(part, rp, rows, n2, S, Xs);
-            BWLA_PSTAMP(4);
             if (tt == t) cluster_wait_acquire();
-            BWLA_PSTAMP(5);
             finish_token(p, tt, C, rank, Xs, slots, amax, rows, a_lo, red_max, &red_sum, tt + p.tok_stride >= p.M);
         }
         return;
@@ -771,7 +676,6 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         if (!p.late_trigger) griddep_launch_dependents();
         cp_async_wait_all();                   // made visible to the block by the barrier behind the load of x
         griddep_wait();                        // x may be the output of the preceding kernel
-        BWLA_PSTAMP(1); BWLA_PBLOCK(2);
         {
             const __nv_bfloat16* xt = p.x + t * p.ldx;
             if ((reinterpret_cast<uintptr_t>(xt) & 15) == 0) {
@@ -782,30 +686,16 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             }
         }
         __syncthreads();
-        BWLA_PSTAMP(2);
         if (p.sp_tr == 8) slab_partial<8, true>(P1s, rp, Xh, n1, n2, S, part);
         else slab_partial<4, true>(P1s, rp, Xh, n1, n2, S, part);
         __syncthreads();
         slab_reduce<true>(part, rp, rows, n2, S, Zt);
         __syncthreads();
-        BWLA_PSTAMP(3);
-#ifdef BWLA_TRACE_REPEAT
-        BWLA_PSTAMP(11);
-        if (p.sp_tr == 8) slab_partial<8, true>(P1s, rp, Xh, n1, n2, S, part);
-        else slab_partial<4, true>(P1s, rp, Xh, n1, n2, S, part);
-        __syncthreads();
-        BWLA_PSTAMP(12);
-        slab_reduce<true>(part, rp, rows, n2, S, Zt);
-        __syncthreads();
-        BWLA_PSTAMP(13);
-#endif
         if (p.sp_tr == 8) slab_partial<8, false>(Zt, rp, P2s, n2, n2, S, part);
         else slab_partial<4, false>(Zt, rp, P2s, n2, n2, S, part);
         __syncthreads();
         amax = slab_reduce<false>(part, rp, rows, n2, S, Xs);
-        BWLA_PSTAMP(4);
         cluster_wait_acquire();
-        BWLA_PSTAMP(5);
     } else if ((n2 & 3) == 0) {
         // ---- one CTA per token: Z = X * P2, Y = P1^T * Z, the factors staged chunk by chunk
         float* Zf = smem + p.slab_cap;         // all of Z
@@ -820,7 +710,6 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
         if (!p.late_trigger) griddep_launch_dependents();
         griddep_wait();                        // x may be the output of the preceding kernel
         load_x(p.x + t * p.ldx, K, Xs);
-        BWLA_PSTAMP(1);
         for (int dc = 0; dc < n2; dc += p.ch1) {
             const int cw = min(p.ch1, n2 - dc);
             if (!p.prefetch) for (int i = threadIdx.x; i < n2 * (cw >> 2); i += blockDim.x) {
@@ -828,7 +717,6 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
                 *reinterpret_cast<float4*>(Ps + b * cw + j) = __ldg(reinterpret_cast<const float4*>(p.P2 + (size_t)b * n2 + dc + j));
             }
             __syncthreads();
-            BWLA_PSTAMP(2);
             switch (p.tr1) {
                 case 8: stage1_chunk<8>(Xs, n1, n2, Ps, dc, cw, Zf); break;
                 case 4: stage1_chunk<4>(Xs, n1, n2, Ps, dc, cw, Zf); break;
@@ -837,14 +725,12 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
             }
             __syncthreads();
         }
-        BWLA_PSTAMP(3);
         // Y overwrites X, which is dead now; one chunk of output rows (columns of P1) at a time
         for (int c0 = 0; c0 < n1; c0 += p.ch2) {
             const int cw = min(p.ch2, n1 - c0), cwp = (cw + 3) & ~3;
             const float* Pc = p.prefetch ? P1s : Ps;
             if (!p.prefetch) load_p1_columns(p.P1, n1, c0, cw, cwp, Ps);
             __syncthreads();
-            BWLA_PSTAMP(5);
             switch (p.tr2) {
                 case 8: stage2_chunk<8>(Zf, n1, n2, Pc, cwp, c0, cw, Xs, amax); break;
                 case 4: stage2_chunk<4>(Zf, n1, n2, Pc, cwp, c0, cw, Xs, amax); break;
@@ -879,297 +765,8 @@ __device__ void rotate_role(const PrologueParams& p, float* smem) {
     finish_token(p, t, C, rank, Xs, slots, amax, rows, a_lo, red_max, &red_sum, true);
 }
 
-// ---------------------------------------------------------------------------------------------
-// T = V x, written as three bf16 terms
-// ---------------------------------------------------------------------------------------------
-// acc += dot of eight bf16 pairs (two packed 128-bit words)
-__device__ __forceinline__ float dot8(float acc, const uint4& v, const uint4& xv) {
-    const uint32_t a[4] = {v.x, v.y, v.z, v.w}, b[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        acc = fmaf(__uint_as_float(a[i] << 16), __uint_as_float(b[i] << 16), acc);
-        acc = fmaf(__uint_as_float(a[i] & 0xFFFF0000u), __uint_as_float(b[i] & 0xFFFF0000u), acc);
-    }
-    return acc;
-}
-
-// One block reduces R rows of V against T tokens (R x T accumulators per thread, threads stride over K).  Few tokens:
-// R = 2, T = 16 (many blocks).  Many tokens: R = T = 8, which reads each operand four times less often from L2.
-template <int R, int T>
-__device__ void lowrank_role(const PrologueParams& p, int b, float* smem) {
-    const int jblocks = p.lr_cols / R;
-    const int jb = b % jblocks;
-    const int64_t t0 = (int64_t)(b / jblocks) * T;
-    if (t0 >= p.M) return;
-    const int j0 = jb * R;
-    const int nt = (int)min((int64_t)T, p.M - t0);
-    float (*red)[R * T] = reinterpret_cast<float (*)[R * T]>(smem);            // [kLrMaxWarps][R * T]
-    const uint4* vs = reinterpret_cast<const uint4*>(smem + kLrMaxWarps * R * T);   // staged rows of V, [R][K / 8]
-    float acc[R][T];
-#pragma unroll
-    for (int j = 0; j < R; ++j)
-#pragma unroll
-        for (int i = 0; i < T; ++i) acc[j][i] = 0.f;
-    const int K = p.K;
-    const int nr = min(R, p.r - j0);                          // rows of V this block really has (<= 0: padding only)
-    const bool vec = ((reinterpret_cast<uintptr_t>(p.V) | reinterpret_cast<uintptr_t>(p.x)) & 15) == 0 && (p.ldx & 7) == 0 && (K & 7) == 0;
-    const bool staged = p.lr_stage && vec && nr > 0;
-    if (staged) {
-        // V is a constant of the layer: in shared memory before the activations exist
-        uint4* dst = reinterpret_cast<uint4*>(smem + kLrMaxWarps * R * T);
-        for (int j = 0; j < R; ++j) {
-            const uint4* src = reinterpret_cast<const uint4*>(p.V + (int64_t)(j0 + min(j, nr - 1)) * K);
-            for (int kc = threadIdx.x; kc < (K >> 3); kc += blockDim.x) dst[j * (K >> 3) + kc] = __ldg(src + kc);
-        }
-    }
-    griddep_launch_dependents();
-    griddep_wait();                                           // x may be the output of the preceding kernel
-    BWLA_PBLOCK(2);
-    if (nr > 0) {
-        const __nv_bfloat16* vrow[R];
-#pragma unroll
-        for (int j = 0; j < R; ++j) vrow[j] = p.V + (int64_t)(j0 + min(j, nr - 1)) * K;
-        const __nv_bfloat16* xt = p.x + t0 * p.ldx;
-        if (vec) {
-            for (int kc = threadIdx.x; kc < (K >> 3); kc += blockDim.x) {
-                uint4 a[R];
-#pragma unroll
-                for (int j = 0; j < R; ++j) a[j] = staged ? vs[j * (K >> 3) + kc] : __ldg(reinterpret_cast<const uint4*>(vrow[j]) + kc);
-#pragma unroll
-                for (int tt = 0; tt < T; ++tt) {
-                    if (tt < nt) {
-                        const uint4 xv = __ldg(reinterpret_cast<const uint4*>(xt + tt * p.ldx) + kc);
-#pragma unroll
-                        for (int j = 0; j < R; ++j) acc[j][tt] = dot8(acc[j][tt], a[j], xv);
-                    }
-                }
-            }
-        } else {
-            for (int k = threadIdx.x; k < K; k += blockDim.x) {
-                float a[R];
-#pragma unroll
-                for (int j = 0; j < R; ++j) a[j] = __bfloat162float(vrow[j][k]);
-#pragma unroll
-                for (int tt = 0; tt < T; ++tt) {
-                    if (tt < nt) {
-                        const float xv = __bfloat162float(xt[tt * p.ldx + k]);
-#pragma unroll
-                        for (int j = 0; j < R; ++j) acc[j][tt] = fmaf(a[j], xv, acc[j][tt]);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < R; ++j)
-            if (j >= nr) {
-#pragma unroll
-                for (int i = 0; i < T; ++i) acc[j][i] = 0.f;
-            }
-    }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int j = 0; j < R; ++j)
-#pragma unroll
-        for (int i = 0; i < T; ++i) {
-            float v = acc[j][i];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-            if (lane == 0) red[warp][j * T + i] = v;
-        }
-    __syncthreads();
-    for (int o = threadIdx.x; o < R * T; o += blockDim.x) {
-        const int j = o / T, i = o % T;
-        if (i < nt) {
-            float s = 0.f;
-            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += red[w][o];
-            // three bf16 terms carry all 24 bits of the fp32 sum
-            const __nv_bfloat16 hi = __float2bfloat16_rn(s);
-            const float r1 = s - __bfloat162float(hi);
-            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-            const int64_t at = (t0 + i) * p.lr_cols + j0 + j;
-            p.Thl[at] = hi;
-            p.Thl[p.M * p.lr_cols + at] = mid;
-            p.Thl[2 * p.M * p.lr_cols + at] = lo;
-        }
-    }
-}
-
-// Few tokens: T for a tile of 16 tokens x 8 columns per block on the warp-level tensor-core path
-// (mma.sync m16n8k16, bf16 in, fp32 accumulate): far fewer instructions than the FMA version, so these blocks do not
-// take issue slots from the rotation blocks they share SMs with.  The warps of the block split K in chunks of 32; a
-// lane reads 16 bytes of two token rows and of one row of V per chunk, and the chunk is contracted by two MMAs whose
-// k order is permuted the same way for both operands (a sum over k does not care).  Partial tiles are added across
-// the warps in shared memory in warp order.
-__device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                                 uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__device__ void lowrank_mma_role(const PrologueParams& p, int b, float* smem) {
-    const int jtiles = p.lr_cols / 8;
-    const int KS = p.lr_ks;
-    const int j0 = (b % jtiles) * 8;
-    const int ks = (b / jtiles) % KS;
-    const int64_t t0 = (int64_t)(b / (jtiles * KS)) * 16;
-    if (t0 >= p.M) return;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int g = lane >> 2, tg = lane & 3;
-    const int K = p.K;
-    griddep_launch_dependents();
-    griddep_wait();                                           // x may be the output of the preceding kernel
-    BWLA_PBLOCK(2);
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    if (j0 < p.r) {
-        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-        const bool row_lo = t0 + g < p.M, row_hi = t0 + g + 8 < p.M, col = j0 + g < p.r;
-        const uint4* xlo = reinterpret_cast<const uint4*>(p.x + (t0 + (row_lo ? g : 0)) * p.ldx) + tg;
-        const uint4* xhi = reinterpret_cast<const uint4*>(p.x + (t0 + (row_hi ? g + 8 : 0)) * p.ldx) + tg;
-        const uint4* vj = reinterpret_cast<const uint4*>(p.V + (int64_t)(j0 + (col ? g : 0)) * K) + tg;
-        const int chunks = K >> 5;
-        const int c_lo = (int)((int64_t)chunks * ks / KS), c_hi = (int)((int64_t)chunks * (ks + 1) / KS);
-#pragma unroll 4
-        for (int c = c_lo + warp; c < c_hi; c += nwarps) {
-            const uint4 a = row_lo ? __ldg(xlo + 4 * c) : zero;
-            const uint4 h = row_hi ? __ldg(xhi + 4 * c) : zero;
-            const uint4 v = col ? __ldg(vj + 4 * c) : zero;
-            mma_bf16_16x8x16(acc, a.x, h.x, a.y, h.y, v.x, v.y);
-            mma_bf16_16x8x16(acc, a.z, h.z, a.w, h.w, v.z, v.w);
-        }
-    }
-    // acc: (token g, columns 2tg, 2tg+1), (token g+8, same columns)
-    float* red = smem;                                        // [nwarps][16 * 8]
-    red[warp * 128 + g * 8 + 2 * tg] = acc[0];
-    red[warp * 128 + g * 8 + 2 * tg + 1] = acc[1];
-    red[warp * 128 + (g + 8) * 8 + 2 * tg] = acc[2];
-    red[warp * 128 + (g + 8) * 8 + 2 * tg + 1] = acc[3];
-    __syncthreads();
-    if (KS > 1) {
-        // Several blocks share this tile of T and split K.  Each leaves its partial tile in the workspace; the last one
-        // to arrive adds them in the order of the K parts (so the result does not depend on who came last).
-        const int tile = (int)(b / (jtiles * KS)) * jtiles + (b % jtiles);
-        float* mine = p.lr_part + ((size_t)tile * KS + ks) * 128;
-        for (int o = threadIdx.x; o < 128; o += blockDim.x) {
-            float s = 0.f;
-            for (int w = 0; w < nwarps; ++w) s += red[w * 128 + o];
-            mine[o] = s;
-        }
-        __threadfence();
-        __syncthreads();
-        __shared__ uint32_t arrived;
-        if (threadIdx.x == 0) arrived = atomicAdd(p.lr_count + tile, 1u);
-        __syncthreads();
-        if (arrived != (uint32_t)(KS - 1)) return;
-        __threadfence();
-        for (int o = threadIdx.x; o < 128; o += blockDim.x) {
-            const int i = o >> 3, j = o & 7;
-            float s = 0.f;
-            for (int k = 0; k < KS; ++k) s += __ldcg(p.lr_part + ((size_t)tile * KS + k) * 128 + o);
-            if (t0 + i < p.M) {
-                const __nv_bfloat16 hi = __float2bfloat16_rn(s);
-                const float r1 = s - __bfloat162float(hi);
-                const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-                const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-                const int64_t at = (t0 + i) * p.lr_cols + j0 + j;
-                p.Thl[at] = hi;
-                p.Thl[p.M * p.lr_cols + at] = mid;
-                p.Thl[2 * p.M * p.lr_cols + at] = lo;
-            }
-        }
-        if (threadIdx.x == 0) p.lr_count[tile] = 0;          // ready for the next call
-        return;
-    }
-    for (int o = threadIdx.x; o < 128; o += blockDim.x) {
-        const int i = o >> 3, j = o & 7;
-        if (t0 + i < p.M) {
-            float s = 0.f;
-            for (int w = 0; w < nwarps; ++w) s += red[w * 128 + o];
-            // three bf16 terms carry all 24 bits of the fp32 sum
-            const __nv_bfloat16 hi = __float2bfloat16_rn(s);
-            const float r1 = s - __bfloat162float(hi);
-            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-            const int64_t at = (t0 + i) * p.lr_cols + j0 + j;
-            p.Thl[at] = hi;
-            p.Thl[p.M * p.lr_cols + at] = mid;
-            p.Thl[2 * p.M * p.lr_cols + at] = lo;
-        }
-    }
-}
-
-// Many tokens: the same on tiles of 16 tokens x all 64 columns, so that x is read once; a lane keeps the eight
-// column tiles' accumulators (32 registers) and reads one row of V per column tile and chunk.
-__device__ void lowrank_mma_wide_role(const PrologueParams& p, int b, float* smem) {
-    const int64_t t0 = (int64_t)b * 16;
-    if (t0 >= p.M) return;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const int g = lane >> 2, tg = lane & 3;
-    const int K = p.K;
-    const int ntiles = p.lr_cols / 8;                         // <= 8
-    griddep_launch_dependents();
-    griddep_wait();                                           // x may be the output of the preceding kernel
-    BWLA_PBLOCK(2);
-    float acc[8][4];
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
-    {
-        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-        const bool row_lo = t0 + g < p.M, row_hi = t0 + g + 8 < p.M;
-        const uint4* xlo = reinterpret_cast<const uint4*>(p.x + (t0 + (row_lo ? g : 0)) * p.ldx) + tg;
-        const uint4* xhi = reinterpret_cast<const uint4*>(p.x + (t0 + (row_hi ? g + 8 : 0)) * p.ldx) + tg;
-        const uint4* vbase = reinterpret_cast<const uint4*>(p.V) + tg;
-        const int chunks = K >> 5;
-#pragma unroll 2
-        for (int c = warp; c < chunks; c += nwarps) {
-            const uint4 a = row_lo ? __ldg(xlo + 4 * c) : zero;
-            const uint4 h = row_hi ? __ldg(xhi + 4 * c) : zero;
-            uint4 v[8];
-#pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                const int j = 8 * nt + g;
-                v[nt] = (nt < ntiles && j < p.r) ? __ldg(vbase + (size_t)j * (K >> 3) + 4 * c) : zero;
-            }
-#pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                mma_bf16_16x8x16(acc[nt], a.x, h.x, a.y, h.y, v[nt].x, v[nt].y);
-                mma_bf16_16x8x16(acc[nt], a.z, h.z, a.w, h.w, v[nt].z, v[nt].w);
-            }
-        }
-    }
-    // partial tiles of the warps, [warp][token 0..15][column 0..63], added in warp order
-    float* red = smem;
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-        float* r = red + warp * 1024 + 8 * nt + 2 * tg;
-        r[g * 64] = acc[nt][0]; r[g * 64 + 1] = acc[nt][1];
-        r[(g + 8) * 64] = acc[nt][2]; r[(g + 8) * 64 + 1] = acc[nt][3];
-    }
-    __syncthreads();
-    for (int o = threadIdx.x; o < 1024; o += blockDim.x) {
-        const int i = o >> 6, j = o & 63;
-        if (t0 + i < p.M && j < p.lr_cols) {
-            float s = 0.f;
-            for (int w = 0; w < nwarps; ++w) s += red[w * 1024 + o];
-            // three bf16 terms carry all 24 bits of the fp32 sum
-            const __nv_bfloat16 hi = __float2bfloat16_rn(s);
-            const float r1 = s - __bfloat162float(hi);
-            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-            const int64_t at = (t0 + i) * p.lr_cols + j;
-            p.Thl[at] = hi;
-            p.Thl[p.M * p.lr_cols + at] = mid;
-            p.Thl[2 * p.M * p.lr_cols + at] = lo;
-        }
-    }
-}
-
 __global__ void prologue_kernel(PrologueParams p) {
     extern __shared__ __align__(16) float smem[];
-    BWLA_PBLOCK(0);
     const int b = (int)blockIdx.x;
     const int lr = p.rot_first ? b : b - p.rot_blocks;        // index among the low-rank blocks (when not a rotation block)
     if (b >= p.rot_first && b < p.rot_first + p.rot_blocks) rotate_role(p, smem);
@@ -1177,7 +774,6 @@ __global__ void prologue_kernel(PrologueParams p) {
     else if (p.lr_wide == 2) lowrank_mma_role(p, lr, smem);
     else if (p.lr_wide == 3) lowrank_mma_wide_role(p, lr, smem);
     else lowrank_role<2, 16>(p, lr, smem);
-    BWLA_PBLOCK(1);
 }
 
 // How many clusters of `c` prologue blocks (threads, dynamic shared memory) the device holds at once; cached.
@@ -1195,7 +791,7 @@ static int clusters_resident(int c, int threads, size_t smem) {
         return 0;
     }
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)(c * 148), 1, 1);
+    cfg.gridDim = dim3((unsigned)(c * (sm_count() > 0 ? sm_count() : 1)), 1, 1);
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cudaLaunchAttribute attr[1];
@@ -1359,7 +955,7 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
             // second wave of clusters would double the latency).
             bool chosen = false;
             for (int c = cmax; c > 1 && !chosen; --c) {
-                if (M * c > 148 || !plan(c)) continue;
+                if (M * c > sm_count() || !plan(c)) continue;
                 if (clusters_resident(c, threads, smem) >= M) { C = c; chosen = true; }
             }
             // Many tokens of a large K: one CTA per token would stage P1 and P2 chunk by chunk for every token.  Clusters

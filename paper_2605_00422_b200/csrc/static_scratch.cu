@@ -44,13 +44,17 @@ extern "C" int bwla_w1ax_linear_static(const void* x_bf16, int64_t M, int64_t K,
                                        const float* P2, int n2, int bits, const uint32_t* packed, const float* alpha,
                                        const float* mu, const void* U_bf16, const void* V_bf16, int r, void* out_bf16,
                                        int64_t N, int64_t ldo, void* stream) {
-    // sizes first: a problem that does not fit is refused before anything touches the GPU
+    // sizes and arguments first: a call that is going to be refused puts nothing on the stream
     const size_t need = bwla_workspace_bytes(M, K, N, r, bits);
     if (need == 0) return BWLA_ERR_INVALID_ARG;
     if (need > (size_t)BWLA_STATIC_SCRATCH_BYTES) return BWLA_ERR_STATIC_SCRATCH;
+    // (the scratch pointer is not known yet; any aligned non-null value passes the workspace check)
+    int st = validate_linear_call(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, packed, alpha, U_bf16, V_bf16, r, out_bf16, N, ldo,
+                                  reinterpret_cast<const void*>((uintptr_t)256), BWLA_STATIC_SCRATCH_BYTES);
+    if (st != BWLA_OK) return st;
     if (M == 0 || N == 0) return BWLA_OK;
     void* scratch = nullptr;
-    int st = static_scratch_address(&scratch);
+    st = static_scratch_address(&scratch);
     if (st != BWLA_OK) return st;
     // The array keeps what the previous call left.  Only the status words have to start at zero (a stale failure
     // flag would make this call skip its work); everything else is written before it is read.

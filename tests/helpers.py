@@ -63,6 +63,35 @@ class DeviceLayer:
             self.packed_host = words_to_host(self.packed)
 
 
+def token_sample(M: int, tile: int = 128) -> list:
+    """Stratified token subset for problems too large for the oracle: every position inside the first tile, the whole
+    last tile, and one (varying) position of every tile in between."""
+    last_start = (M - 1) // tile * tile
+    picked = set(range(min(tile, M))) | set(range(last_start, M))
+    picked |= {i * tile + (i * 37) % tile for i in range(1, last_start // tile)}
+    return sorted(picked)
+
+
+def deinterleave_codes(stored: torch.Tensor) -> torch.Tensor:
+    """Codes as the tensor-core contraction wants them (inside each group of 32 consecutive k, byte 4*j + i holds
+    k = j + 8*i) back in natural order."""
+    M, K = stored.shape
+    return stored.view(M, K // 32, 8, 4).transpose(2, 3).reshape(M, K).contiguous()
+
+
+def fused_call_codes(bwla, ws: torch.Tensor, M: int, shape, bits: int):
+    """The int8 codes (natural order) and scales that bwla_w1ax_linear left in its workspace."""
+    off, nb = bwla.bwla_workspace_section(M, shape.K, shape.N, shape.r, bits, bwla.BWLA_WS_CODES)
+    stored = ws[off:off + nb].view(torch.int8).view(M, shape.K)
+    if bwla.bwla_chosen_path(M, shape.K, shape.N, shape.r, bits) != bwla.BWLA_PATH_SIMPLE:
+        codes = deinterleave_codes(stored)
+    else:
+        codes = stored.clone()
+    off, nb = bwla.bwla_workspace_section(M, shape.K, shape.N, shape.r, bits, bwla.BWLA_WS_SCALES)
+    scales = ws[off:off + nb].view(torch.float32).clone()
+    return codes, scales
+
+
 def summand_magnitude(ref: dict, alpha: np.ndarray) -> np.ndarray:
     """|alpha * s * acc| + |y - alpha * s * acc| of an oracle result: the size of what the output sum adds up."""
     main = alpha.astype(np.float64)[None, :] * ref["scales"].astype(np.float64)[:, None] * ref["acc"].astype(np.float64)
@@ -107,4 +136,5 @@ def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray, mag: np.ndarray = None
     slack = 0.0 if mag is None else 2.0 ** -18 * mag
     ulps = np.maximum(np.abs(got - ref_val) - slack, 0.0) / step
     return {"rel_l2": rel_l2, "max_abs_over_rms": float(np.abs(err).max() / max(rms, 1e-300)),
+            "over_literal_bound": int(np.count_nonzero(np.abs(err) > 1e-2 * rms)),
             "max_bf16_steps": float(ulps.max()), "exact_bf16": float(np.mean(gpu_bits == ref_bits))}

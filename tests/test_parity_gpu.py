@@ -261,6 +261,35 @@ def test_accumulators_stay_exact_when_the_gpu_was_idle_before_the_call(bwla):
         assert np.array_equal(acc.cpu().numpy().astype(np.int64), want)
 
 
+def test_a_set_status_word_is_reported_cleared_and_the_next_call_is_clean(bwla):
+    """The device-timeout path without making any wait run long: a bounded wait that gives up sets the workspace
+    status word, and a call that finds the word set skips its work.  Here the word is set by the test; the call must
+    leave the context usable, bwla_check_status must report and clear the condition, and the next call must match
+    the oracle."""
+    shape = gen.CONFIG_SHAPES[0][0]
+    lay = gen.make_layer(0, shape, 6)
+    xb = gen.make_activations(0, shape, 16)
+    dl = H.DeviceLayer(lay, bwla)
+    xd = H.bf16_to_dev(xb)
+    ws = bwla.new_workspace(16, shape.K, shape.N, shape.r, 6)
+    ws[:4].view(torch.int32)[0] = 1
+    bwla.bwla_w1ax_linear(xd, dl.P1, dl.P2, 6, dl.packed, dl.alpha, dl.U, dl.V, workspace=ws)
+    assert bwla.bwla_check_status(ws) == bwla.BWLA_ERR_DEVICE_TIMEOUT
+    assert bwla.bwla_check_status(ws) == 0                      # reading it cleared it
+    out = bwla.bwla_w1ax_linear(xd, dl.P1, dl.P2, 6, dl.packed, dl.alpha, dl.U, dl.V, workspace=ws)
+    assert bwla.bwla_check_status(ws) == 0
+    ref = oracle.linear(xb, lay.P1, lay.P2, 6, dl.packed_host, lay.alpha, lay.U, lay.V)
+    H.check_output(H.bf16_to_host(out), ref["y"])
+
+
+def test_accumulator_range_guard_of_the_tensor_core_path(bwla):
+    """The tensor core sums -128 * code over the set sign bits; where 128 * K * qmax could leave int32 the shape must
+    go to the simple kernel."""
+    assert bwla.bwla_chosen_path(16, 132096, 1024, 0, 8) == bwla.BWLA_PATH_I8      # 128 * K * 127 < 2^31
+    assert bwla.bwla_chosen_path(16, 132224, 1024, 0, 8) == bwla.BWLA_PATH_SIMPLE  # ... > 2^31
+    assert bwla.bwla_chosen_path(16, 132224, 1024, 0, 6) == bwla.BWLA_PATH_I8      # qmax = 31 leaves room
+
+
 def test_empty_batch_and_argument_errors(bwla):
     shape = gen.small_shape(64, 16, 8, 8, 0)
     lay = gen.make_layer(0, shape, 6)

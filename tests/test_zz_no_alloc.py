@@ -44,3 +44,20 @@ def test_static_scratch_entry_refuses_what_does_not_fit():
     with pytest.raises(bwla.BwlaError) as e:
         bwla.bwla_w1ax_linear_static(x, dl.P1, dl.P2, 6, dl.packed, dl.alpha)
     assert e.value.status == bwla.BWLA_ERR_STATIC_SCRATCH
+
+
+def test_static_scratch_entry_refuses_bad_arguments_before_touching_the_stream():
+    from paper_2605_00422_b200 import bwla
+    shape = gen.small_shape(64, 16, 8, 8, 0)
+    lay = gen.make_layer(0, shape, 6)
+    dl = H.DeviceLayer(lay, bwla)
+    x = H.bf16_to_dev(gen.make_activations(0, shape, 2))
+    with pytest.raises(bwla.BwlaError) as e:
+        bwla.bwla_w1ax_linear_static(x, dl.P1, dl.P2, 5, dl.packed, dl.alpha)                      # bits not in {4,6,8}
+    assert e.value.status == bwla.BWLA_ERR_INVALID_ARG
+    with pytest.raises(bwla.BwlaError) as e:
+        bwla.bwla_w1ax_linear_static(x, dl.P1, dl.P2[:4, :4].contiguous(), 6, dl.packed, dl.alpha)  # K != n1*n2
+    assert e.value.status == bwla.BWLA_ERR_INVALID_ARG
+    out = bwla.bwla_w1ax_linear_static(x, dl.P1, dl.P2, 6, dl.packed, dl.alpha)                    # and a good call still works
+    torch.cuda.synchronize()
+    assert out.shape == (2, 16)
