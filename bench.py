@@ -210,11 +210,16 @@ def run_reference(args):
 # our arm
 # ----------------------------------------------------------------------------------------------
 class Linear:
-    __slots__ = ("shape", "P1", "P2", "packed", "alpha", "U", "V")
+    __slots__ = ("shape", "P1", "P2", "packed", "alpha", "U", "V", "layer")
 
 
-def build_stack(layers: int, device, torch):
-    """Per-layer seeded weights generated on the device (same distributions as the host recipe of the tests)."""
+# the linears of one transformer block that read the same activations go through one grouped call
+GROUPS = (("qkv", (0, 1, 2)), ("o", (3,)), ("gate_up", (4, 5)), ("down", (6,)))
+
+
+def build_stack(layers: int, device, torch, bwla=None):
+    """Per-layer seeded weights generated on the device (same distributions as the host recipe of the tests); with
+    `bwla` every linear also gets its prepared-layer handle (constants put into kernel form once, not per call)."""
     stack = []
     for layer in range(layers):
         row = []
@@ -230,6 +235,7 @@ def build_stack(layers: int, device, torch):
             lin.alpha = torch.exp(-4.0 + 0.3 * torch.randn(sh.N, device=device, generator=g))
             lin.U = (0.01 * torch.randn(sh.N, sh.r, device=device, generator=g)).to(torch.bfloat16)
             lin.V = (0.01 * torch.randn(sh.r, sh.K, device=device, generator=g)).to(torch.bfloat16)
+            lin.layer = bwla.Layer(lin.P1, lin.P2, BITS, lin.packed, lin.alpha, lin.U, lin.V) if bwla is not None else None
             row.append(lin)
         stack.append(row)
     return stack
@@ -244,6 +250,74 @@ def student_t_activations(M: int, K: int, device, torch, seed: int):
     ch = torch.randperm(K, device=device, generator=g)[:8]
     x[:, ch] *= 50.0
     return x.to(torch.bfloat16)
+
+
+def oracle_spot_check(stack, xs, M, bwla, torch, tokens=8):
+    """Outside every timed region: the first layer's seven linears on a few tokens against the CPU oracle, through
+    the same grouped calls the timed step makes.  Returns counts for the JSON line (nothing is asserted here; the
+    parity tests assert)."""
+    import oracle
+    nt = min(tokens, M)
+    rep = {"layer": 0, "tokens": nt, "elements_codes": 0, "near_ties": 0, "code_mismatches": 0,
+           "code_mismatches_outside_window": 0, "outputs": 0, "over_literal_bound": 0, "max_abs_over_rms": 0.0, "rel_l2_max": 0.0}
+    window = oracle.near_tie_window(BITS)
+    for _, idx in GROUPS:
+        lins = [stack[0][i] for i in idx]
+        x = xs[lins[0].shape.K][:nt].contiguous()
+        outs = bwla.bwla_w1ax_linear_group([l.layer for l in lins], x)
+        torch.cuda.synchronize()
+        xb = x.view(torch.int16).cpu().numpy().view(np.uint16)
+        for lin, out in zip(lins, outs):
+            packed = lin.packed.cpu().numpy().view(np.uint32)
+            U = lin.U.view(torch.int16).cpu().numpy().view(np.uint16)
+            V = lin.V.view(torch.int16).cpu().numpy().view(np.uint16)
+            ref = oracle.linear(xb, lin.P1.cpu().numpy(), lin.P2.cpu().numpy(), BITS, packed, lin.alpha.cpu().numpy(), U, V)
+            codes, _, _ = bwla.bwla_layer_rotate_quant(lin.layer, x)
+            q = oracle.quantize(ref["Y"], BITS, "f64")
+            bad = codes.cpu().numpy().astype(np.int32) != q["codes"].astype(np.int32)
+            flagged = q["dist"] <= window
+            got = gen.f32_from_bf16_bits(out.view(torch.int16).cpu().numpy().view(np.uint16)).astype(np.float64)
+            err = np.abs(got - ref["y"])
+            rms = float(np.sqrt(np.mean(ref["y"] ** 2)))
+            rep["elements_codes"] += int(bad.size)
+            rep["near_ties"] += int(flagged.sum())
+            rep["code_mismatches"] += int(bad.sum())
+            rep["code_mismatches_outside_window"] += int((bad & ~flagged).sum())
+            rep["outputs"] += int(err.size)
+            rep["over_literal_bound"] += int(np.count_nonzero(err > 1e-2 * rms))
+            rep["max_abs_over_rms"] = max(rep["max_abs_over_rms"], float(err.max() / rms))
+            rep["rel_l2_max"] = max(rep["rel_l2_max"], float(np.linalg.norm(got - ref["y"]) / np.linalg.norm(ref["y"])))
+    return rep
+
+
+def cublas_bf16_context(shapes, layers, Ms, device, torch, distinct=8, reps=3):
+    """Context only: the same stack as plain bf16 GEMMs (torch.matmul -> cuBLAS), x [M][K] times W^T [K][N] for the 7
+    shapes of every layer.  62 GB of bf16 weights would be needed for 64 distinct layers; `distinct` layers (7.8 GB, far
+    above L2) are cycled instead."""
+    out = {"distinct_layers": distinct, "note": "torch.matmul bf16, weights of %d distinct layers cycled over %d layers" % (distinct, layers)}
+    W = [[torch.randn(sh.N, sh.K, device=device, dtype=torch.bfloat16) for sh in shapes] for _ in range(distinct)]
+    for M in Ms:
+        xs = {sh.K: torch.randn(M, sh.K, device=device, dtype=torch.bfloat16) for sh in shapes}
+        ys = [torch.empty(M, sh.N, device=device, dtype=torch.bfloat16) for sh in shapes]
+
+        def run():
+            for l in range(layers):
+                for i, sh in enumerate(shapes):
+                    torch.matmul(xs[sh.K], W[l % distinct][i].t(), out=ys[i])
+        run()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        flops = layers * sum(2 * M * sh.K * sh.N for sh in shapes)
+        wbytes = layers * sum(2 * sh.K * sh.N for sh in shapes)
+        out[f"M{M}"] = {"ms_per_step": ms, "tflops": flops / (ms * 1e-3) / 1e12, "weight_gb_per_s": wbytes / (ms * 1e-3) / 1e9}
+    del W
+    return out
 
 
 def run_ours(args):
@@ -261,23 +335,24 @@ def run_ours(args):
 
     peaks = measured_peaks()
     shapes = gen.CONFIG_SHAPES[4]
-    stack = build_stack(args.layers, device, torch)
+    stack = build_stack(args.layers, device, torch, bwla)
+    torch.cuda.synchronize()
     Ks = sorted({sh.K for sh in shapes})
-    Ns = sorted({sh.N for sh in shapes})
 
     def make_io(M):
         xs = {K: student_t_activations(M, K, device, torch, 7000 + K + M) for K in Ks}
-        outs = {N: torch.empty(M, N, dtype=torch.bfloat16, device=device) for N in Ns}
-        ws_bytes = max(bwla.bwla_workspace_bytes(M, sh.K, sh.N, sh.r, BITS) for sh in shapes)
+        outs = {sh.name: torch.empty(M, sh.N, dtype=torch.bfloat16, device=device) for sh in shapes}
+        ws_bytes = max(bwla.bwla_group_workspace_bytes([stack[0][i].layer for i in idx], M) for _, idx in GROUPS)
         ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=device)
         return xs, outs, ws
 
     def step(xs, outs, ws, layers=None):
         n = 0
         for row in (stack if layers is None else stack[:layers]):
-            for lin in row:
-                bwla.bwla_w1ax_linear(xs[lin.shape.K], lin.P1, lin.P2, BITS, lin.packed, lin.alpha, lin.U, lin.V,
-                                      out=outs[lin.shape.N], workspace=ws)
+            for _, idx in GROUPS:
+                lins = [row[i] for i in idx]
+                bwla.bwla_w1ax_linear_group([l.layer for l in lins], xs[lins[0].shape.K],
+                                            outs=[outs[l.shape.name] for l in lins], workspace=ws)
                 n += bwla.bwla_last_launch_count()
         return n
 
@@ -335,18 +410,18 @@ def run_ours(args):
 
     # end to end: activations arrive from pinned host memory and the last layer's outputs go back, every step
     h_xs = {K: xs[K].cpu().pin_memory() for K in Ks}
-    h_outs = {N: torch.empty(M, N, dtype=torch.bfloat16).pin_memory() for N in Ns}
+    h_outs = {n: torch.empty_like(o, device="cpu").pin_memory() for n, o in outs.items()}
 
     def e2e_step():
         for K in Ks:
             xs[K].copy_(h_xs[K], non_blocking=True)
         graph.replay()
-        for N in Ns:
-            h_outs[N].copy_(outs[N], non_blocking=True)
+        for n in h_outs:
+            h_outs[n].copy_(outs[n], non_blocking=True)
 
     e2e_ms = timed(e2e_step, args.steps, 3)
     h2d = sum(h_xs[K].numel() * 2 for K in Ks)
-    d2h = sum(h_outs[N].numel() * 2 for N in Ns)
+    d2h = sum(h.numel() * 2 for h in h_outs.values())
     e2e_value = replica_rate(world, step_bytes, args.steps, e2e_ms) / 1e9
 
     prof = kernel_profile(xs, outs, ws)
@@ -361,6 +436,7 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": (k_bytes / k_n) if k_n else None,
                 "algorithmic_bytes_per_step": k_bytes}
     del graph
+    spot = oracle_spot_check(stack, xs, M, bwla, torch) if (rank == 0 and not args.no_cpu_baseline) else None
 
     # the other decode batch sizes of the workload, whole-step only
     decode_other = {}
@@ -392,12 +468,17 @@ def run_ours(args):
         prof_p = kernel_profile(xs_p, outs_p, ws_p, layers=Lp)
         kp_ms, kp_n = prof_p.get("contraction", (0.0, 0))
         k_tops = ops / (kp_ms * 1e-3) / 1e12 if kp_ms > 0 else None
-        i8_peak = 2.0 * peaks["bf16_tflops_sustained"]   # int8 dense = 2 x bf16 (nominal ratio) of the measured bf16 rate
+        # int8 dense = 2 x bf16 (nominal ratio) of the measured bf16 rate; the burst figure is the denominator (the
+        # clocks stay at their maximum in this step), the sustained and the nominal ones are printed beside it
+        i8_peak = 2.0 * peaks["bf16_tflops"]
         prefill = {"metric": "prefill INT8 TOPS (2*M*K*N of the contraction / whole-step time)", "value": tops,
                    "unit": "TOPS", "M": Mp, "layers": Lp, "steps": steps_p, "ms_per_step": ms_p / steps_p, "clocks": clocks_p,
                    "roofline": {"bound": "tensor", "kernel": "umma_w1a_kernel, prefill stack", "achieved": k_tops,
-                                "peak": i8_peak, "peak_source": peaks["source"] + " bf16 sustained x 2 (int8:bf16 nominal ratio)",
+                                "peak": i8_peak, "peak_source": peaks["source"] + " bf16 burst x 2 (int8:bf16 nominal ratio)",
                                 "unit": "TOP/s", "frac": (k_tops / i8_peak) if k_tops else None, "traffic": None,
+                                "frac_of_sustained": (k_tops / (2.0 * peaks["bf16_tflops_sustained"])) if k_tops else None,
+                                "frac_of_nominal_4500": (k_tops / 4500.0) if k_tops else None,
+                                "whole_call_frac_of_nominal_4500": tops / 4500.0,
                                 "launches_per_step": kp_n},
                    "kernel_ms_per_step": {k: round(v[0], 4) for k, v in prof_p.items()},
                    "status": bwla.bwla_check_status(ws_p)}
@@ -422,6 +503,12 @@ def run_ours(args):
                "cores": oracle.num_threads(), "kind": "oracle",
                "sample": f"{reps} pass(es) over one layer (7 linears) at M={M}; {dt:.1f} s"}
 
+    cublas = None
+    if rank == 0 and world == 1 and not args.no_cublas:
+        del stack
+        torch.cuda.empty_cache()
+        cublas = cublas_bf16_context(shapes, args.layers, [M] + ([args.prefill_m] if args.prefill_m > 0 else []), device, torch)
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
@@ -436,6 +523,7 @@ def run_ours(args):
             "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
             "kernel_ms_per_step": {k: round(v[0], 4) for k, v in prof.items()},
             "cpu_baseline": cpu, "decode_other_batches": decode_other, "prefill": prefill, "device_status": status,
+            "parity_spot_check": spot, "cublas_bf16_context": cublas,
         }
         print(json.dumps(line))
     if world > 1:
@@ -454,6 +542,7 @@ def main():
     ap.add_argument("--prefill-m", type=int, default=2048)
     ap.add_argument("--prefill-layers", type=int, default=0, help="layers in the prefill step (0 = all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cublas", action="store_true", help="skip the cuBLAS bf16 context measurement")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -137,6 +137,49 @@ int bwla_w1ax_linear_static(const void* x_bf16, int64_t M, int64_t K, int64_t ld
                             void* out_bf16, int64_t N, int64_t ldo, void* stream);
 
 /*
+ * ---- Prepared layers ------------------------------------------------------------------------------------------
+ * A layer's constants can be put once into the form the kernels read, instead of on every call: the Kronecker
+ * factors P1, P2 (Sec. 3.1) split into bf16 terms and laid out as tensor-core operands.  A bwla_layer is a small
+ * host object that remembers the layer's device pointers (it copies nothing and owns no device memory: the caller
+ * keeps P1 ... V and the `prepared` buffer alive and unchanged until bwla_layer_destroy) and the launch plan.
+ * Calls through a prepared layer compute exactly what bwla_w1ax_linear computes.
+ *
+ *   bwla_layer_prepared_bytes  device bytes `prepared` must have for these sizes (a multiple of 256; never 0 for
+ *                              valid sizes)
+ *   bwla_layer_create          checks the arguments as bwla_w1ax_linear does, launches the preparation on `stream`
+ *                              and returns the handle in *layer (host memory from malloc).  `prepared` must be
+ *                              256-byte aligned.
+ *   bwla_layer_destroy         frees the host object only.
+ */
+typedef struct bwla_layer bwla_layer;
+size_t bwla_layer_prepared_bytes(int64_t K, int64_t N, int n1, int n2, int r);
+int bwla_layer_create(bwla_layer** layer, int64_t K, int64_t N, const float* P1, int n1, const float* P2, int n2,
+                      int bits, const uint32_t* packed, const float* alpha, const float* mu,
+                      const void* U_bf16, const void* V_bf16, int r,
+                      void* prepared, size_t prepared_bytes, void* stream);
+void bwla_layer_destroy(bwla_layer* layer);
+
+/*
+ * Online OKT + per-token quantiser of a prepared layer (what bwla_rotate_quant_act computes; Sec. 3.1, Sec. 4.1).
+ *   codes device int8 [M][K] (natural k order), scales device fp32 [M]
+ *   y_f32 device fp32 [M][K] or NULL: receives the rotated activations Y_t before the quantiser
+ */
+int bwla_layer_rotate_quant(const bwla_layer* layer, const void* x_bf16, int64_t M, int64_t ldx,
+                            int8_t* codes, float* scales, float* y_f32, void* stream);
+
+/*
+ * Several layers that read the same activations (q, k, v of an attention block; gate and up of an MLP) in one
+ * call: x is rotated and quantised for every layer (each has its own P1, P2) by one launch, and the contractions
+ * follow.  All layers must have the same K, n1, n2 and bits; count <= 4.
+ *   outs  host array of `count` device pointers, bf16 [M][ldos[i]];  ldos host array, ldos[i] >= N_i
+ *   workspace: 256-byte aligned device scratch of bwla_group_workspace_bytes; its first 256 bytes must be zero
+ *   before the first call (status words, as for bwla_w1ax_linear; bwla_check_status applies to it)
+ */
+size_t bwla_group_workspace_bytes(const bwla_layer* const* layers, int count, int64_t M);
+int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const void* x_bf16, int64_t M, int64_t ldx,
+                           void* const* outs, const int64_t* ldos, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Contraction + epilogue from given codes (the part of the layer after the quantiser), so that
  * integer accumulators can be compared for identical codes.
  *   codes device int8 [M][K]; scales device fp32 [M]
@@ -175,6 +218,12 @@ int bwla_workspace_section(int64_t M, int64_t K, int64_t N, int r, int bits, int
 /* Force every later call of the calling thread onto one kernel family (benchmarking the non-chosen path,
  * cross-checks); the setting is per thread.  Returns BWLA_ERR_INVALID_ARG for an unknown value. */
 int bwla_force_path(int path);
+
+/* The same for the kernel that evaluates the online OKT + quantiser: BWLA_ROT_AUTO (per shape), BWLA_ROT_SIMT (the
+ * kernel with fp32 FMA tiles, P1/P2 staged in shared memory and warp-shuffle reductions; takes every shape) or
+ * BWLA_ROT_UMMA (the tcgen05 kernel; shapes it does not take still go to the other one). */
+enum { BWLA_ROT_AUTO = 0, BWLA_ROT_SIMT = 1, BWLA_ROT_UMMA = 2 };
+int bwla_force_rotation(int which);
 
 /* The family BWLA_PATH_AUTO resolves to for this problem (no launch). */
 int bwla_chosen_path(int64_t M, int64_t K, int64_t N, int r, int bits);

@@ -24,6 +24,8 @@ BWLA_ERR_DEVICE_TIMEOUT = -5
 BWLA_ERR_STATIC_SCRATCH = -6
 BWLA_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 
+BWLA_ROT_AUTO, BWLA_ROT_SIMT, BWLA_ROT_UMMA = 0, 1, 2
+
 BWLA_PATH_AUTO = 0
 BWLA_PATH_SIMPLE = 1
 BWLA_PATH_BITPLANE = 2
@@ -33,7 +35,8 @@ EXPORTS = [
     "bwla_pack_signs", "bwla_rotate_quant_act", "bwla_workspace_bytes", "bwla_w1ax_linear", "bwla_w1a_gemm_codes",
     "bwla_check_status", "bwla_force_path", "bwla_chosen_path", "bwla_last_launch_count", "bwla_last_cuda_error",
     "bwla_status_string", "bwla_profile_enable", "bwla_profile_collect", "bwla_w1ax_linear_static",
-    "bwla_workspace_section",
+    "bwla_workspace_section", "bwla_force_rotation", "bwla_layer_prepared_bytes", "bwla_layer_create",
+    "bwla_layer_destroy", "bwla_layer_rotate_quant", "bwla_group_workspace_bytes", "bwla_w1ax_linear_group",
 ]
 
 
@@ -63,6 +66,20 @@ def _load() -> C.CDLL:
     lib.bwla_w1ax_linear_static.argtypes = [vp, i64, i64, i64, vp, ci, vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, i64, i64, vp]
     lib.bwla_w1ax_linear_static.restype = ci
     lib.bwla_force_path.argtypes = [ci]
+    lib.bwla_force_rotation.argtypes = [ci]
+    lib.bwla_force_rotation.restype = ci
+    lib.bwla_layer_prepared_bytes.argtypes = [i64, i64, ci, ci, ci]
+    lib.bwla_layer_prepared_bytes.restype = sz
+    lib.bwla_layer_create.argtypes = [C.POINTER(vp), i64, i64, vp, ci, vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, sz, vp]
+    lib.bwla_layer_create.restype = ci
+    lib.bwla_layer_destroy.argtypes = [vp]
+    lib.bwla_layer_destroy.restype = None
+    lib.bwla_layer_rotate_quant.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    lib.bwla_layer_rotate_quant.restype = ci
+    lib.bwla_group_workspace_bytes.argtypes = [C.POINTER(vp), ci, i64]
+    lib.bwla_group_workspace_bytes.restype = sz
+    lib.bwla_w1ax_linear_group.argtypes = [C.POINTER(vp), ci, vp, i64, i64, C.POINTER(vp), C.POINTER(i64), vp, sz, vp]
+    lib.bwla_w1ax_linear_group.restype = ci
     lib.bwla_chosen_path.argtypes = [i64, i64, i64, ci, ci]
     lib.bwla_profile_enable.argtypes = [ci]
     lib.bwla_profile_collect.argtypes = [vp, vp]
@@ -112,6 +129,10 @@ def bwla_last_launch_count() -> int:
 
 def bwla_force_path(path: int) -> None:
     _check(_lib.bwla_force_path(path), "bwla_force_path")
+
+
+def bwla_force_rotation(which: int) -> None:
+    _check(_lib.bwla_force_rotation(which), "bwla_force_rotation")
 
 
 def bwla_chosen_path(M: int, K: int, N: int, r: int, bits: int) -> int:
@@ -214,6 +235,105 @@ def bwla_w1ax_linear_static(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor,
                                       _ptr(out), N, out.stride(0) if M > 0 else N, _stream())
     _check(st, "bwla_w1ax_linear_static")
     return out
+
+
+class Layer:
+    """A prepared layer (bwla_layer_create): keeps the handle, the tensors it points into and the prepared buffer."""
+
+    def __init__(self, P1, P2, bits, packed, alpha, U=None, V=None, mu=None):
+        _need(packed, torch.int32, "packed", 2)
+        _need(alpha, torch.float32, "alpha", 1)
+        _need(P1, torch.float32, "P1", 2)
+        _need(P2, torch.float32, "P2", 2)
+        if not (packed.is_contiguous() and P1.is_contiguous() and P2.is_contiguous()):
+            raise TypeError("packed, P1 and P2 must be contiguous")
+        self.N, self.K = packed.shape[0], packed.shape[1] * 32
+        self.n1, self.n2, self.bits = P1.shape[0], P2.shape[0], bits
+        self.r = 0
+        if U is not None:
+            _need(U, torch.bfloat16, "U", 2)
+            _need(V, torch.bfloat16, "V", 2)
+            self.r = U.shape[1]
+            if not (U.is_contiguous() and V.is_contiguous()) or tuple(V.shape) != (self.r, self.K) or U.shape[0] != self.N:
+                raise TypeError("U must be contiguous [N][r] and V contiguous [r][K]")
+        if mu is not None:
+            _need(mu, torch.float32, "mu", 1)
+        self.tensors = (P1, P2, packed, alpha, U, V, mu)
+        nbytes = int(_lib.bwla_layer_prepared_bytes(self.K, self.N, self.n1, self.n2, self.r))
+        if nbytes == 0:
+            raise BwlaError(BWLA_ERR_INVALID_ARG, "bwla_layer_prepared_bytes")
+        self.prepared = torch.empty(nbytes, dtype=torch.uint8, device=packed.device)
+        self.handle = C.c_void_p()
+        st = _lib.bwla_layer_create(C.byref(self.handle), self.K, self.N, _ptr(P1), self.n1, _ptr(P2), self.n2, bits,
+                                    _ptr(packed), _ptr(alpha), _ptr(mu), _ptr(U), _ptr(V), self.r, _ptr(self.prepared),
+                                    nbytes, _stream())
+        _check(st, "bwla_layer_create")
+
+    def __del__(self):
+        h = getattr(self, "handle", None)
+        if h is not None and h.value:
+            _lib.bwla_layer_destroy(h)
+            self.handle = C.c_void_p()
+
+
+def bwla_layer_prepared_bytes(K: int, N: int, n1: int, n2: int, r: int) -> int:
+    return int(_lib.bwla_layer_prepared_bytes(K, N, n1, n2, r))
+
+
+def bwla_layer_create(P1, P2, bits, packed, alpha, U=None, V=None, mu=None) -> Layer:
+    """Prepares a layer's constants once (launches on the current stream) and returns the handle object."""
+    return Layer(P1, P2, bits, packed, alpha, U, V, mu)
+
+
+def bwla_layer_destroy(layer: Layer) -> None:
+    layer.__del__()
+
+
+def bwla_layer_rotate_quant(layer: Layer, x: torch.Tensor, want_y: bool = False):
+    """(codes int8 [M][K], scales fp32 [M], Y fp32 [M][K] or None) through a prepared layer."""
+    _need(x, torch.bfloat16, "x", 2)
+    M, K = x.shape
+    codes = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    scales = torch.empty((M,), dtype=torch.float32, device=x.device)
+    y = torch.empty((M, K), dtype=torch.float32, device=x.device) if want_y else None
+    st = _lib.bwla_layer_rotate_quant(layer.handle, _ptr(x), M, x.stride(0) if M > 0 else K, _ptr(codes), _ptr(scales),
+                                      _ptr(y), _stream())
+    _check(st, "bwla_layer_rotate_quant")
+    return codes, scales, y
+
+
+def _handles(layers):
+    arr = (C.c_void_p * len(layers))(*[l.handle.value for l in layers])
+    return arr
+
+
+def bwla_group_workspace_bytes(layers, M: int) -> int:
+    return int(_lib.bwla_group_workspace_bytes(_handles(layers), len(layers), M))
+
+
+def new_group_workspace(layers, M: int, device="cuda") -> torch.Tensor:
+    n = bwla_group_workspace_bytes(layers, M)
+    if n == 0:
+        raise ValueError("invalid group")
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def bwla_w1ax_linear_group(layers, x: torch.Tensor, outs=None, workspace: Optional[torch.Tensor] = None):
+    """Layers that share x (q/k/v, gate/up) in one call; returns the list of bf16 outputs [M][N_i]."""
+    _need(x, torch.bfloat16, "x", 2)
+    M, K = x.shape
+    if outs is None:
+        outs = [torch.empty((M, l.N), dtype=torch.bfloat16, device=x.device) for l in layers]
+    for o in outs:
+        _need(o, torch.bfloat16, "out", 2)
+    if workspace is None:
+        workspace = new_group_workspace(layers, M, x.device)
+    optr = (C.c_void_p * len(layers))(*[o.data_ptr() for o in outs])
+    ldos = (C.c_int64 * len(layers))(*[(o.stride(0) if M > 0 else l.N) for o, l in zip(outs, layers)])
+    st = _lib.bwla_w1ax_linear_group(_handles(layers), len(layers), _ptr(x), M, x.stride(0) if M > 0 else K, optr, ldos,
+                                     _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "bwla_w1ax_linear_group")
+    return outs
 
 
 def bwla_w1a_gemm_codes(codes: torch.Tensor, scales: torch.Tensor, bits: int, packed: torch.Tensor,

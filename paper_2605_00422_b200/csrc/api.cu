@@ -1,4 +1,5 @@
 // extern "C" boundary: argument validation, workspace carving and per-shape dispatch.  No compute happens here.
+#include <cstdlib>
 #include <vector>
 
 #include "bwla_common.cuh"
@@ -8,6 +9,7 @@ namespace bwla {
 thread_local int g_last_cuda_error = 0;
 thread_local int g_launch_count = 0;
 static thread_local int g_forced_path = BWLA_PATH_AUTO;   // per calling thread, like the other bookkeeping
+static thread_local int g_forced_rotation = 0;            // 0: per shape; 1: the FMA / warp-level MMA kernel; 2: tcgen05
 
 // ---- optional kernel timing -------------------------------------------------------------------
 struct ProfPair { cudaEvent_t a, b; int kind; };
@@ -70,6 +72,18 @@ static int run_contraction(int path, GemmArgs& g, const int8_t* codes, cudaStrea
 }  // namespace bwla
 
 using namespace bwla;
+
+// What a prepared layer remembers: the caller's device pointers and the plan of the rotation kernel.
+struct bwla_layer {
+    int64_t K, N;
+    int n1, n2, bits, r;
+    const float *P1, *P2, *alpha, *mu;
+    const uint32_t* packed;
+    const void *U, *V;
+    uint8_t* prepared;
+    bool okt;                 // the tcgen05 rotation takes these factor sizes
+    OktGeom geom;
+};
 
 extern "C" {
 
@@ -152,8 +166,19 @@ int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, cons
     int8_t* codes = (int8_t*)(base + ws.codes);
     const int path = resolve_path(M, K, N, r, bits);
 
-    st = launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum,
-                         V_bf16, r, Thl, r > 0 ? (float*)(base + ws.lr_part) : nullptr, (uint32_t*)(base + ws.status), s);
+    OktGeom geom;
+    if (g_forced_rotation != 1 && okt_geometry(n1, n2, &geom) && okt_accepts_x(x_bf16, ldx) && okt_prepared_bytes(geom) <= kOktPreparedMax) {
+        // the Kronecker factors are handed over raw: their bf16 terms go into the workspace first (a prepared layer
+        // does this once instead)
+        st = launch_prepare_okt(geom, P1, P2, base + ws.prep, s);
+        if (st != BWLA_OK) return st;
+        OktProblem pr{(const uint8_t*)(base + ws.prep), codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum, nullptr};
+        OktLowrank lr{V_bf16, r, Thl, r > 0 ? (float*)(base + ws.lr_part) : nullptr, (uint32_t*)(base + ws.status) + kLrCounterWord};
+        st = launch_okt(geom, x_bf16, M, ldx, bits, 1, &pr, &lr, (uint32_t*)(base + ws.status), s);
+    } else {
+        st = launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum,
+                             V_bf16, r, Thl, r > 0 ? (float*)(base + ws.lr_part) : nullptr, (uint32_t*)(base + ws.status), s);
+    }
     if (st != BWLA_OK) return st;
     GemmArgs g{};
     g.scales = scales; g.qsum = qsum; g.M = M; g.K = K; g.N = N; g.bits = bits; g.packed = packed; g.alpha = alpha;
@@ -210,6 +235,142 @@ int bwla_workspace_section(int64_t M, int64_t K, int64_t N, int r, int bits, int
     }
 }
 
+// ---- prepared layers -------------------------------------------------------------------------------------------
+
+size_t bwla_layer_prepared_bytes(int64_t K, int64_t N, int n1, int n2, int r) {
+    if (!valid_rotation_dims(K, n1, n2) || N < 0 || r < 0 || r > 256) return 0;
+    OktGeom g;
+    return okt_geometry(n1, n2, &g) ? align_up(okt_prepared_bytes(g), 256) : 256;
+}
+
+int bwla_layer_create(bwla_layer** layer, int64_t K, int64_t N, const float* P1, int n1, const float* P2, int n2, int bits,
+                      const uint32_t* packed, const float* alpha, const float* mu, const void* U_bf16, const void* V_bf16,
+                      int r, void* prepared, size_t prepared_bytes, void* stream) {
+    g_launch_count = 0;
+    if (!layer) return BWLA_ERR_INVALID_ARG;
+    *layer = nullptr;
+    if (!valid_rotation_dims(K, n1, n2) || N <= 0 || r < 0 || r > 256 || !valid_bits(bits)) return BWLA_ERR_INVALID_ARG;
+    if (!P1 || !P2 || !packed || !alpha || (r > 0 && (!U_bf16 || !V_bf16))) return BWLA_ERR_INVALID_ARG;
+    if (((uintptr_t)P1 & 15) || ((uintptr_t)P2 & 15) || ((uintptr_t)packed & 15)) return BWLA_ERR_INVALID_ARG;
+    const size_t need = bwla_layer_prepared_bytes(K, N, n1, n2, r);
+    if (!prepared || ((uintptr_t)prepared & 255) || prepared_bytes < need) return BWLA_ERR_WORKSPACE;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+    bwla_layer* L = (bwla_layer*)malloc(sizeof(bwla_layer));
+    if (!L) return BWLA_ERR_INVALID_ARG;
+    L->K = K; L->N = N; L->n1 = n1; L->n2 = n2; L->bits = bits; L->r = r;
+    L->P1 = P1; L->P2 = P2; L->packed = packed; L->alpha = alpha; L->mu = mu; L->U = U_bf16; L->V = V_bf16;
+    L->prepared = (uint8_t*)prepared;
+    L->okt = okt_geometry(n1, n2, &L->geom);
+    if (L->okt) {
+        st = launch_prepare_okt(L->geom, P1, P2, prepared, (cudaStream_t)stream);
+        if (st != BWLA_OK) { free(L); return st; }
+    }
+    *layer = L;
+    return BWLA_OK;
+}
+
+void bwla_layer_destroy(bwla_layer* layer) { free(layer); }
+
+int bwla_layer_rotate_quant(const bwla_layer* L, const void* x_bf16, int64_t M, int64_t ldx, int8_t* codes, float* scales,
+                            float* y_f32, void* stream) {
+    g_launch_count = 0;
+    if (!L || M < 0 || ldx < L->K) return BWLA_ERR_INVALID_ARG;
+    if (M == 0) return BWLA_OK;
+    if (!x_bf16 || !codes || !scales || ((uintptr_t)codes & 15)) return BWLA_ERR_INVALID_ARG;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+    if (L->okt && g_forced_rotation != BWLA_ROT_SIMT && okt_accepts_x(x_bf16, ldx)) {
+        OktProblem pr{L->prepared, codes, 0, scales, nullptr, y_f32};
+        return launch_okt(L->geom, x_bf16, M, ldx, L->bits, 1, &pr, nullptr, nullptr, (cudaStream_t)stream);
+    }
+    if (y_f32) return BWLA_ERR_UNSUPPORTED;      // only the tensor-core kernel can hand out Y
+    return launch_prologue(x_bf16, M, L->K, ldx, L->P1, L->n1, L->P2, L->n2, L->bits, codes, 0, scales, nullptr, nullptr, 0,
+                           nullptr, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+static bool valid_group(const bwla_layer* const* layers, int count) {
+    if (!layers || count < 1 || count > kOktMaxProblems) return false;
+    for (int i = 0; i < count; ++i) {
+        if (!layers[i]) return false;
+        if (layers[i]->K != layers[0]->K || layers[i]->n1 != layers[0]->n1 || layers[i]->n2 != layers[0]->n2 ||
+            layers[i]->bits != layers[0]->bits)
+            return false;
+    }
+    return true;
+}
+
+size_t bwla_group_workspace_bytes(const bwla_layer* const* layers, int count, int64_t M) {
+    if (!valid_group(layers, count) || M < 0) return 0;
+    size_t total = 0;
+    for (int i = 0; i < count; ++i) total += workspace_layout(M, layers[i]->K, layers[i]->N, layers[i]->r, layers[i]->bits, false).total;
+    return total;
+}
+
+int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const void* x_bf16, int64_t M, int64_t ldx,
+                           void* const* outs, const int64_t* ldos, void* workspace, size_t workspace_bytes, void* stream) {
+    g_launch_count = 0;
+    if (!valid_group(layers, count) || M < 0 || !outs || !ldos || ldx < layers[0]->K) return BWLA_ERR_INVALID_ARG;
+    for (int i = 0; i < count; ++i)
+        if (ldos[i] < layers[i]->N || (M > 0 && !outs[i])) return BWLA_ERR_INVALID_ARG;
+    if (M == 0) return BWLA_OK;
+    if (!x_bf16) return BWLA_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < bwla_group_workspace_bytes(layers, count, M))
+        return BWLA_ERR_WORKSPACE;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const bwla_layer* L0 = layers[0];
+    char* base = (char*)workspace;
+    uint32_t* status = (uint32_t*)base;                  // the status word of the whole call: the first layer's
+    Workspace ws[kOktMaxProblems];
+    char* wbase[kOktMaxProblems];
+    int path[kOktMaxProblems];
+    size_t off = 0;
+    for (int i = 0; i < count; ++i) {
+        ws[i] = workspace_layout(M, layers[i]->K, layers[i]->N, layers[i]->r, layers[i]->bits, false);
+        wbase[i] = base + off;
+        off += ws[i].total;
+        path[i] = resolve_path(M, layers[i]->K, layers[i]->N, layers[i]->r, layers[i]->bits);
+    }
+    bool okt = g_forced_rotation != BWLA_ROT_SIMT && okt_accepts_x(x_bf16, ldx);
+    for (int i = 0; i < count; ++i) okt = okt && layers[i]->okt;
+    if (okt) {
+        OktProblem pr[kOktMaxProblems];
+        OktLowrank lr[kOktMaxProblems];
+        for (int i = 0; i < count; ++i) {
+            const bwla_layer* L = layers[i];
+            pr[i] = OktProblem{L->prepared, (int8_t*)(wbase[i] + ws[i].codes), path[i] == BWLA_PATH_I8 ? 1 : 0,
+                               (float*)(wbase[i] + ws[i].scales), (int32_t*)(wbase[i] + ws[i].qsum), nullptr};
+            lr[i] = OktLowrank{L->V, L->r, wbase[i] + ws[i].T, L->r > 0 ? (float*)(wbase[i] + ws[i].lr_part) : nullptr,
+                               (uint32_t*)(wbase[i] + ws[i].status) + kLrCounterWord};
+        }
+        st = launch_okt(L0->geom, x_bf16, M, ldx, L0->bits, count, pr, lr, status, s);
+        if (st != BWLA_OK) return st;
+    } else {
+        for (int i = 0; i < count; ++i) {
+            const bwla_layer* L = layers[i];
+            st = launch_prologue(x_bf16, M, L->K, ldx, L->P1, L->n1, L->P2, L->n2, L->bits, (int8_t*)(wbase[i] + ws[i].codes),
+                                 path[i] == BWLA_PATH_I8 ? 1 : 0, (float*)(wbase[i] + ws[i].scales),
+                                 (int32_t*)(wbase[i] + ws[i].qsum), L->V, L->r, wbase[i] + ws[i].T,
+                                 L->r > 0 ? (float*)(wbase[i] + ws[i].lr_part) : nullptr, (uint32_t*)(wbase[i] + ws[i].status), s);
+            if (st != BWLA_OK) return st;
+        }
+    }
+    for (int i = 0; i < count; ++i) {
+        const bwla_layer* L = layers[i];
+        GemmArgs g{};
+        g.scales = (float*)(wbase[i] + ws[i].scales); g.qsum = (int32_t*)(wbase[i] + ws[i].qsum);
+        g.M = M; g.K = L->K; g.N = L->N; g.bits = L->bits; g.packed = L->packed; g.alpha = L->alpha; g.mu = L->mu;
+        g.Thl = L->r > 0 ? wbase[i] + ws[i].T : nullptr; g.U = L->U; g.r = L->r; g.out = outs[i]; g.ldo = ldos[i];
+        g.acc_debug = nullptr; g.status = status;
+        st = run_contraction(path[i], g, (int8_t*)(wbase[i] + ws[i].codes), s);
+        if (st != BWLA_OK) return st;
+    }
+    return BWLA_OK;
+}
+
 int bwla_check_status(void* workspace, void* stream) {
     if (!workspace) return BWLA_ERR_INVALID_ARG;
     uint32_t host[4] = {0, 0, 0, 0};
@@ -227,6 +388,12 @@ int bwla_check_status(void* workspace, void* stream) {
 int bwla_force_path(int path) {
     if (path < BWLA_PATH_AUTO || path > BWLA_PATH_I8) return BWLA_ERR_INVALID_ARG;
     g_forced_path = path;
+    return BWLA_OK;
+}
+
+int bwla_force_rotation(int which) {
+    if (which < BWLA_ROT_AUTO || which > BWLA_ROT_UMMA) return BWLA_ERR_INVALID_ARG;
+    g_forced_rotation = which;
     return BWLA_OK;
 }
 

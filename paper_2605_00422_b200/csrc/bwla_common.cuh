@@ -84,10 +84,14 @@ constexpr int kLrCounterWord = 4;
 __host__ __device__ inline int lowrank_cols(int r) { return r > kLowrankPad ? (r + 1) / 2 * 2 : kLowrankPad; }
 
 struct Workspace {
-    size_t status, scales, qsum, T, lr_part, codes, total;
+    size_t status, scales, qsum, T, lr_part, codes, prep, total;
 };
 
-inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bits) {
+// Room for the prepared Kronecker factors of one call (bf16 terms of P2^T and P1^T for the largest factor sizes the
+// tensor-core rotation takes): calls that are handed raw P1, P2 prepare them into the workspace every time.
+constexpr size_t kOktPreparedMax = 640 * 1024;
+
+inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bits, bool with_prepared = true) {
     Workspace w{};
     size_t off = 0;
     w.status = off; off += kStatusBytes;
@@ -97,6 +101,7 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     w.T = off;      off += align_up((size_t)M * lr_cols * 6, 256);     // bf16 [3][M][cols]
     w.lr_part = off; off += r > 0 ? align_up((size_t)kLrKSplitMax * 16 * lr_cols * 4, 256) : 0;   // fp32 [KS][16][cols]
     w.codes = off;  off += align_up((size_t)M * (size_t)K, 256);
+    w.prep = off;   off += with_prepared ? kOktPreparedMax : 0;
     (void)N; (void)bits;
     w.total = off;
     return w;
@@ -123,6 +128,40 @@ int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ld
 int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1, const float* P2, int n2,
                     int bits, int8_t* codes, int codes_layout, float* scales, int32_t* qsum, const void* V, int r,
                     void* Thl, float* lr_part, uint32_t* status, cudaStream_t stream);
+
+// ---- tcgen05 version of the rotation + quantiser (okt_umma.cu) ----
+// Geometry of the kernel for one pair of Kronecker factor sizes; computed on the host, passed to the kernels by value.
+struct OktGeom {
+    int n1, n2, K;
+    int n1p, n2p;           // n1, n2 rounded up to 16: columns of Z^T / Y^T, contraction depth of the first stage
+    int atom2, atom1;       // bytes of one K-atom row (the swizzle span) of operands contracted over b / over a
+    int dt_count, dt_rows;  // tiles of the rows d of P2^T (= tensor-memory lanes) and rows per tile (a multiple of 8)
+    int cs_count, cs_cols;  // slabs of the rows c of P1^T (= output columns) and columns per slab (a multiple of 16)
+    int p2t_bytes, p1t_bytes, x_bytes;      // one tile of P2^T terms, one slab of P1^T terms, one token's X tile
+    int p1t_off, x_off, stage_off, bar_off; // shared-memory offsets (P2^T tile at 0)
+    int stage_bytes;                        // room for one token's codes when one CTA owns the whole token, else 0
+    int tmem_cols, smem_bytes;
+};
+constexpr int kOktMaxProblems = 4;          // linears that share one x and are rotated by one launch
+struct OktProblem {
+    const uint8_t* prepared;    // bf16 terms of P2^T tiles and P1^T slabs (launch_prepare_okt)
+    int8_t* codes;              // [M][K]
+    int codes_layout;           // 0: natural k order; 1: the interleaved order of the tensor-core contraction
+    float* scales;              // [M]
+    int32_t* qsum;              // [M][kQsumParts] or NULL
+    float* y_debug;             // [M][K] fp32 rotated activations before the quantiser, or NULL
+};
+struct OktLowrank { const void* V; int r; void* Thl; float* lr_part; uint32_t* lr_count; };   // V == NULL: no T = V x blocks
+// false when the factor sizes are outside what the kernel takes (n2 a multiple of 8 up to 256, n1 up to 192, ...)
+bool okt_geometry(int n1, int n2, OktGeom* out);
+// false when x cannot be read by tiled TMA loads (16-byte aligned base, row stride a multiple of 8 elements)
+bool okt_accepts_x(const void* x, int64_t ldx);
+size_t okt_prepared_bytes(const OktGeom& g);
+int launch_prepare_okt(const OktGeom& g, const float* P1, const float* P2, void* prepared, cudaStream_t stream);
+// One launch for up to kOktMaxProblems linears that read the same x: rotation + quantiser for each, and the T = V x
+// blocks of those with a low-rank branch.
+int launch_okt(const OktGeom& g, const void* x, int64_t M, int64_t ldx, int bits, int n_problems,
+               const OktProblem* problems, const OktLowrank* lowrank, uint32_t* status, cudaStream_t stream);
 
 // qsum[t][0] = sum_k codes[t][k] (the other parts zero); optionally rewrites natural-order codes into the interleaved order.
 int launch_prepare_codes(const int8_t* codes, int64_t M, int64_t K, int8_t* codes_interleaved, int32_t* qsum,

@@ -36,6 +36,8 @@
 
 #include "bwla_common.cuh"
 #include "umma_ptx.cuh"
+#include "umma_wait.cuh"
+#include "tensor_map.cuh"
 
 namespace bwla {
 
@@ -45,9 +47,6 @@ constexpr int kRowsPerCta = 128;
 constexpr int kUnitK = 1024;             // weights per row in one packed-word stage (128 bytes)
 constexpr int kBlockK = 128;             // K per code sub-block / per tensor-memory A stage
 constexpr int kFirstExpander = 192;      // warps 0, 1: TMA; warps 2..5: MMA issue; warps 6..: expand + epilogue
-constexpr uint32_t kParkNs = 4000;          // longest a single poll of a barrier may park its thread
-constexpr uint32_t kWaitLimit = 1u << 15;   // polls per wait before giving up (about a tenth of a second when nothing arrives)
-
 struct UmmaParams {
     int M, N, K;
     int total_units, splits;
@@ -98,41 +97,6 @@ struct UmmaCfg {
     static_assert(AS >= 2 * EW, "tensor memory: no room for the expanded-weight ring");
     static_assert(N_TOK * kRowsPerCta * 2 <= u_off, "output tile does not fit the stage memory");
 };
-
-__device__ __forceinline__ void give_up(uint32_t* status, volatile int* abort_flag, uint32_t where) {
-    if (status) {
-        atomicExch(status, 1u);
-        status[1] = where;
-        status[2] = blockIdx.x | (blockIdx.y << 16);
-    }
-    *abort_flag = 1;
-}
-
-__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    // Each poll may park the thread for up to kParkNs while the phase is open: a warp that spun on the barrier would
-    // take issue slots from the expander warps that share its scheduler.
-    // a phase that is already complete is seen by the non-blocking probe in a fraction of the time try_wait takes
-    if (mbar_test_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        if (mbar_try_wait_parked(bar, parity, kParkNs)) return true;
-        if (*abort_flag) return false;
-    }
-    return false;
-}
-
-// A whole warp waits on a barrier and leaves the call converged, as the .sync.aligned tcgen05 instructions that follow
-// such a wait require (lanes that each ran their own polling loop may come out of it at different times, and a
-// warp-wide tensor-memory store issued by part of a warp lands late): every lane polls, the warp goes on when all saw
-// the phase complete.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    if (__all_sync(0xFFFFFFFFu, mbar_test_wait(bar, parity))) return true;
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        const bool done = mbar_try_wait_parked(bar, parity, kParkNs);
-        if (__all_sync(0xFFFFFFFFu, done)) return true;
-        if (*abort_flag) return false;
-    }
-    return false;
-}
 
 // One output value from its two accumulators (mu_sc is zero when the layer has no row shift).
 __device__ __forceinline__ float finish_value(int32_t d, float l, float alpha_sc, float mu_sc, int32_t qs) {
@@ -214,6 +178,8 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         // ---------------- packed sign words: HBM -> shared memory (independent of the preceding kernel) ----------------
         if (elect_one()) {
             tma_prefetch_desc(&w_map);
+            // every sign word is read once per call: it should not push codes, constants and kernel code out of the L2
+            const uint64_t stream_once = l2_policy_evict_first();
             int ws = 0; uint32_t wph = 0;
             for (int u = unit_begin; u < unit_end && !*abort_flag; ++u) {
                 // A stage that is not free yet is released by the expansion, which in the end waits for the preceding
@@ -223,7 +189,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     if (!wait_or_abort(&w_empty[ws], wph ^ 1, abort_flag)) { give_up(p.status, abort_flag, 0x10); break; }
                 }
                 mbar_expect_tx(&w_full[ws], L::w_bytes);
-                tma_load_2d(wbuf + ws * L::w_bytes, &w_map, u * (kUnitK / 32), n0, &w_full[ws]);
+                tma_load_2d_hint(wbuf + ws * L::w_bytes, &w_map, u * (kUnitK / 32), n0, &w_full[ws], stream_once);
                 if (++ws == WS) { ws = 0; wph ^= 1; }
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);   // let copies in flight land
@@ -565,36 +531,6 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
 // -------------------------------------------------------------------------------------------------
 // host side
 // -------------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-
-// rank 2 or 3; dims/box innermost first; strides in bytes for dimensions 1..rank-1
-static int make_map(CUtensorMap* map, CUtensorMapDataType dt, int rank, const void* base, const uint64_t* dims,
-                    const uint64_t* strides, const uint32_t* box, CUtensorMapSwizzle sw, CUtensorMapL2promotion promo) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return BWLA_ERR_CUDA;
-    cuuint64_t d[3]; cuuint64_t s[2]; cuuint32_t b[3]; cuuint32_t estr[3] = {1, 1, 1};
-    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; }
-    for (int i = 0; i + 1 < rank; ++i) s[i] = strides[i];
-    CUresult r = fn(map, dt, (cuuint32_t)rank, const_cast<void*>(base), d, s, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                    promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)r; return BWLA_ERR_CUDA; }
-    return BWLA_OK;
-}
-
 template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS, int EW>
 static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUtensorMap& tm, const UmmaParams& p,
                          dim3 grid, cudaStream_t s) {

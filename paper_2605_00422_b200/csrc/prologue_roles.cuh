@@ -5,6 +5,8 @@
 
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "bwla_common.cuh"
 #include "umma_ptx.cuh"
 
@@ -230,6 +232,11 @@ static __device__ void lowrank_mma_role(const PrologueParams& p, int b, float* s
         const uint4* vj = reinterpret_cast<const uint4*>(p.V + (int64_t)(j0 + (col ? g : 0)) * K) + tg;
         const int chunks = K >> 5;
         const int c_lo = (int)((int64_t)chunks * ks / KS), c_hi = (int)((int64_t)chunks * (ks + 1) / KS);
+        // The tensor core adds each group of 16 products into the accumulator with truncation; over the hundreds of
+        // steps of a large K that bias would reach 1e-5 of the sum.  Every four chunks the accumulator is added into a
+        // running fp32 sum with an ordinary rounded addition and starts from zero again.
+        float run[4] = {0.f, 0.f, 0.f, 0.f};
+        int since = 0;
 #pragma unroll 4
         for (int c = c_lo + warp; c < c_hi; c += nwarps) {
             const uint4 a = row_lo ? __ldg(xlo + 4 * c) : zero;
@@ -237,7 +244,14 @@ static __device__ void lowrank_mma_role(const PrologueParams& p, int b, float* s
             const uint4 v = col ? __ldg(vj + 4 * c) : zero;
             mma_bf16_16x8x16(acc, a.x, h.x, a.y, h.y, v.x, v.y);
             mma_bf16_16x8x16(acc, a.z, h.z, a.w, h.w, v.z, v.w);
+            if (++since == 4) {
+                since = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { run[i] += acc[i]; acc[i] = 0.f; }
+            }
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] += run[i];
     }
     // acc: (token g, columns 2tg, 2tg+1), (token g+8, same columns)
     float* red = smem;                                        // [nwarps][16 * 8]
@@ -310,11 +324,12 @@ static __device__ void lowrank_mma_wide_role(const PrologueParams& p, int b, flo
     const int ntiles = p.lr_cols / 8;                         // <= 8
     griddep_launch_dependents();
     griddep_wait();                                           // x may be the output of the preceding kernel
-    float acc[8][4];
+    float acc[8][4], run[8][4];
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+        for (int i = 0; i < 4; ++i) { acc[nt][i] = 0.f; run[nt][i] = 0.f; }
+    int since = 0;
     {
         const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
         const bool row_lo = t0 + g < p.M, row_hi = t0 + g + 8 < p.M;
@@ -337,7 +352,19 @@ static __device__ void lowrank_mma_wide_role(const PrologueParams& p, int b, flo
                 mma_bf16_16x8x16(acc[nt], a.x, h.x, a.y, h.y, v[nt].x, v[nt].y);
                 mma_bf16_16x8x16(acc[nt], a.z, h.z, a.w, h.w, v[nt].z, v[nt].w);
             }
+            // short in-core sums only (see lowrank_mma_role): every four chunks into a rounded running sum
+            if (++since == 4) {
+                since = 0;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) { run[nt][i] += acc[nt][i]; acc[nt][i] = 0.f; }
+            }
         }
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[nt][i] += run[nt][i];
     }
     // partial tiles of the warps, [warp][token 0..15][column 0..63], added in warp order
     float* red = smem;
@@ -364,6 +391,35 @@ static __device__ void lowrank_mma_wide_role(const PrologueParams& p, int b, flo
             p.Thl[2 * p.M * p.lr_cols + at] = lo;
         }
     }
+}
+
+// Host side: chooses the kind of low-rank blocks for the problem in p (x, M, K, ldx, V, r, lr_cols, Thl set), fills the
+// lr_* fields and returns the number of blocks; *smem receives the dynamic shared memory one such block needs.
+// lr_part / lr_count (either may be NULL): workspace for blocks that share a tile of T and split K.
+inline int plan_lowrank(PrologueParams& p, float* lr_part, uint32_t* lr_count, size_t smem_limit, size_t* smem) {
+    const int64_t M = p.M;
+    const int K = p.K;
+    // few tokens: the tensor-core version (needs 16-byte rows); many tokens: tiles that re-read little
+    const bool rows16 = ((reinterpret_cast<uintptr_t>(p.x) | reinterpret_cast<uintptr_t>(p.V)) & 15) == 0 && p.ldx % 8 == 0 &&
+                        K % 32 == 0 && p.lr_cols % 8 == 0;
+    // (the wide tiles read x once but need enough token tiles to fill the device: 16 tokens x 64 columns per block)
+    p.lr_wide = rows16 ? ((M >= 1024 && p.lr_cols == 64) ? 3 : 2) : ((M >= 64 && p.lr_cols % 8 == 0) ? 1 : 0);
+    int blocks = p.lr_wide == 1 ? (p.lr_cols / 8) * (int)((M + 7) / 8)
+               : p.lr_wide == 2 ? (p.lr_cols / 8) * (int)((M + 15) / 16)
+               : p.lr_wide == 3 ? (int)((M + 15) / 16) : (p.lr_cols / 2) * (int)((M + 15) / 16);
+    // One tile of 16 tokens and a large K: eight blocks would stream all of V (cold: from HBM) through eight SMs and
+    // become the longest part of the launch; more blocks take a part of K each.
+    p.lr_ks = 1; p.lr_part = lr_part; p.lr_count = lr_count;
+    if (p.lr_wide == 2 && M <= 16 && lr_part && lr_count && p.lr_cols / 8 <= 8) {
+        const int ksplit = (int)std::min<int64_t>(kLrKSplitMax, (K >> 5) / 100);
+        if (ksplit > 1) { p.lr_ks = ksplit; blocks *= ksplit; }
+    }
+    // shared memory of a low-rank block: per-warp partial sums, and its rows of V when those are staged (few tokens)
+    const size_t red_bytes = (size_t)kLrMaxWarps * 4 * (p.lr_wide == 3 ? 1024 : p.lr_wide == 2 ? 128 : 64);
+    const size_t stage_bytes = (size_t)2 * (size_t)K * 2;
+    p.lr_stage = (p.lr_wide == 0 && red_bytes + stage_bytes <= smem_limit) ? 1 : 0;
+    *smem = red_bytes + (p.lr_stage ? stage_bytes : 0);
+    return blocks;
 }
 
 }  // namespace bwla

@@ -982,26 +982,9 @@ int launch_prologue(const void* x, int64_t M, int64_t K, int64_t ldx, const floa
     }
     int lr_blocks = 0;
     if (r > 0 && Thl) {
-        // few tokens: the tensor-core version (needs 16-byte rows); many tokens: FMA tiles that re-read little
-        const bool rows16 = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(V)) & 15) == 0 && ldx % 8 == 0 &&
-                            K % 32 == 0 && p.lr_cols % 8 == 0;
-        // (the wide tiles read x once but need enough token tiles to fill the device: 16 tokens x 64 columns per block)
-        p.lr_wide = rows16 ? ((M >= 1024 && p.lr_cols == 64) ? 3 : 2) : ((M >= 64 && p.lr_cols % 8 == 0) ? 1 : 0);
-        lr_blocks = p.lr_wide == 1 ? (p.lr_cols / 8) * (int)((M + 7) / 8)
-                  : p.lr_wide == 2 ? (p.lr_cols / 8) * (int)((M + 15) / 16)
-                  : p.lr_wide == 3 ? (int)((M + 15) / 16) : (p.lr_cols / 2) * (int)((M + 15) / 16);
-        // One tile of 16 tokens and a large K: eight blocks would stream all of V (cold: from HBM) through eight SMs and
-        // become the longest part of the launch; more blocks take a part of K each.
-        p.lr_ks = 1; p.lr_part = lr_part; p.lr_count = status ? status + kLrCounterWord : nullptr;
-        if (p.lr_wide == 2 && M <= 16 && lr_part && status && p.lr_cols / 8 <= 8) {
-            const int ksplit = (int)std::min<int64_t>(kLrKSplitMax, (K >> 5) / 100);
-            if (ksplit > 1) { p.lr_ks = ksplit; lr_blocks *= ksplit; }
-        }
-        // shared memory of a low-rank block: per-warp partial sums, and its rows of V when those are staged (few tokens)
-        const size_t red_bytes = (size_t)kLrMaxWarps * 4 * (p.lr_wide == 3 ? 1024 : p.lr_wide == 2 ? 128 : 64);
-        const size_t stage_bytes = (size_t)2 * (size_t)K * 2;
-        p.lr_stage = (p.lr_wide == 0 && red_bytes + stage_bytes <= (size_t)kPrologueSmemFloats * 4) ? 1 : 0;
-        smem = std::max(smem, red_bytes + (p.lr_stage ? stage_bytes : 0));
+        size_t lr_smem = 0;
+        lr_blocks = plan_lowrank(p, lr_part, status ? status + kLrCounterWord : nullptr, kPrologueSmemFloats * 4, &lr_smem);
+        smem = std::max(smem, lr_smem);
     }
     // A block with this much shared memory leaves no room on its SM for a block of the next kernel of the stream.  Let
     // in early, that kernel would crowd onto the SMs this one leaves free and stay there; so it is let in late, when

@@ -9,7 +9,10 @@ Tolerances (all stated here, used by every parity test):
     n1 + n2 = 320 terms; sqrt(320) * 2^-24 ~ 1e-6 of the row's scale).
   * bf16 output: relative L2 error <= 2e-3 (asserted for outputs of >= 1024 elements); every element within
     1e-2 * rms(y) + 2^-8 * |y| of the fp64 oracle value (a correctly rounded bf16 is already up to 2^-9 * |y| away,
-    so the absolute bound alone cannot hold for elements several rms large).
+    so the absolute bound alone cannot hold for elements several rms large).  A code that legitimately differs from
+    the oracle's by one step at a near-tie moves every output of its token by alpha[n] * s_t; for a token with f such
+    codes the bound grows by f * alpha[n] * s_t and the token is left out of the L2 figure (with 4-bit codes and
+    heavy-tailed activations one step is already more than 1e-2 * rms(y)).
   * where the test also knows the two summands of the output (the scaled integer term and the low-rank term):
     every element within 1 bf16 step of the correctly rounded oracle value plus 2^-18 * (|term1| + |term2|).  The
     kernel evaluates the sum in fp32 (tensor-core fp32 accumulation for the low-rank term), whose error is
@@ -118,16 +121,25 @@ def check_codes(gpu_codes: np.ndarray, gpu_scales: np.ndarray, Y: np.ndarray, bi
             "scale_rel_err": float(scale_err.max())}
 
 
-def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray, mag: np.ndarray = None) -> dict:
+def code_step_slack(gpu_codes: np.ndarray, ref: dict, alpha: np.ndarray, mu: np.ndarray = None) -> np.ndarray:
+    """[tokens][N]: how far the outputs of a token may move because f of its codes differ from the oracle's by one step
+    (check_codes has verified that these are near-ties): f * (|alpha[n]| + |mu[n]|) * s_t."""
+    flips = np.count_nonzero(gpu_codes.astype(np.int32) != ref["codes"].astype(np.int32), axis=1).astype(np.float64)
+    per_row = np.abs(alpha.astype(np.float64)) + (0.0 if mu is None else np.abs(mu.astype(np.float64)))
+    return flips[:, None] * per_row[None, :] * ref["scales"].astype(np.float64)[:, None]
+
+
+def check_output(gpu_bits: np.ndarray, y_ref: np.ndarray, mag: np.ndarray = None, step_slack: np.ndarray = None) -> dict:
     got = gen.f32_from_bf16_bits(gpu_bits).astype(np.float64)
     err = got - y_ref
-    rel_l2 = float(np.linalg.norm(err) / max(np.linalg.norm(y_ref), 1e-300))
+    same_codes = np.ones(y_ref.shape[0], bool) if step_slack is None else (step_slack.max(axis=1) == 0)
+    rel_l2 = float(np.linalg.norm(err[same_codes]) / max(np.linalg.norm(y_ref[same_codes]), 1e-300))
     rms = float(np.sqrt(np.mean(y_ref ** 2)))
     # the L2 figure is a statistic of the output rounding (a single correctly rounded bf16 can be 2^-8 away),
     # so it is only asserted where there are enough elements for it to mean something
-    if y_ref.size >= 1024:
+    if y_ref[same_codes].size >= 1024:
         assert rel_l2 <= 2e-3, f"relative L2 error {rel_l2:.3e} > 2e-3"
-    bound = 1e-2 * rms + 2.0 ** -8 * np.abs(y_ref)
+    bound = 1e-2 * rms + 2.0 ** -8 * np.abs(y_ref) + (0.0 if step_slack is None else step_slack)
     assert np.all(np.abs(err) <= bound), f"max |err| {np.abs(err).max():.3e} exceeds 1e-2*rms + 2^-8*|y|"
     # distance to the correctly rounded value, in bf16 steps of the reference
     ref_bits = oracle.bf16_round(y_ref)

@@ -125,7 +125,9 @@ def _run_layer_case(bwla, cfg, shape, M, bits, with_mu=False, direct_words=False
         out = bwla.bwla_w1ax_linear(xd, dl.P1, dl.P2, bits, dl.packed, dl.alpha, dl.U, dl.V, dl.mu, workspace=ws)
         assert bwla.bwla_check_status(ws) == 0
         ref = oracle.linear(xb, lay.P1, lay.P2, bits, dl.packed_host, lay.alpha, lay.U, lay.V, lay.mu)
-        rep = H.check_output(H.bf16_to_host(out), ref["y"])
+        gpu_codes, gpu_scales = H.fused_call_codes(bwla, ws, M, shape, bits)
+        H.check_codes(gpu_codes.cpu().numpy(), gpu_scales.cpu().numpy(), ref["Y"], bits)
+        rep = H.check_output(H.bf16_to_host(out), ref["y"], step_slack=H.code_step_slack(gpu_codes.cpu().numpy(), ref, lay.alpha, lay.mu))
         # identical codes in -> identical integer accumulators out
         codes = torch.from_numpy(ref["codes"]).cuda()
         scales = torch.from_numpy(ref["scales"]).cuda()

@@ -8,8 +8,9 @@ configuration the benchmark times.  What is compared on the sample:
   * the codes and scales the fused call itself left in its workspace (read back through bwla_workspace_section),
     against the fp64 quantiser of the oracle's rotation, with the near-tie rule of tests/helpers.py;
   * the bf16 outputs against the oracle's fp64 layer output;
-  * the int32 accumulators of bwla_w1a_gemm_codes for identical codes (the ones the GPU produced, so that no full-size
-    oracle rotation is needed), bit-exact against the oracle's integer contraction.
+  * the int32 accumulators of bwla_w1a_gemm_codes for identical codes, bit-exact against the oracle's integer
+    contraction, and the outputs for identical codes within one bf16 step: the sampled tokens are given the oracle's
+    codes and scales, the other tokens seeded random codes (they only have to keep every tile of the launch busy).
 """
 import numpy as np
 import pytest
@@ -43,19 +44,27 @@ def run_sampled_case(bwla, cfg, shape, M, bits, check_acc=True):
     ref = oracle.linear(xb[sample], lay.P1, lay.P2, bits, dl.packed_host, lay.alpha, lay.U, lay.V)
     rep = H.check_codes(gpu_codes[sample].cpu().numpy(), gpu_scales[sample].cpu().numpy(), ref["Y"], bits)
     assert rep["mismatches"] <= max(4, rep["elements"] // 10000)
-    rep.update(H.check_output(H.bf16_to_host(out[sample]), ref["y"]))
+    slack = H.code_step_slack(gpu_codes[sample].cpu().numpy(), ref, lay.alpha)
+    rep.update(H.check_output(H.bf16_to_host(out[sample]), ref["y"], step_slack=slack))
     assert rep["rel_l2"] <= 2e-3
 
     if check_acc:
-        # identical codes in (the GPU's own, all M tokens) -> identical integer accumulators out
-        _, acc = bwla.bwla_w1a_gemm_codes(gpu_codes, gpu_scales, bits, dl.packed, dl.alpha, xd, dl.U, dl.V,
-                                          want_out=False, want_acc=True, workspace=ws)
+        # identical codes in -> identical integer accumulators out
+        qmax = (1 << (bits - 1)) - 1
+        rng = np.random.default_rng([422, cfg, shape.shape_id, M, bits])
+        codes_in = rng.integers(-qmax, qmax + 1, size=(M, shape.K), dtype=np.int8)
+        scales_in = np.ones(M, np.float32)
+        codes_in[sample] = ref["codes"]
+        scales_in[sample] = ref["scales"]
+        out2, acc = bwla.bwla_w1a_gemm_codes(torch.from_numpy(codes_in).cuda(), torch.from_numpy(scales_in).cuda(), bits,
+                                             dl.packed, dl.alpha, xd, dl.U, dl.V, want_acc=True, workspace=ws)
         assert bwla.bwla_check_status(ws) == 0
-        want = oracle.gemm(gpu_codes[sample].cpu().numpy(), dl.packed_host)
         got = acc[sample].cpu().numpy().astype(np.int64)
-        wrong = np.argwhere(got != want)
+        wrong = np.argwhere(got != ref["acc"])
         assert wrong.size == 0, (f"{len(wrong)} integer accumulators differ; first (sampled token, row) pairs "
                                  f"{wrong[:8].tolist()}")
+        rep2 = H.check_output(H.bf16_to_host(out2[sample]), ref["y"], H.summand_magnitude(ref, lay.alpha))
+        assert rep2["max_bf16_steps"] <= 1.0 + 1e-9
     print(f"\n[{shape.name} M={M} b={bits}] sampled tokens {len(sample)}, near ties {rep['near_ties']}, code mismatches "
           f"{rep['mismatches']} of {rep['elements']}, rel L2 {rep['rel_l2']:.2e}, max |err|/rms {rep['max_abs_over_rms']:.3f}, "
           f"elements over the literal 1e-2*rms bound {rep['over_literal_bound']}")

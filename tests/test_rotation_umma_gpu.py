@@ -1,0 +1,118 @@
+"""The tcgen05 rotation + quantiser (reached through prepared layers) against the CPU oracle, in three stages:
+
+  (A) the rotated activations the kernel hands out, against the oracle's fp64 rotation: the error must stay below
+      the code window, 1e-6 of the token's full scale (the tensor core adds each group of 16 products into its fp32
+      accumulator with truncation, about half an ulp of the running sum per step, so the error grows with n1 + n2:
+      2e-7 at 32 x 32, 7e-7 at 160 x 160);
+  (B) the oracle's quantiser with the fp32 decision rule, applied to the GPU's own Y, must give the GPU's codes and
+      scales exactly: the quantiser itself is then tested bit for bit, whatever the rotation error;
+  (C) the GPU codes against the fp64 definition, with the near-tie rule of tests/helpers.py.
+
+And grouped calls (several layers reading one x) against the oracle layer by layer.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_00422_b200 import inputs as gen
+from tests import helpers as H
+from tests.test_parity_gpu import ROT_CASES
+
+pytestmark = pytest.mark.gpu
+
+# factor sizes the tensor-core kernel takes: n2 a multiple of 8
+UMMA_CASES = [c for c in ROT_CASES if c[1] % 8 == 0] + [
+    (64, 80, 300, 6),     # more tokens than SMs: CTAs stay and take tokens in turn
+    (64, 64, 130, 6),     # LLaMA hidden size
+    (86, 128, 160, 6),
+    (160, 160, 75, 6),    # clusters of four per token, two tokens per cluster and a ragged tail
+    (16, 16, 7, 8),       # a single 16-column chunk
+    (192, 8, 3, 6),       # the widest n1, the narrowest n2
+    (40, 200, 5, 4),      # two lane tiles of 104 + 96 rows
+]
+
+
+@pytest.fixture(scope="module")
+def bwla():
+    from paper_2605_00422_b200 import bwla as b
+    b.bwla_force_path(b.BWLA_PATH_AUTO)
+    b.bwla_force_rotation(b.BWLA_ROT_AUTO)
+    return b
+
+
+def _layer_for_rotation(bwla, lay, shape, bits):
+    packed = torch.zeros((8, shape.K // 32), dtype=torch.int32, device="cuda")
+    alpha = torch.ones(8, device="cuda")
+    return bwla.Layer(H.f32_to_dev(lay.P1), H.f32_to_dev(lay.P2), bits, packed, alpha)
+
+
+@pytest.mark.parametrize("n1,n2,M,bits", UMMA_CASES)
+def test_rotation_stages_a_b_c(bwla, n1, n2, M, bits):
+    K = n1 * n2
+    shape = gen.small_shape(K, 32, n1, n2, 0, shape_id=n1 * 1000 + n2)
+    lay = gen.make_layer(0, shape, bits)
+    xb = gen.make_activations(0, shape, M)
+    L = _layer_for_rotation(bwla, lay, shape, bits)
+    codes, scales, y = bwla.bwla_layer_rotate_quant(L, H.bf16_to_dev(xb), want_y=True)
+    torch.cuda.synchronize()
+    codes, scales, y = codes.cpu().numpy(), scales.cpu().numpy(), y.cpu().numpy().astype(np.float64)
+    Y = oracle.rotate(xb, lay.P1, lay.P2)
+    # (A)
+    amax = np.abs(Y).max(axis=1, keepdims=True)
+    amax[amax == 0] = 1.0
+    rel = float((np.abs(y - Y) / amax).max())
+    assert rel <= 9e-7, f"rotation error {rel:.2e} of the token's full scale"
+    # (B)
+    q32 = oracle.quantize(y, bits, "f32")
+    assert np.array_equal(q32["codes"], codes)
+    assert np.array_equal(q32["scales"], scales)
+    # (C)
+    rep = H.check_codes(codes, scales, Y, bits)
+    assert rep["mismatches"] <= max(4, rep["elements"] // 10000)
+    print(f"\n[{n1}x{n2} M={M} b={bits}] rotation error {rel:.2e} of full scale, near ties {rep['near_ties']}, "
+          f"mismatches {rep['mismatches']} of {rep['elements']}")
+
+
+def test_forced_rotation_kernels_agree_with_the_oracle(bwla):
+    """Both rotation kernels behind bwla_w1ax_linear on the same problem."""
+    shape = gen.CONFIG_SHAPES[2][1]
+    lay = gen.make_layer(2, shape, 6, direct_words=True)
+    xb = gen.make_activations(2, shape, 24)
+    dl = H.DeviceLayer(lay, bwla)
+    ref = oracle.linear(xb, lay.P1, lay.P2, 6, dl.packed_host, lay.alpha, lay.U, lay.V)
+    try:
+        for which in (bwla.BWLA_ROT_SIMT, bwla.BWLA_ROT_UMMA):
+            bwla.bwla_force_rotation(which)
+            ws = bwla.new_workspace(24, shape.K, shape.N, shape.r, 6)
+            out = bwla.bwla_w1ax_linear(H.bf16_to_dev(xb), dl.P1, dl.P2, 6, dl.packed, dl.alpha, dl.U, dl.V, workspace=ws)
+            assert bwla.bwla_check_status(ws) == 0
+            c, s = H.fused_call_codes(bwla, ws, 24, shape, 6)
+            H.check_codes(c.cpu().numpy(), s.cpu().numpy(), ref["Y"], 6)
+            H.check_output(H.bf16_to_host(out), ref["y"])
+    finally:
+        bwla.bwla_force_rotation(bwla.BWLA_ROT_AUTO)
+
+
+@pytest.mark.parametrize("idxs,M", [((0, 1, 2), 16), ((4, 5), 16), ((4, 5), 1), ((0, 1, 2), 200), ((6,), 16), ((3,), 5)])
+def test_grouped_layers_match_the_oracle_layer_by_layer(bwla, idxs, M):
+    """q/k/v and gate/up of the Qwen3-32B shapes through bwla_w1ax_linear_group: one x, one rotation launch, every
+    layer's output against its own oracle result."""
+    bits = 6
+    shapes = [gen.CONFIG_SHAPES[2][i] for i in idxs]
+    lays = [gen.make_layer(2, sh, bits, direct_words=True) for sh in shapes]
+    xb = gen.make_activations(2, shapes[0], M)
+    dls = [H.DeviceLayer(l, bwla) for l in lays]
+    layers = [bwla.Layer(d.P1, d.P2, bits, d.packed, d.alpha, d.U, d.V) for d in dls]
+    ws = bwla.new_group_workspace(layers, M)
+    outs = bwla.bwla_w1ax_linear_group(layers, H.bf16_to_dev(xb), workspace=ws)
+    assert bwla.bwla_check_status(ws) == 0
+    for lay, d, out in zip(lays, dls, outs):
+        ref = oracle.linear(xb, lay.P1, lay.P2, bits, d.packed_host, lay.alpha, lay.U, lay.V)
+        rep = H.check_output(H.bf16_to_host(out), ref["y"])
+        assert rep["rel_l2"] <= 2e-3
+    # the same call again on the same workspace gives the same bits
+    outs2 = bwla.bwla_w1ax_linear_group(layers, H.bf16_to_dev(xb), workspace=ws)
+    assert bwla.bwla_check_status(ws) == 0
+    for a, b in zip(outs, outs2):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
