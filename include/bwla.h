@@ -44,10 +44,14 @@ enum {
 
 /* Kernel families the layer can run its contraction on (see bwla_force_path). */
 enum {
-    BWLA_PATH_AUTO = 0,       /* per-shape choice */
-    BWLA_PATH_SIMPLE = 1,     /* one-thread-per-output CUDA kernel: slow, used as an on-device cross-check */
-    BWLA_PATH_BITPLANE = 2,   /* activation bit-planes x packed weight bits, AND-popcount tensor-core MMA */
-    BWLA_PATH_I8 = 3          /* weights expanded to +-1 int8 in shared memory, tcgen05 kind::i8 into TMEM */
+    BWLA_PATH_AUTO = 0,       /* per-shape choice from measurement: I8 wherever it can run; up to four tokens of a shape
+                                 it cannot take go to BITPLANE, the rest to SIMPLE */
+    BWLA_PATH_SIMPLE = 1,     /* one-warp-per-output-row CUDA kernel: slow, the on-device cross-check and the path of
+                                 shapes the other two do not take */
+    BWLA_PATH_BITPLANE = 2,   /* up to four tokens: two's-complement bit-planes of the codes against the packed sign
+                                 words with and + popc on the integer pipes; the weights are never expanded */
+    BWLA_PATH_I8 = 3          /* sign words expanded to int8 in tensor memory, tcgen05 kind::i8 with int32 accumulators
+                                 in tensor memory; needs K % 128 == 0 and r <= 64 */
 };
 
 #define BWLA_DTYPE_F32 0

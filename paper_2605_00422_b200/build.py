@@ -48,5 +48,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_microbench() -> str:
+    """The instruction-rate probes (a stand-alone program; not part of the library)."""
+    src = os.path.join(_HERE, "microbench", "issue_rates.cu")
+    out = os.path.join(_HERE, "microbench", "issue_rates")
+    nvcc = os.environ.get("NVCC", "nvcc")
+    res = subprocess.run([nvcc, "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a", "-o", out, src],
+                         capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed building the microbenchmark")
+    return out
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--microbench" in sys.argv:
+        print(build_microbench())
+    else:
+        print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))

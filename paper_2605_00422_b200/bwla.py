@@ -271,7 +271,7 @@ class Layer:
 
     def __del__(self):
         h = getattr(self, "handle", None)
-        if h is not None and h.value:
+        if h is not None and h.value and _lib is not None:      # (_lib is None while the interpreter shuts down)
             _lib.bwla_layer_destroy(h)
             self.handle = C.c_void_p()
 

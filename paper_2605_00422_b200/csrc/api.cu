@@ -54,11 +54,21 @@ static bool valid_rotation_dims(int64_t K, int n1, int n2) {
     return K > 0 && K % 32 == 0 && K <= 25600 && n1 > 0 && n2 > 0 && (int64_t)n1 * n2 == K;
 }
 
+// Up to how many tokens the bit-plane kernel is chosen over the tcgen05 one (0: never).  Measured per launch with cold
+// weights on the Qwen3-32B and LLaMA-2-7B shapes (profiles/contraction_paths_small_m.md): at these sizes both kernels are
+// bound by fixed latencies rather than by the stream of sign words, the tensor-core kernel's are the shorter ones
+// (21 against 27 microseconds for 5120 -> 25600 at one token), and the bit-plane kernel's time grows with tokens x bits.
+// It is therefore only taken where the tensor-core kernel cannot run (K not a multiple of 128, rank above 64).
+static int bitplane_max_tokens(int64_t K, int64_t N, int bits) {
+    (void)N; (void)bits;
+    return (K % 128 != 0) ? 4 : 0;
+}
+
 // Which kernel family runs the contraction.  A forced family that cannot take the shape falls back to the simple one.
 static int resolve_path(int64_t M, int64_t K, int64_t N, int r, int bits) {
     int path = g_forced_path;
-    if (path == BWLA_PATH_AUTO) path = BWLA_PATH_I8;
-    if (path == BWLA_PATH_BITPLANE) path = BWLA_PATH_SIMPLE;   // not built yet
+    if (path == BWLA_PATH_AUTO) path = (M <= bitplane_max_tokens(K, N, bits) && bitplane_supports(M, K, N, r, bits)) ? BWLA_PATH_BITPLANE : BWLA_PATH_I8;
+    if (path == BWLA_PATH_BITPLANE && !bitplane_supports(M, K, N, r, bits)) path = BWLA_PATH_SIMPLE;
     if (path == BWLA_PATH_I8 && !umma_supports(M, K, N, r, bits)) path = BWLA_PATH_SIMPLE;
     return path;
 }
@@ -66,6 +76,7 @@ static int resolve_path(int64_t M, int64_t K, int64_t N, int r, int bits) {
 static int run_contraction(int path, GemmArgs& g, const int8_t* codes, cudaStream_t stream) {
     if (path == BWLA_PATH_I8) return launch_gemm_umma(g, codes, stream);
     g.codes = codes;
+    if (path == BWLA_PATH_BITPLANE) return launch_gemm_bitplane(g, stream);
     return launch_gemm_simple(g, stream);
 }
 

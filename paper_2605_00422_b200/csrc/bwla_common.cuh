@@ -187,6 +187,11 @@ struct GemmArgs {
 
 int launch_gemm_simple(const GemmArgs& a, cudaStream_t stream);
 
+// One to four tokens: activation bit-planes against the packed sign words (and + popc), weights never expanded.
+// a.codes in natural k order.
+bool bitplane_supports(int64_t M, int64_t K, int64_t N, int r, int bits);
+int launch_gemm_bitplane(const GemmArgs& a, cudaStream_t stream);
+
 // tcgen05 path with the fused epilogue.  codes_interleaved: int8 [M][K] in the interleaved order.
 bool umma_supports(int64_t M, int64_t K, int64_t N, int r, int bits);
 int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream);

@@ -86,7 +86,7 @@ def fused_call_codes(bwla, ws: torch.Tensor, M: int, shape, bits: int):
     """The int8 codes (natural order) and scales that bwla_w1ax_linear left in its workspace."""
     off, nb = bwla.bwla_workspace_section(M, shape.K, shape.N, shape.r, bits, bwla.BWLA_WS_CODES)
     stored = ws[off:off + nb].view(torch.int8).view(M, shape.K)
-    if bwla.bwla_chosen_path(M, shape.K, shape.N, shape.r, bits) != bwla.BWLA_PATH_SIMPLE:
+    if bwla.bwla_chosen_path(M, shape.K, shape.N, shape.r, bits) == bwla.BWLA_PATH_I8:
         codes = deinterleave_codes(stored)
     else:
         codes = stored.clone()

@@ -201,6 +201,33 @@ def test_small_and_ragged_shapes(bwla, K, N, n1, n2, r, M, bits):
     _run_layer_case(bwla, 0, gen.small_shape(K, N, n1, n2, r, shape_id=K + N), M, bits)
 
 
+@pytest.mark.parametrize("K,N,n1,n2,r,M,bits", [
+    (96, 40, 8, 12, 4, 3, 6),        # three sign words per row, ragged rows, three tokens in a four-token kernel
+    (32, 1, 4, 8, 0, 1, 8),          # one word, one row, one token
+    (1024, 300, 32, 32, 16, 4, 4),
+    (2048, 129, 32, 64, 0, 2, 8),
+    (1056, 77, 32, 33, 8, 2, 6),     # 33 sign words: the second chunk of word positions holds a single word
+])
+def test_bitplane_path_small_and_ragged_shapes(bwla, K, N, n1, n2, r, M, bits):
+    _run_layer_case(bwla, 0, gen.small_shape(K, N, n1, n2, r, shape_id=K + N), M, bits, with_mu=(r == 16),
+                    path=bwla.BWLA_PATH_BITPLANE)
+
+
+@pytest.mark.parametrize("idx,M,bits", [(4, 1, 6), (6, 1, 6), (1, 2, 6), (6, 4, 4), (0, 1, 8), (6, 2, 8)])
+def test_bitplane_path_qwen32b_shapes(bwla, idx, M, bits):
+    _run_layer_case(bwla, 2, gen.CONFIG_SHAPES[2][idx], M, bits, direct_words=True, path=bwla.BWLA_PATH_BITPLANE)
+
+
+def test_path_choice_follows_the_measured_table(bwla):
+    """The tcgen05 kernel wherever it can run (it was measured faster at every token count on the workload shapes); a few
+    tokens of a shape it cannot take go to the bit-plane kernel, more tokens to the simple one."""
+    sh = gen.CONFIG_SHAPES[2][4]
+    for M in (1, 16, 2048):
+        assert bwla.bwla_chosen_path(M, sh.K, sh.N, sh.r, 6) == bwla.BWLA_PATH_I8
+    assert bwla.bwla_chosen_path(2, 1056, 77, 8, 6) == bwla.BWLA_PATH_BITPLANE      # K % 128 != 0
+    assert bwla.bwla_chosen_path(9, 1056, 77, 8, 6) == bwla.BWLA_PATH_SIMPLE
+
+
 def test_mu_shift_is_applied(bwla):
     _run_layer_case(bwla, 0, gen.small_shape(512, 96, 16, 32, 8, shape_id=5), 6, 6, with_mu=True)
 
