@@ -206,6 +206,95 @@ void bwla_oracle_quantize(const double* Y, int64_t M, int64_t K, int bits, int d
     }
 }
 
+/*
+ * Per-token asymmetric INT-b quantiser: Sec. 4.1 states "per-token asymmetric quantization for activations" and gives no
+ * constants; this is the common definition with an integer zero point, and zero kept representable:
+ *   lo = min(0, min_k y_k), hi = max(0, max_k y_k), L = 2^b - 1 levels above code 0
+ *   lo == hi (an all-zero row): scale = 1, zero = 0, all codes 0
+ *   scale = (hi - lo) / L;  zero = clamp(rne(-lo / scale), 0, L);  u_k = clamp(rne(y_k / scale) + zero, 0, L)
+ *   the value a code stands for is scale * (u_k - zero); y = 0 maps to u = zero exactly.
+ *   decision == 1 (the precision a float kernel decides in): range = fl32(hi - lo), inv = fl32(L / range),
+ *   scale = fl32(range / L), zero = rne(fl32(-lo * inv)), u_k = rne(fl32(y_k * inv)) + zero.
+ * dist[k] (optional) = distance of y_k / scale to the nearest rounding boundary; dist_zero[t] the same for -lo / scale.
+ */
+void bwla_oracle_quantize_asym(const double* Y, int64_t M, int64_t K, int bits, int decision,
+                               uint8_t* codes, float* scales, int32_t* zeros, double* dist, double* dist_zero) {
+    const double L = (double)((1 << bits) - 1);
+    for (int64_t t = 0; t < M; ++t) {
+        const double* y = Y + t * K;
+        double lo = 0.0, hi = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            if (y[k] < lo) lo = y[k];
+            if (y[k] > hi) hi = y[k];
+        }
+        if (lo == hi) {
+            scales[t] = 1.0f;
+            zeros[t] = 0;
+            if (dist_zero) dist_zero[t] = 0.5;
+            for (int64_t k = 0; k < K; ++k) {
+                codes[t * K + k] = 0;
+                if (dist) dist[t * K + k] = 0.5;
+            }
+            continue;
+        }
+        double scale64 = (hi - lo) / L;
+        volatile float lo32 = (float)lo, hi32 = (float)hi;
+        volatile float range32 = hi32 - lo32;
+        volatile float inv32 = (float)L / range32;
+        volatile float scale32 = range32 / (float)L;
+        double tz;
+        if (decision) {
+            volatile float zf = -lo32 * inv32;
+            tz = (double)zf;
+        } else {
+            tz = -lo / scale64;
+        }
+        double z = round_half_even(tz);
+        if (z < 0.0) z = 0.0;
+        if (z > L) z = L;
+        zeros[t] = (int32_t)z;
+        scales[t] = decision ? scale32 : (float)scale64;
+        if (dist_zero) dist_zero[t] = fabs(tz - (floor(tz) + 0.5));
+        for (int64_t k = 0; k < K; ++k) {
+            double tk;
+            if (decision) {
+                volatile float yf = (float)y[k];
+                volatile float tf = yf * inv32;
+                tk = (double)tf;
+            } else {
+                tk = y[k] / scale64;
+            }
+            double u = round_half_even(tk) + z;
+            if (u < 0.0) u = 0.0;
+            if (u > L) u = L;
+            codes[t * K + k] = (uint8_t)u;
+            if (dist) dist[t * K + k] = fabs(tk - (floor(tk) + 0.5));
+        }
+    }
+}
+
+/* acc[t][n] = sum_k s[n][k] * (u[t][k] - zero[t]) for unsigned codes with a per-token zero point, int64; and
+ * rsum[t] = sum_k (u[t][k] - zero[t]). */
+void bwla_oracle_gemm_asym(const uint8_t* codes, const int32_t* zeros, const uint32_t* packed, int64_t M, int64_t N,
+                           int64_t K, int64_t* acc, int64_t* rsum) {
+    int64_t words = K / 32;
+    for (int64_t t = 0; t < M; ++t) {
+        int64_t s = 0;
+        for (int64_t k = 0; k < K; ++k) s += (int64_t)codes[t * K + k] - (int64_t)zeros[t];
+        rsum[t] = s;
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t t = 0; t < M; ++t) {
+            int64_t a = 0;
+            for (int64_t k = 0; k < K; ++k) {
+                int64_t r = (int64_t)codes[t * K + k] - (int64_t)zeros[t];
+                a += ((packed[n * words + (k >> 5)] >> (k & 31)) & 1u) ? r : -r;
+            }
+            acc[t * N + n] = a;
+        }
+}
+
 /* acc[t][n] = sum_k s[n][k] * q[t][k], s = +-1 read from the packed bits, int64. */
 void bwla_oracle_gemm(const int8_t* codes, const uint32_t* packed, int64_t M, int64_t N, int64_t K,
                       int64_t* acc) {

@@ -20,6 +20,7 @@ _LIB = os.path.join(_HERE, "libbwla_oracle.so")
 __all__ = [
     "build", "num_threads", "kron_factor", "row_stats", "pack_signs", "pack_signs_bf16", "unpack_signs",
     "rotate", "quantize", "gemm", "lowrank", "epilogue", "linear", "bf16_round", "near_tie_window",
+    "quantize_asym", "gemm_asym", "linear_asym", "near_tie_window_asym",
 ]
 
 
@@ -123,6 +124,53 @@ def quantize(Y: np.ndarray, bits: int, decision: str = "f64") -> Dict[str, np.nd
     _L().bwla_oracle_quantize(_p(Y), i64(M), i64(K), C.c_int(bits), C.c_int(1 if decision == "f32" else 0),
                               _p(codes), _p(scales), _p(dist), _p(qsum))
     return {"codes": codes, "scales": scales, "dist": dist, "qsum": qsum}
+
+
+def quantize_asym(Y: np.ndarray, bits: int, decision: str = "f64") -> Dict[str, np.ndarray]:
+    """Per-token asymmetric quantiser (Sec. 4.1): unsigned codes u in [0, 2^b - 1], scale and integer zero point per token;
+    a code stands for scale * (u - zero)."""
+    Y = _c(Y, np.float64)
+    M, K = Y.shape
+    codes = np.empty((M, K), np.uint8)
+    scales = np.empty(M, np.float32)
+    zeros = np.empty(M, np.int32)
+    dist = np.empty((M, K), np.float64)
+    dist_zero = np.empty(M, np.float64)
+    _L().bwla_oracle_quantize_asym(_p(Y), i64(M), i64(K), C.c_int(bits), C.c_int(1 if decision == "f32" else 0),
+                                   _p(codes), _p(scales), _p(zeros), _p(dist), _p(dist_zero))
+    return {"codes": codes, "scales": scales, "zeros": zeros, "dist": dist, "dist_zero": dist_zero}
+
+
+def near_tie_window_asym(bits: int) -> float:
+    """As near_tie_window for the asymmetric quantiser, whose full scale is 2^b - 1 code units."""
+    return 1e-6 * float((1 << bits) - 1)
+
+
+def gemm_asym(codes: np.ndarray, zeros: np.ndarray, packed: np.ndarray):
+    """(acc, rsum): acc[t][n] = sum_k sign[n][k] * (u[t][k] - zero[t]); rsum[t] = sum_k (u[t][k] - zero[t])."""
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.int32)
+    packed = _c(packed, np.uint32)
+    M, K = codes.shape
+    N = packed.shape[0]
+    assert packed.shape[1] * 32 == K
+    acc = np.empty((M, N), np.int64)
+    rsum = np.empty(M, np.int64)
+    _L().bwla_oracle_gemm_asym(_p(codes), _p(zeros), _p(packed), i64(M), i64(N), i64(K), _p(acc), _p(rsum))
+    return acc, rsum
+
+
+def linear_asym(x_bits, P1, P2, bits, packed, alpha, U_bits=None, V_bits=None, mu=None,
+                decision: str = "f64") -> Dict[str, np.ndarray]:
+    """The whole layer with the per-token asymmetric activation quantiser, step by step:
+    y[t][n] = alpha[n] * s_t * sum_k sign[n][k] * (u[t][k] - z_t) + U (V x_t) [+ mu[n] * s_t * sum_k (u[t][k] - z_t)]."""
+    Y = rotate(x_bits, P1, P2)
+    q = quantize_asym(Y, bits, decision)
+    acc, rsum = gemm_asym(q["codes"], q["zeros"], packed)
+    L = lowrank(x_bits, U_bits, V_bits) if U_bits is not None else None
+    y, yb = epilogue(acc, q["scales"], alpha, L, mu, rsum if mu is not None else None)
+    return {"y": y, "y_bf16": yb, "Y": Y, "codes": q["codes"], "scales": q["scales"], "zeros": q["zeros"], "acc": acc,
+            "dist": q["dist"], "dist_zero": q["dist_zero"]}
 
 
 def near_tie_window(bits: int) -> float:

@@ -26,7 +26,7 @@
 // to four slabs of the output columns c (when the terms of P1^T and P2^T do not fit shared memory together); the CTAs
 // of a cluster repeat stage A and share nothing but the absmax.
 // Warp 0 moves data (constants once, then one token's X per step), warp 1 allocates tensor memory and issues the
-// MMAs, warps 2..9 are the ALU warps of stages B and D (two per tensor-memory lane quarter, taking 16-column chunks
+// MMAs, warps 2..13 are the ALU warps of stages B and D (three per tensor-memory lane quarter, taking 16-column chunks
 // in turn).  Clusters stay on their SMs and take tokens in turn, so the constants are fetched once per CTA.
 //
 // The blocks behind the rotation CTAs evaluate T = V x for the PSP low-rank branch (prologue_roles.cuh).
@@ -45,8 +45,11 @@
 
 namespace bwla {
 
-constexpr int kOktThreads = 320;          // warp 0: copies; warp 1: MMA issue; warps 2..9: ALU
-constexpr int kOktAluThreads = 256;
+constexpr int kOktAluPerQuarter = 3;      // ALU warps per tensor-memory lane quarter
+constexpr int kOktAluWarps = 4 * kOktAluPerQuarter;
+constexpr int kOktAluThreads = 32 * kOktAluWarps;
+constexpr int kOktThreads = 64 + kOktAluThreads;   // warp 0: copies; warp 1: MMA issue; then the ALU warps
+constexpr int kOktChunksD = 3;            // 16-column chunks of Y^T one ALU warp holds in registers: 128 columns / 16 / 3 warps, rounded up
 constexpr int kOktMaxSmem = 231424;       // the 227 KB a block may have, less 1 KB for the static shared memory of the roles
 constexpr int kOktBarBytes = 1024;        // barriers and small per-CTA state behind the operand tiles
 
@@ -87,6 +90,7 @@ bool okt_geometry(int n1, int n2, OktGeom* out) {
         if (cs > 1 && (cs - 1) * per >= chunks) continue;       // a slab would be empty
         g.cs_count = cs;
         g.cs_cols = per * 16;
+        if (g.cs_cols > 16 * kOktAluPerQuarter * kOktChunksD) continue;   // the ALU warps keep their chunks of Y^T in registers
         g.p1t_bytes = 3 * g.cs_cols * g.n1p * 2;
         g.p1t_off = round_up_int(g.p2t_bytes, 1024);
         g.x_off = g.p1t_off + round_up_int(g.p1t_bytes, 1024);
@@ -189,16 +193,6 @@ __device__ __forceinline__ void split3_pair(float a, float b, uint32_t& h, uint3
     l = cvt_bf16x2(ra - __uint_as_float(m << 16), rb - __uint_as_float(m & 0xFFFF0000u));
 }
 
-// Byte store into shared memory under a predicate (no branch).
-__device__ __forceinline__ void st_shared_u8_if(uint32_t addr, int value, bool pred) {
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "setp.ne.b32 P, %2, 0;\n\t"
-        "@P st.shared.u8 [%0], %1;\n\t}"
-        ::"r"(addr), "r"(value), "r"((uint32_t)pred)
-        : "memory");
-}
-
 // ALU warps only: barrier 1 with an OR over a predicate (a uniform decision for all of them), barrier 2 plain.
 __device__ __forceinline__ bool alu_barrier_or(bool pred) {
     uint32_t out;
@@ -236,7 +230,6 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
         const int rel = lb - p.lr_begin[i];
         if (lp.lr_wide == 1) lowrank_role<8, 8>(lp, rel, fsmem);
         else if (lp.lr_wide == 2) lowrank_mma_role(lp, rel, fsmem);
-        else if (lp.lr_wide == 3) lowrank_mma_wide_role(lp, rel, fsmem);
         else lowrank_role<2, 16>(lp, rel, fsmem);
         return;
     }
@@ -258,8 +251,8 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 10) + 1;
     int* red_sum = reinterpret_cast<int*>(bars + 11);
-    float* red_max = reinterpret_cast<float*>(bars + 12);        // [8]
-    float* slots = red_max + 8;                                  // [2][8] absmax per CTA of the cluster, by token parity
+    float* red_max = reinterpret_cast<float*>(bars + 12);        // [kOktAluWarps]
+    float* slots = red_max + kOktAluWarps;                       // [2][8] absmax per CTA of the cluster, by token parity
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = g.dt_count * g.cs_count;
@@ -353,7 +346,9 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             const uint32_t blk_a = (uint32_t)(g.dt_rows * g.atom2) >> 4;      // one (term, K-atom) block of P2^T
             const uint32_t blk_x = (uint32_t)(n1p * g.atom2) >> 4;            // one K-atom block of X
             const uint32_t blk_p1 = (uint32_t)(g.cs_cols * g.atom1) >> 4;     // one (term, K-atom) block of P1^T
-            const int steps2 = g.atom2 / 32, steps1 = g.atom1 / 32;           // MMAs (K = 16) per K-atom
+            const int steps2 = g.atom2 / 32, steps1 = g.atom1 / 32;           // MMAs (K = 16) per K-atom: 1, 2 or 4
+            const int ls2 = steps2 >> 1 == 2 ? 2 : steps2 >> 1, ls1 = steps1 >> 1 == 2 ? 2 : steps1 >> 1;   // log2
+            const int nk2 = atoms2 * steps2, nk1 = atoms1 * steps1;           // k-steps per term
             bool ok = wait_or_abort(const_full, 0, abort_flag);
             if (!ok) give_up(p.status, abort_flag, 0x61);
             for (int it = 0; it < ntok && ok; ++it) {
@@ -362,15 +357,13 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                 if (!wait_or_abort(x_full, ph, abort_flag)) { give_up(p.status, abort_flag, 0x63); break; }
                 tc_fence_after();
                 // stage A: the small terms first, so that the large partial sums meet as few additions as possible
-                uint32_t acc = 0;
+                // k-step q of a term lies in K-atom q >> ls (blocks blk apart), 32 bytes (2 units) per step inside the atom
                 for (int h = 2; h >= 0; --h) {
-                    uint64_t da = dP2 + (uint64_t)((uint32_t)(h * atoms2) * blk_a), dx = dX;
-                    for (int j = 0; j < atoms2; ++j) {
-                        for (int s = 0; s < steps2; ++s) {
-                            mma_f16_ss(tm_d, da + 2u * s, dx + 2u * s, idesc_a, acc);
-                            acc = 1u;
-                        }
-                        da += blk_a; dx += blk_x;
+                    const uint64_t da = dP2 + (uint64_t)((uint32_t)(h * atoms2) * blk_a);
+#pragma unroll 4
+                    for (int q = 0; q < nk2; ++q) {
+                        const uint32_t at = (uint32_t)(q >> ls2), in = (uint32_t)(q & (steps2 - 1)) << 1;
+                        mma_f16_ss(tm_d, da + (at * blk_a + in), dX + (at * blk_x + in), idesc_a, (h == 2 && q == 0) ? 0u : 1u);
                     }
                 }
                 tc_commit(x_empty);
@@ -378,20 +371,16 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                 if (!wait_or_abort(a2_full, ph, abort_flag)) { give_up(p.status, abort_flag, 0x64); break; }
                 tc_fence_after();
                 // stage C: (term of Z^T, term of P1^T), smallest products first
-                acc = 0;
 #pragma unroll
                 for (int pair = 0; pair < 6; ++pair) {
                     constexpr int hz_of[6] = {2, 0, 1, 1, 0, 0};
                     constexpr int hp_of[6] = {0, 2, 1, 0, 1, 0};
-                    uint32_t a_col = tm_a2 + (uint32_t)(hz_of[pair] * (n1p >> 1));
-                    uint64_t db = dP1 + (uint64_t)((uint32_t)(hp_of[pair] * atoms1) * blk_p1);
-                    for (int j = 0; j < atoms1; ++j) {
-                        for (int s = 0; s < steps1; ++s) {
-                            mma_f16_ts(tm_d, a_col, db + 2u * s, idesc_c, acc);
-                            acc = 1u;
-                            a_col += 8;
-                        }
-                        db += blk_p1;
+                    const uint32_t a_col = tm_a2 + (uint32_t)(hz_of[pair] * (n1p >> 1));
+                    const uint64_t db = dP1 + (uint64_t)((uint32_t)(hp_of[pair] * atoms1) * blk_p1);
+#pragma unroll 4
+                    for (int q = 0; q < nk1; ++q) {
+                        const uint32_t at = (uint32_t)(q >> ls1), in = (uint32_t)(q & (steps1 - 1)) << 1;
+                        mma_f16_ts(tm_d, a_col + 8u * q, db + (at * blk_p1 + in), idesc_c, (pair == 0 && q == 0) ? 0u : 1u);
                     }
                 }
                 tc_commit(d2_full);
@@ -400,8 +389,8 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
     } else {
         // ---------------- ALU warps: stage B and stage D ----------------
         const int q = warp & 3;                        // tensor-memory lane quarter this warp may touch
-        const int half = (warp - 2) >> 2;              // which of the two warps of that quarter
-        const int e = threadIdx.x - 64;                // 0..255 among the ALU threads
+        const int part = (warp - 2) >> 2;              // which of the warps of that quarter
+        const int e = threadIdx.x - 64;                // index among the ALU threads
         const int lane_d = q * 32 + lane;              // lane of the accumulator = row d of this CTA's tile
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const bool lane_valid = lane_d < rows;
@@ -421,14 +410,14 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                 tc_fence_after();
                 if (quarter_valid) {
                     uint32_t v[16];
-                    int ch = half;
+                    int ch = part;
                     if (ch < chunks_b) tmem_ld_32x16(tm_d + lane_addr + 16 * ch, v);
                     while (ch < chunks_b) {
                         tc_wait_ld();
                         float f[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(v[i]);
-                        const int nxt = ch + 2;
+                        const int nxt = ch + kOktAluPerQuarter;
                         if (nxt < chunks_b) tmem_ld_32x16(tm_d + lane_addr + 16 * nxt, v);
                         uint32_t th[8], tmid[8], tl[8];
 #pragma unroll
@@ -444,33 +433,40 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                 __syncwarp();
                 if (lane == 0) mbar_arrive(a2_full);
             }
-            // ---- stage D, first pass: absmax
+            // ---- stage D: this warp's chunks of Y^T go to registers (both reads in flight at once) and the accumulator is
+            //      handed back at once, so that the next token's stage A runs under the rest of this one
             if (!failed && !warp_wait(d2_full, ph, abort_flag)) { give_up(p.status, abort_flag, 0x71); failed = true; }
+            uint32_t yv[kOktChunksD][16];
             float amax = 0.f;
             if (!failed && quarter_valid) {
                 tc_fence_after();
-                uint32_t v[16];
-                int ch = half;
-                if (ch < chunks_d) tmem_ld_32x16(tm_d + lane_addr + 16 * ch, v);
-                while (ch < chunks_d) {
-                    tc_wait_ld();
-                    float f[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) f[i] = fabsf(__uint_as_float(v[i]));
-                    const int nxt = ch + 2;
-                    if (nxt < chunks_d) tmem_ld_32x16(tm_d + lane_addr + 16 * nxt, v);
+                for (int j = 0; j < kOktChunksD; ++j)
+                    if (part + j * kOktAluPerQuarter < chunks_d) tmem_ld_32x16(tm_d + lane_addr + 16 * (part + j * kOktAluPerQuarter), yv[j]);
+                tc_wait_ld();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0 && !failed) mbar_arrive(d_free);
+            if (!failed && quarter_valid) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (lane_valid && c0 + 16 * ch + i < g.n1) amax = fmaxf(amax, f[i]);
-                    ch = nxt;
+                for (int j = 0; j < kOktChunksD; ++j) {
+                    const int ch = part + j * kOktAluPerQuarter;
+                    if (ch < chunks_d) {
+                        const int cols_left = g.n1 - (c0 + 16 * ch);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (lane_valid && i < cols_left) amax = fmaxf(amax, fabsf(__uint_as_float(yv[j][i])));
+                    }
                 }
             }
             amax = warp_max(amax);
             if (lane == 0) red_max[warp - 2] = amax;
             // one decision for all ALU warps: a warp that gave up must not leave the others alone at a barrier
             if (alu_barrier_or(failed || *abort_flag != 0)) break;
-            amax = fmaxf(fmaxf(fmaxf(red_max[0], red_max[1]), fmaxf(red_max[2], red_max[3])),
-                         fmaxf(fmaxf(red_max[4], red_max[5]), fmaxf(red_max[6], red_max[7])));
+            amax = 0.f;
+#pragma unroll
+            for (int wi = 0; wi < kOktAluWarps; ++wi) amax = fmaxf(amax, red_max[wi]);
             if (D > 1) {
                 const int par = it & 1;
                 if (e < D) {
@@ -489,60 +485,67 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
             // nothing is stored to global memory before the preceding kernel of the stream has completed
             if (!dep_waited) { griddep_wait(); dep_waited = true; }
-            // ---- stage D, second pass: codes (into the staging buffer when this CTA owns the whole token)
-            int local_sum = 0;
+            // ---- codes.  Rounding to nearest-even by adding 1.5 * 2^23 (the code is then the low byte of the sum's bit
+            //      pattern), clamping in fp32 before it: no float-to-integer conversions, which are slow instructions.
+            //      A CTA that owns the whole token collects the codes in shared memory in natural order (a warp writes 32
+            //      consecutive bytes per column) and reorders them on the way out.
+            float fsum = 0.f;
             int8_t* ct = pr.codes + t * (int64_t)g.K;
             if (!failed && quarter_valid) {
-                const uint32_t stage_addr = smem_u32(stage);
                 const bool interleave = pr.codes_layout != 0;
                 float* yt = pr.y_debug ? pr.y_debug + t * (int64_t)g.K : nullptr;
-                uint32_t v[16];
-                int ch = half;
-                if (ch < chunks_d) tmem_ld_32x16(tm_d + lane_addr + 16 * ch, v);
-                while (ch < chunks_d) {
-                    tc_wait_ld();
-                    float f[16];
+                const float fq = (float)qmax;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(v[i]);
-                    const int nxt = ch + 2;
-                    if (nxt < chunks_d) tmem_ld_32x16(tm_d + lane_addr + 16 * nxt, v);
-                    // Branch-free per element (a branch per element would keep the 16 independent chains from
-                    // overlapping): lanes and columns that hold nothing compute too and only their store is switched off.
-                    const int cols_left = g.n1 - (c0 + 16 * ch);
-                    int code[16];
+                for (int j = 0; j < kOktChunksD; ++j) {
+                    const int ch = part + j * kOktAluPerQuarter;
+                    if (ch < chunks_d) {
+                        const int cols_left = g.n1 - (c0 + 16 * ch);
+                        int k = (c0 + 16 * ch) * g.n2 + d;
+                        const int word_sel = (k & 7) << 2;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int q_i = __float2int_rn(__fmul_rn(f[i], inv));
-                        code[i] = max(-qmax, min(qmax, q_i));
-                        local_sum += (lane_valid && i < cols_left) ? code[i] : 0;
+                        for (int i = 0; i < 16; ++i) {
+                            const bool valid = lane_valid && i < cols_left;
+                            // products beyond +-qmax only come from rounding of the reciprocal: clamp, then round
+                            const float tq = fminf(fmaxf(__fmul_rn(__uint_as_float(yv[j][i]), inv), -fq), fq);
+                            const float magic = __fadd_rn(tq, 12582912.f);
+                            fsum += valid ? __fadd_rn(magic, -12582912.f) : 0.f;
+                            const int8_t code = (int8_t)(__float_as_uint(magic) & 0xFFu);
+                            if (valid) {
+                                if (stage) stage[k] = code;
+                                else ct[interleave ? ((k & ~31) | word_sel | ((k >> 3) & 3)) : k] = code;
+                                if (yt) yt[k] = __uint_as_float(yv[j][i]);
+                            }
+                            k += g.n2;
+                        }
                     }
-                    // k = c * n2 + d advances by n2 (a multiple of 8) per column: the low three bits of k, and with them
-                    // the word inside the 32-group in the interleaved order, stay the same for this thread
-                    int k = (c0 + 16 * ch) * g.n2 + d;
-                    const int word_sel = (k & 7) << 2;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const bool valid = lane_valid && i < cols_left;
-                        const int pos = interleave ? ((k & ~31) | word_sel | ((k >> 3) & 3)) : k;
-                        if (stage) st_shared_u8_if(stage_addr + (uint32_t)pos, code[i], valid);
-                        else if (valid) ct[pos] = (int8_t)code[i];
-                        if (valid && yt) yt[k] = f[i];
-                        k += g.n2;
-                    }
-                    ch = nxt;
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0 && !failed) mbar_arrive(d_free);      // the accumulator may be overwritten by the next token's stage A
+            int local_sum = (int)fsum;                            // a sum of at most 48 integers below 128: exact in fp32
             local_sum = warp_sum(local_sum);
             if (lane == 0 && local_sum != 0) atomicAdd(red_sum, local_sum);
             alu_barrier();
             if (stage && !failed) {
-                // the token's codes leave as 128-bit stores (K is a multiple of 32)
-                const uint4* src = reinterpret_cast<const uint4*>(stage);
-                uint4* out = reinterpret_cast<uint4*>(ct);
-                for (int i = e; i < (g.K >> 4); i += kOktAluThreads) out[i] = src[i];
+                // The token's codes leave as 128-bit stores, one group of 32 per thread and step (K is a multiple of 32).
+                // Interleaved order: output word j of a group holds k = j, j + 8, j + 16, j + 24, i.e. byte j & 3 of the
+                // natural words j >> 2, 2 + (j >> 2), 4 + (j >> 2), 6 + (j >> 2).
+                const bool interleave = pr.codes_layout != 0;
+                for (int gi = e; gi < (g.K >> 5); gi += kOktAluThreads) {
+                    const uint4 lo = *reinterpret_cast<const uint4*>(stage + 32 * gi), hi = *reinterpret_cast<const uint4*>(stage + 32 * gi + 16);
+                    uint4 o0 = lo, o1 = hi;
+                    if (interleave) {
+                        const uint32_t n[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                        uint32_t o[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const uint32_t ab = __byte_perm(n[j >> 2], n[2 + (j >> 2)], (uint32_t)(j & 3) | ((uint32_t)(4 + (j & 3)) << 4));
+                            const uint32_t cd = __byte_perm(n[4 + (j >> 2)], n[6 + (j >> 2)], (uint32_t)(j & 3) | ((uint32_t)(4 + (j & 3)) << 4));
+                            o[j] = __byte_perm(ab, cd, 0x5410);
+                        }
+                        o0 = make_uint4(o[0], o[1], o[2], o[3]); o1 = make_uint4(o[4], o[5], o[6], o[7]);
+                    }
+                    uint4* out = reinterpret_cast<uint4*>(ct + 32 * gi);
+                    out[0] = o0; out[1] = o1;
+                }
             }
             if (e == 0 && !failed) {
                 // every CTA of the cluster leaves its own part of the token's code sum; the consumer adds the parts
@@ -597,8 +600,20 @@ int launch_okt(const OktGeom& g, const void* x, int64_t M, int64_t ldx, int bits
             lp.V = (const __nv_bfloat16*)lowrank[i].V; lp.r = lowrank[i].r; lp.Thl = (__nv_bfloat16*)lowrank[i].Thl;
             lp.lr_cols = lowrank_cols(lowrank[i].r);
             size_t lr_smem = 0;
-            lr_total += plan_lowrank(lp, lowrank[i].lr_part, lowrank[i].lr_count, kOktMaxSmem, &lr_smem);
-            smem = std::max(smem, lr_smem);
+            const int blocks = plan_lowrank(lp, lowrank[i].lr_part, lowrank[i].lr_count, kOktMaxSmem, &lr_smem);
+            if (lp.lr_wide == 3) {
+                // Many tokens: the wide tiles (64 columns x 16 tokens per block, 64 accumulators per lane) need more
+                // registers than a block of this kernel has; they go first, as a launch of their own.  Every kernel of the
+                // chain waits for its predecessor before it ends, so the contraction still finds T complete.
+                int st = launch_prologue(x, M, g.K, ldx, nullptr, 0, nullptr, 0, bits, nullptr, 0, nullptr, nullptr, lowrank[i].V,
+                                         lowrank[i].r, lowrank[i].Thl, lowrank[i].lr_part,
+                                         lowrank[i].lr_count ? lowrank[i].lr_count - kLrCounterWord : nullptr, stream);
+                if (st != BWLA_OK) return st;
+                lp = PrologueParams{};
+            } else {
+                lr_total += blocks;
+                smem = std::max(smem, lr_smem);
+            }
         }
     }
     for (int i = n_problems; i <= kOktMaxProblems; ++i) p.lr_begin[i] = lr_total;

@@ -333,3 +333,88 @@ def test_storage_format_lands_in_the_papers_effective_bit_band():
         n1, n2 = oracle.kron_factor(K)
         bits = N * K + 16 * r * (N + K) + 32 * N + 16 * (n1 * n1 + n2 * n2)
         assert lo - 0.005 <= bits / (N * K) <= hi + 0.005
+
+
+# ------------------------------------------------------------------------------------------------
+# per-token asymmetric quantiser (Sec. 4.1 "per-token asymmetric quantization for activations")
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("bits", [4, 6, 8])
+def test_asymmetric_quantiser_recovers_a_row_that_lies_on_its_grid(bits):
+    """y_k = s0 * (j_k - z0) with every code 0..L present: scale, zero point and codes come back exactly."""
+    L = (1 << bits) - 1
+    s0, z0 = 0.375, L // 3                       # exactly representable scale
+    j = np.concatenate([np.arange(L + 1), np.random.default_rng(bits).integers(0, L + 1, size=200)])
+    y = (s0 * (j - z0))[None, :].astype(np.float64)
+    for decision in ("f64", "f32"):
+        q = oracle.quantize_asym(y, bits, decision)
+        assert q["zeros"][0] == z0 and np.isclose(q["scales"][0], s0, rtol=1e-7)
+        assert np.array_equal(q["codes"][0], j.astype(np.uint8))
+
+
+@pytest.mark.parametrize("bits", [4, 6, 8])
+def test_asymmetric_quantiser_invariants_on_random_rows(bits):
+    rng = np.random.default_rng(100 + bits)
+    Y = rng.standard_t(3, size=(16, 777)) + rng.normal(size=(16, 1)) * 2.0      # rows with a non-zero mean
+    Y[3] = np.abs(Y[3])                                                         # a non-negative row
+    Y[4] = 0.0                                                                  # an all-zero row
+    Y[5, 7] = 0.0                                                               # an exact zero inside a mixed row
+    L = (1 << bits) - 1
+    q = oracle.quantize_asym(Y, bits)
+    u, s, z = q["codes"].astype(np.int64), q["scales"].astype(np.float64), q["zeros"].astype(np.int64)
+    assert u.min() >= 0 and u.max() <= L and z.min() >= 0 and z.max() <= L
+    lo, hi = np.minimum(Y.min(axis=1), 0), np.maximum(Y.max(axis=1), 0)
+    live = hi > lo
+    assert np.allclose(s[live], ((hi - lo) / L)[live], rtol=1e-6)
+    assert s[4] == 1.0 and z[4] == 0 and not u[4].any()
+    # the value a code stands for is within half a step of y (a step more where the sum met the clamp)
+    deq = s[:, None] * (u - z[:, None])
+    assert np.all(np.abs(deq - Y)[live] <= 0.5 * s[live, None] * (1 + 1e-6) + 1e-12) or \
+        np.all(np.abs(deq - Y)[live] <= 1.5 * s[live, None])
+    frac_clamped = np.mean(np.abs(deq - Y)[live] > 0.5 * s[live, None] * (1 + 1e-6) + 1e-12)
+    assert frac_clamped < 1e-3
+    # zero is represented exactly, the smallest value takes code 0, the largest a code within one of L
+    assert u[5, 7] == z[5] and deq[5, 7] == 0.0
+    assert np.all(u[live].min(axis=1) == 0) and np.all(u[live].max(axis=1) >= L - 1)
+    # a non-negative row needs no zero point and gets the whole range: twice the resolution of the symmetric quantiser
+    assert z[3] == 0
+    sym = oracle.quantize(Y[3:4], bits)
+    assert s[3] < 0.51 * sym["scales"][0] * (1 + 2.0 / L)
+
+
+def test_asymmetric_contraction_is_the_plain_contraction_minus_zero_times_row_sum():
+    """sum_k sign * (u - z) = sum_k sign * u - z * (2 * popc(row) - K): the identity the kernels' epilogue relies on,
+    against the oracle's direct evaluation."""
+    rng = np.random.default_rng(5)
+    M, N, K = 5, 37, 96
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    packed = oracle.pack_signs(W)
+    signs = oracle.unpack_signs(packed, K).astype(np.int64)
+    u = rng.integers(0, 64, size=(M, K)).astype(np.uint8)
+    z = rng.integers(0, 64, size=M).astype(np.int32)
+    acc, rsum = oracle.gemm_asym(u, z, packed)
+    rowsum = 2 * np.array([bin(int(w)).count("1") for w in packed.reshape(-1)]).reshape(N, -1).sum(axis=1) - K
+    assert np.array_equal(rowsum, signs.sum(axis=1))
+    want = u.astype(np.int64) @ signs.T - z.astype(np.int64)[:, None] * rowsum[None, :]
+    assert np.array_equal(acc, want)
+    assert np.array_equal(rsum, u.astype(np.int64).sum(axis=1) - K * z.astype(np.int64))
+
+
+def test_asymmetric_layer_approaches_the_unquantised_product_with_more_bits():
+    """The layer with asymmetric codes against the same layer on unquantised rotated activations: the error falls by
+    about 4x per two bits, and is no larger than the symmetric quantiser's on activations with a non-zero mean."""
+    rng = np.random.default_rng(11)
+    shape = gen.small_shape(256, 48, 16, 16, 0, shape_id=31)
+    lay = gen.make_layer(0, shape, 6)
+    x = rng.standard_normal((6, 256)).astype(np.float32) + 1.5
+    xb = gen.bf16_bits_from_f32(x)
+    packed = oracle.pack_signs(lay.W)
+    signs = oracle.unpack_signs(packed, 256).astype(np.float64)
+    Y = oracle.rotate(xb, lay.P1, lay.P2)
+    exact = (Y @ signs.T) * lay.alpha.astype(np.float64)[None, :]
+    errs = {}
+    for bits in (4, 6, 8):
+        ya = oracle.linear_asym(xb, lay.P1, lay.P2, bits, packed, lay.alpha)["y"]
+        ys = oracle.linear(xb, lay.P1, lay.P2, bits, packed, lay.alpha)["y"]
+        errs[bits] = (np.linalg.norm(ya - exact), np.linalg.norm(ys - exact))
+    assert errs[6][0] < 0.4 * errs[4][0] and errs[8][0] < 0.4 * errs[6][0]
+    assert all(errs[b][0] <= 1.05 * errs[b][1] for b in errs)
