@@ -493,29 +493,41 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             int8_t* ct = pr.codes + t * (int64_t)g.K;
             if (!failed && quarter_valid) {
                 const bool interleave = pr.codes_layout != 0;
-                float* yt = pr.y_debug ? pr.y_debug + t * (int64_t)g.K : nullptr;
                 const float fq = (float)qmax;
 #pragma unroll
                 for (int j = 0; j < kOktChunksD; ++j) {
                     const int ch = part + j * kOktAluPerQuarter;
                     if (ch < chunks_d) {
                         const int cols_left = g.n1 - (c0 + 16 * ch);
-                        int k = (c0 + 16 * ch) * g.n2 + d;
-                        const int word_sel = (k & 7) << 2;
+                        const int k0 = (c0 + 16 * ch) * g.n2 + d;
+                        uint32_t code[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            const bool valid = lane_valid && i < cols_left;
                             // products beyond +-qmax only come from rounding of the reciprocal: clamp, then round
                             const float tq = fminf(fmaxf(__fmul_rn(__uint_as_float(yv[j][i]), inv), -fq), fq);
                             const float magic = __fadd_rn(tq, 12582912.f);
-                            fsum += valid ? __fadd_rn(magic, -12582912.f) : 0.f;
-                            const int8_t code = (int8_t)(__float_as_uint(magic) & 0xFFu);
-                            if (valid) {
-                                if (stage) stage[k] = code;
-                                else ct[interleave ? ((k & ~31) | word_sel | ((k >> 3) & 3)) : k] = code;
-                                if (yt) yt[k] = __uint_as_float(yv[j][i]);
+                            fsum += (lane_valid && i < cols_left) ? __fadd_rn(magic, -12582912.f) : 0.f;
+                            code[i] = __float_as_uint(magic);
+                        }
+                        // one simple guarded store per element, so that the compiler predicates it instead of branching
+                        if (stage) {
+                            int8_t* dst = stage + k0;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                if (lane_valid && i < cols_left) dst[i * g.n2] = (int8_t)code[i];
+                        } else {
+                            const int word_sel = (k0 & 7) << 2;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const int k = k0 + i * g.n2;
+                                if (lane_valid && i < cols_left) ct[interleave ? ((k & ~31) | word_sel | ((k >> 3) & 3)) : k] = (int8_t)code[i];
                             }
-                            k += g.n2;
+                        }
+                        if (pr.y_debug) {
+                            float* yt = pr.y_debug + t * (int64_t)g.K + k0;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                if (lane_valid && i < cols_left) yt[i * g.n2] = __uint_as_float(yv[j][i]);
                         }
                     }
                 }
