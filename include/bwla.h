@@ -172,6 +172,23 @@ int bwla_layer_rotate_quant(const bwla_layer* layer, const void* x_bf16, int64_t
                             int8_t* codes, float* scales, float* y_f32, void* stream);
 
 /*
+ * Activation quantiser of a prepared layer.  BWLA_ACT_SYMMETRIC (the default): codes in [-qmax, qmax] and one scale per
+ * token.  BWLA_ACT_ASYMMETRIC: the paper's stated setting (Sec. 4.1, "per-token asymmetric quantization for
+ * activations"): lo = min(0, min y), hi = max(0, max y), scale = (hi - lo) / (2^b - 1), an integer zero point
+ * z = rne(-lo / scale), codes u = clamp(rne(y / scale) + z, 0, 2^b - 1); the layer then computes
+ *   out = bf16( alpha[n] * s_t * (sum_k sign[n][k] * u_k - z_t * rowsum[n]) + U (V x_t) [+ mu[n] * s_t * sum_k (u_k - z_t)] ),
+ * rowsum[n] = sum_k sign[n][k] (prepared once per layer).  Returns BWLA_ERR_UNSUPPORTED for factor sizes only the
+ * fallback rotation kernel takes.
+ */
+enum { BWLA_ACT_SYMMETRIC = 0, BWLA_ACT_ASYMMETRIC = 1 };
+int bwla_layer_set_activation_quant(bwla_layer* layer, int mode);
+
+/* The asymmetric quantiser alone: codes device uint8 [M][K] (u), scales device fp32 [M], zeros device int32 [M] (z),
+ * y_f32 device fp32 [M][K] or NULL. */
+int bwla_layer_rotate_quant_asym(const bwla_layer* layer, const void* x_bf16, int64_t M, int64_t ldx,
+                                 uint8_t* codes, float* scales, int32_t* zeros, float* y_f32, void* stream);
+
+/*
  * Several layers that read the same activations (q, k, v of an attention block; gate and up of an MLP) in one
  * call: x is rotated and quantised for every layer (each has its own P1, P2) by one launch, and the contractions
  * follow.  All layers must have the same K, n1, n2 and bits; count <= 4.
@@ -213,10 +230,12 @@ int bwla_check_status(void* workspace, void* stream);
  *          BWLA_WS_T       bf16 [3][M][max(64, r)]         T = V x as hi + mid + lo
  *          BWLA_WS_CODES   int8 [M][K]                     codes; on the tensor-core path inside each group of 32
  *                                                          consecutive k, byte 4*j + i holds k = j + 8*i
+ *          BWLA_WS_ZEROS   int32 [M]                       asymmetric quantiser only: zero points; codes and zero
+ *                                                          points are both kept minus 2^(b-1) so that codes fit int8
  *   offset, bytes: host pointers that receive the section's position and size.
  * Returns BWLA_ERR_INVALID_ARG for invalid dimensions or an unknown section.
  */
-enum { BWLA_WS_SCALES = 0, BWLA_WS_QSUM = 1, BWLA_WS_T = 2, BWLA_WS_CODES = 3 };
+enum { BWLA_WS_SCALES = 0, BWLA_WS_QSUM = 1, BWLA_WS_T = 2, BWLA_WS_CODES = 3, BWLA_WS_ZEROS = 4 };
 int bwla_workspace_section(int64_t M, int64_t K, int64_t N, int r, int bits, int which, size_t* offset, size_t* bytes);
 
 /* Force every later call of the calling thread onto one kernel family (benchmarking the non-chosen path,

@@ -37,6 +37,7 @@ EXPORTS = [
     "bwla_status_string", "bwla_profile_enable", "bwla_profile_collect", "bwla_w1ax_linear_static",
     "bwla_workspace_section", "bwla_force_rotation", "bwla_layer_prepared_bytes", "bwla_layer_create",
     "bwla_layer_destroy", "bwla_layer_rotate_quant", "bwla_group_workspace_bytes", "bwla_w1ax_linear_group",
+    "bwla_layer_set_activation_quant", "bwla_layer_rotate_quant_asym",
 ]
 
 
@@ -76,6 +77,10 @@ def _load() -> C.CDLL:
     lib.bwla_layer_destroy.restype = None
     lib.bwla_layer_rotate_quant.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
     lib.bwla_layer_rotate_quant.restype = ci
+    lib.bwla_layer_set_activation_quant.argtypes = [vp, ci]
+    lib.bwla_layer_set_activation_quant.restype = ci
+    lib.bwla_layer_rotate_quant_asym.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
+    lib.bwla_layer_rotate_quant_asym.restype = ci
     lib.bwla_group_workspace_bytes.argtypes = [C.POINTER(vp), ci, i64]
     lib.bwla_group_workspace_bytes.restype = sz
     lib.bwla_w1ax_linear_group.argtypes = [C.POINTER(vp), ci, vp, i64, i64, C.POINTER(vp), C.POINTER(i64), vp, sz, vp]
@@ -240,7 +245,7 @@ def bwla_w1ax_linear_static(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor,
 class Layer:
     """A prepared layer (bwla_layer_create): keeps the handle, the tensors it points into and the prepared buffer."""
 
-    def __init__(self, P1, P2, bits, packed, alpha, U=None, V=None, mu=None):
+    def __init__(self, P1, P2, bits, packed, alpha, U=None, V=None, mu=None, asymmetric=False):
         _need(packed, torch.int32, "packed", 2)
         _need(alpha, torch.float32, "alpha", 1)
         _need(P1, torch.float32, "P1", 2)
@@ -268,6 +273,8 @@ class Layer:
                                     _ptr(packed), _ptr(alpha), _ptr(mu), _ptr(U), _ptr(V), self.r, _ptr(self.prepared),
                                     nbytes, _stream())
         _check(st, "bwla_layer_create")
+        if asymmetric:
+            bwla_layer_set_activation_quant(self, BWLA_ACT_ASYMMETRIC)
 
     def __del__(self):
         h = getattr(self, "handle", None)
@@ -280,13 +287,31 @@ def bwla_layer_prepared_bytes(K: int, N: int, n1: int, n2: int, r: int) -> int:
     return int(_lib.bwla_layer_prepared_bytes(K, N, n1, n2, r))
 
 
-def bwla_layer_create(P1, P2, bits, packed, alpha, U=None, V=None, mu=None) -> Layer:
+def bwla_layer_create(P1, P2, bits, packed, alpha, U=None, V=None, mu=None, asymmetric=False) -> Layer:
     """Prepares a layer's constants once (launches on the current stream) and returns the handle object."""
-    return Layer(P1, P2, bits, packed, alpha, U, V, mu)
+    return Layer(P1, P2, bits, packed, alpha, U, V, mu, asymmetric)
 
 
 def bwla_layer_destroy(layer: Layer) -> None:
     layer.__del__()
+
+
+def bwla_layer_set_activation_quant(layer: Layer, mode: int) -> None:
+    _check(_lib.bwla_layer_set_activation_quant(layer.handle, mode), "bwla_layer_set_activation_quant")
+
+
+def bwla_layer_rotate_quant_asym(layer: Layer, x: torch.Tensor, want_y: bool = False):
+    """(codes uint8 [M][K], scales fp32 [M], zeros int32 [M], Y fp32 [M][K] or None): the per-token asymmetric quantiser."""
+    _need(x, torch.bfloat16, "x", 2)
+    M, K = x.shape
+    codes = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((M,), dtype=torch.float32, device=x.device)
+    zeros = torch.empty((M,), dtype=torch.int32, device=x.device)
+    y = torch.empty((M, K), dtype=torch.float32, device=x.device) if want_y else None
+    st = _lib.bwla_layer_rotate_quant_asym(layer.handle, _ptr(x), M, x.stride(0) if M > 0 else K, _ptr(codes), _ptr(scales),
+                                           _ptr(zeros), _ptr(y), _stream())
+    _check(st, "bwla_layer_rotate_quant_asym")
+    return codes, scales, zeros, y
 
 
 def bwla_layer_rotate_quant(layer: Layer, x: torch.Tensor, want_y: bool = False):
@@ -370,7 +395,8 @@ def bwla_w1a_gemm_codes(codes: torch.Tensor, scales: torch.Tensor, bits: int, pa
     return out, acc
 
 
-BWLA_WS_SCALES, BWLA_WS_QSUM, BWLA_WS_T, BWLA_WS_CODES = 0, 1, 2, 3
+BWLA_WS_SCALES, BWLA_WS_QSUM, BWLA_WS_T, BWLA_WS_CODES, BWLA_WS_ZEROS = 0, 1, 2, 3, 4
+BWLA_ACT_SYMMETRIC, BWLA_ACT_ASYMMETRIC = 0, 1
 
 
 def bwla_workspace_section(M: int, K: int, N: int, r: int, bits: int, which: int):

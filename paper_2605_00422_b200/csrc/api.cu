@@ -94,6 +94,8 @@ struct bwla_layer {
     uint8_t* prepared;
     bool okt;                 // the tcgen05 rotation takes these factor sizes
     OktGeom geom;
+    int asym;                 // activation quantiser: 0 symmetric, 1 asymmetric (per-token zero point)
+    int32_t* rowsum;          // [N] sign sums of the rows, inside `prepared`
 };
 
 extern "C" {
@@ -183,9 +185,9 @@ int bwla_w1ax_linear(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, cons
         // does this once instead)
         st = launch_prepare_okt(geom, P1, P2, base + ws.prep, s);
         if (st != BWLA_OK) return st;
-        OktProblem pr{(const uint8_t*)(base + ws.prep), codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum, nullptr};
+        OktProblem pr{(const uint8_t*)(base + ws.prep), codes, path == BWLA_PATH_I8 ? 1 : 0, nullptr, 0, scales, qsum, nullptr};
         OktLowrank lr{V_bf16, r, Thl, r > 0 ? (float*)(base + ws.lr_part) : nullptr, (uint32_t*)(base + ws.status) + kLrCounterWord};
-        st = launch_okt(geom, x_bf16, M, ldx, bits, 1, &pr, &lr, (uint32_t*)(base + ws.status), s);
+        st = launch_okt(geom, x_bf16, M, ldx, bits, 0, 1, &pr, &lr, (uint32_t*)(base + ws.status), s);
     } else {
         st = launch_prologue(x_bf16, M, K, ldx, P1, n1, P2, n2, bits, codes, path == BWLA_PATH_I8 ? 1 : 0, scales, qsum,
                              V_bf16, r, Thl, r > 0 ? (float*)(base + ws.lr_part) : nullptr, (uint32_t*)(base + ws.status), s);
@@ -242,6 +244,7 @@ int bwla_workspace_section(int64_t M, int64_t K, int64_t N, int r, int bits, int
         case BWLA_WS_QSUM:   *offset = w.qsum;   *bytes = (size_t)M * 4 * kQsumParts; return BWLA_OK;
         case BWLA_WS_T:      *offset = w.T;      *bytes = (size_t)M * lowrank_cols(r) * 6; return BWLA_OK;
         case BWLA_WS_CODES:  *offset = w.codes;  *bytes = (size_t)M * (size_t)K; return BWLA_OK;
+        case BWLA_WS_ZEROS:  *offset = w.zp;     *bytes = (size_t)M * 4; return BWLA_OK;
         default: return BWLA_ERR_INVALID_ARG;
     }
 }
@@ -251,7 +254,8 @@ int bwla_workspace_section(int64_t M, int64_t K, int64_t N, int r, int bits, int
 size_t bwla_layer_prepared_bytes(int64_t K, int64_t N, int n1, int n2, int r) {
     if (!valid_rotation_dims(K, n1, n2) || N < 0 || r < 0 || r > 256) return 0;
     OktGeom g;
-    return okt_geometry(n1, n2, &g) ? align_up(okt_prepared_bytes(g), 256) : 256;
+    // the terms of the Kronecker factors for the tensor-core rotation, then the sign sums of the rows
+    return (okt_geometry(n1, n2, &g) ? align_up(okt_prepared_bytes(g), 256) : 256) + align_up((size_t)N * 4, 256);
 }
 
 int bwla_layer_create(bwla_layer** layer, int64_t K, int64_t N, const float* P1, int n1, const float* P2, int n2, int bits,
@@ -273,15 +277,40 @@ int bwla_layer_create(bwla_layer** layer, int64_t K, int64_t N, const float* P1,
     L->P1 = P1; L->P2 = P2; L->packed = packed; L->alpha = alpha; L->mu = mu; L->U = U_bf16; L->V = V_bf16;
     L->prepared = (uint8_t*)prepared;
     L->okt = okt_geometry(n1, n2, &L->geom);
+    L->asym = 0;
+    L->rowsum = (int32_t*)((uint8_t*)prepared + (L->okt ? align_up(okt_prepared_bytes(L->geom), 256) : 256));
     if (L->okt) {
         st = launch_prepare_okt(L->geom, P1, P2, prepared, (cudaStream_t)stream);
         if (st != BWLA_OK) { free(L); return st; }
     }
+    st = launch_row_sums(packed, N, K, L->rowsum, (cudaStream_t)stream);
+    if (st != BWLA_OK) { free(L); return st; }
     *layer = L;
     return BWLA_OK;
 }
 
 void bwla_layer_destroy(bwla_layer* layer) { free(layer); }
+
+int bwla_layer_set_activation_quant(bwla_layer* layer, int mode) {
+    if (!layer || (mode != BWLA_ACT_SYMMETRIC && mode != BWLA_ACT_ASYMMETRIC)) return BWLA_ERR_INVALID_ARG;
+    if (mode == BWLA_ACT_ASYMMETRIC && !layer->okt) return BWLA_ERR_UNSUPPORTED;   // only the tensor-core rotation has it
+    layer->asym = mode;
+    return BWLA_OK;
+}
+
+int bwla_layer_rotate_quant_asym(const bwla_layer* L, const void* x_bf16, int64_t M, int64_t ldx, uint8_t* codes, float* scales,
+                                 int32_t* zeros, float* y_f32, void* stream) {
+    g_launch_count = 0;
+    if (!L || M < 0 || ldx < L->K) return BWLA_ERR_INVALID_ARG;
+    if (M == 0) return BWLA_OK;
+    if (!x_bf16 || !codes || !scales || !zeros || ((uintptr_t)codes & 15)) return BWLA_ERR_INVALID_ARG;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+    if (!L->okt || !okt_accepts_x(x_bf16, ldx)) return BWLA_ERR_UNSUPPORTED;
+    // the kernel keeps u - 2^(b-1) so that codes fit int8; the bias puts u and the zero point back in [0, 2^b - 1]
+    OktProblem pr{L->prepared, (int8_t*)codes, 0, zeros, 1 << (L->bits - 1), scales, nullptr, y_f32};
+    return launch_okt(L->geom, x_bf16, M, ldx, L->bits, 1, 1, &pr, nullptr, nullptr, (cudaStream_t)stream);
+}
 
 int bwla_layer_rotate_quant(const bwla_layer* L, const void* x_bf16, int64_t M, int64_t ldx, int8_t* codes, float* scales,
                             float* y_f32, void* stream) {
@@ -292,8 +321,8 @@ int bwla_layer_rotate_quant(const bwla_layer* L, const void* x_bf16, int64_t M, 
     int st = check_device();
     if (st != BWLA_OK) return st;
     if (L->okt && g_forced_rotation != BWLA_ROT_SIMT && okt_accepts_x(x_bf16, ldx)) {
-        OktProblem pr{L->prepared, codes, 0, scales, nullptr, y_f32};
-        return launch_okt(L->geom, x_bf16, M, ldx, L->bits, 1, &pr, nullptr, nullptr, (cudaStream_t)stream);
+        OktProblem pr{L->prepared, codes, 0, nullptr, 0, scales, nullptr, y_f32};
+        return launch_okt(L->geom, x_bf16, M, ldx, L->bits, 0, 1, &pr, nullptr, nullptr, (cudaStream_t)stream);
     }
     if (y_f32) return BWLA_ERR_UNSUPPORTED;      // only the tensor-core kernel can hand out Y
     return launch_prologue(x_bf16, M, L->K, ldx, L->P1, L->n1, L->P2, L->n2, L->bits, codes, 0, scales, nullptr, nullptr, 0,
@@ -305,7 +334,7 @@ static bool valid_group(const bwla_layer* const* layers, int count) {
     for (int i = 0; i < count; ++i) {
         if (!layers[i]) return false;
         if (layers[i]->K != layers[0]->K || layers[i]->n1 != layers[0]->n1 || layers[i]->n2 != layers[0]->n2 ||
-            layers[i]->bits != layers[0]->bits)
+            layers[i]->bits != layers[0]->bits || layers[i]->asym != layers[0]->asym)
             return false;
     }
     return true;
@@ -347,17 +376,19 @@ int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const voi
     }
     bool okt = g_forced_rotation != BWLA_ROT_SIMT && okt_accepts_x(x_bf16, ldx);
     for (int i = 0; i < count; ++i) okt = okt && layers[i]->okt;
+    if (L0->asym && !okt) return BWLA_ERR_UNSUPPORTED;     // the asymmetric quantiser lives in the tensor-core rotation
     if (okt) {
         OktProblem pr[kOktMaxProblems];
         OktLowrank lr[kOktMaxProblems];
         for (int i = 0; i < count; ++i) {
             const bwla_layer* L = layers[i];
             pr[i] = OktProblem{L->prepared, (int8_t*)(wbase[i] + ws[i].codes), path[i] == BWLA_PATH_I8 ? 1 : 0,
+                               L->asym ? (int32_t*)(wbase[i] + ws[i].zp) : nullptr, 0,
                                (float*)(wbase[i] + ws[i].scales), (int32_t*)(wbase[i] + ws[i].qsum), nullptr};
             lr[i] = OktLowrank{L->V, L->r, wbase[i] + ws[i].T, L->r > 0 ? (float*)(wbase[i] + ws[i].lr_part) : nullptr,
                                (uint32_t*)(wbase[i] + ws[i].status) + kLrCounterWord};
         }
-        st = launch_okt(L0->geom, x_bf16, M, ldx, L0->bits, count, pr, lr, status, s);
+        st = launch_okt(L0->geom, x_bf16, M, ldx, L0->bits, L0->asym, count, pr, lr, status, s);
         if (st != BWLA_OK) return st;
     } else {
         for (int i = 0; i < count; ++i) {
@@ -374,6 +405,7 @@ int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const voi
         GemmArgs g{};
         g.scales = (float*)(wbase[i] + ws[i].scales); g.qsum = (int32_t*)(wbase[i] + ws[i].qsum);
         g.M = M; g.K = L->K; g.N = L->N; g.bits = L->bits; g.packed = L->packed; g.alpha = L->alpha; g.mu = L->mu;
+        g.zp = L->asym ? (int32_t*)(wbase[i] + ws[i].zp) : nullptr; g.rowsum = L->rowsum;
         g.Thl = L->r > 0 ? wbase[i] + ws[i].T : nullptr; g.U = L->U; g.r = L->r; g.out = outs[i]; g.ldo = ldos[i];
         g.acc_debug = nullptr; g.status = status;
         st = run_contraction(path[i], g, (int8_t*)(wbase[i] + ws[i].codes), s);

@@ -84,7 +84,7 @@ constexpr int kLrCounterWord = 4;
 __host__ __device__ inline int lowrank_cols(int r) { return r > kLowrankPad ? (r + 1) / 2 * 2 : kLowrankPad; }
 
 struct Workspace {
-    size_t status, scales, qsum, T, lr_part, codes, prep, total;
+    size_t status, scales, zp, qsum, T, lr_part, codes, prep, total;
 };
 
 // Room for the prepared Kronecker factors of one call (bf16 terms of P2^T and P1^T for the largest factor sizes the
@@ -96,6 +96,7 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     size_t off = 0;
     w.status = off; off += kStatusBytes;
     w.scales = off; off += align_up((size_t)M * 4, 256);
+    w.zp = off;     off += align_up((size_t)M * 4, 256);        // per-token zero points (asymmetric activations)
     w.qsum = off;   off += align_up((size_t)M * 4 * kQsumParts, 256);
     const size_t lr_cols = (size_t)lowrank_cols(r);
     w.T = off;      off += align_up((size_t)M * lr_cols * 6, 256);     // bf16 [3][M][cols]
@@ -119,6 +120,8 @@ int validate_linear_call(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, 
 // ---------------------------------------------------------------------------------------------
 int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw, uint32_t* packed,
                       cudaStream_t stream);
+// rowsum[n] = sum_k sign(n,k) = 2 * popc(row n) - K
+int launch_row_sums(const uint32_t* packed, int64_t N, int64_t K, int32_t* rowsum, cudaStream_t stream);
 
 // One launch: fused rotate + absmax + quantise (skipped when codes == NULL) and T = V x (skipped when r == 0 or
 // Thl == NULL).  codes_layout: 0 = natural k order, 1 = interleaved order used by the tensor-core contraction (inside
@@ -147,6 +150,8 @@ struct OktProblem {
     const uint8_t* prepared;    // bf16 terms of P2^T tiles and P1^T slabs (launch_prepare_okt)
     int8_t* codes;              // [M][K]
     int codes_layout;           // 0: natural k order; 1: the interleaved order of the tensor-core contraction
+    int32_t* zp;                // [M] zero points (asymmetric quantiser), or NULL
+    int code_bias;              // added to every stored code and to the stored zero point (see launch_okt)
     float* scales;              // [M]
     int32_t* qsum;              // [M][kQsumParts] or NULL
     float* y_debug;             // [M][K] fp32 rotated activations before the quantiser, or NULL
@@ -160,7 +165,10 @@ size_t okt_prepared_bytes(const OktGeom& g);
 int launch_prepare_okt(const OktGeom& g, const float* P1, const float* P2, void* prepared, cudaStream_t stream);
 // One launch for up to kOktMaxProblems linears that read the same x: rotation + quantiser for each, and the T = V x
 // blocks of those with a low-rank branch.
-int launch_okt(const OktGeom& g, const void* x, int64_t M, int64_t ldx, int bits, int n_problems,
+// asym == 0: symmetric codes in [-qmax, qmax], qmax = 2^(b-1) - 1.  asym == 1 (Sec. 4.1, per-token asymmetric): with
+// u in [0, 2^b - 1] and the integer zero point z of the token, the stored code is u - 2^(b-1) + code_bias and the
+// stored zero point z - 2^(b-1) + code_bias; a code minus the zero point times the scale is the value it stands for.
+int launch_okt(const OktGeom& g, const void* x, int64_t M, int64_t ldx, int bits, int asym, int n_problems,
                const OktProblem* problems, const OktLowrank* lowrank, uint32_t* status, cudaStream_t stream);
 
 // qsum[t][0] = sum_k codes[t][k] (the other parts zero); optionally rewrites natural-order codes into the interleaved order.
@@ -176,6 +184,8 @@ struct GemmArgs {
     const uint32_t* packed;   // [N][K/32]
     const float* alpha;       // [N]
     const float* mu;          // [N] or NULL
+    const int32_t* zp;        // [M] per-token zero points of the codes, or NULL (symmetric codes)
+    const int32_t* rowsum;    // [N] sum_k sign(n,k) = 2 * popc(row n) - K; read only when zp is given
     const void* Thl;          // bf16 [3][M][lowrank_cols(r)] or NULL
     const void* U;            // bf16 [N][r] or NULL
     int r;

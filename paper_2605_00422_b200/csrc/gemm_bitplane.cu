@@ -38,6 +38,7 @@ struct BitplaneParams {
     const int32_t* qsum;      // [M][kQsumParts]
     const uint32_t* packed;   // [N][K/32]
     const float* alpha; const float* mu;
+    const int32_t* zp; const int32_t* rowsum;       // asymmetric codes: per-token zero points, per-row sign sums (or NULL)
     const __nv_bfloat16* U; const __nv_bfloat16* Thl; int r, lr_cols;
     __nv_bfloat16* out; int64_t ldo; int32_t* acc_debug;
     int M, N, K, bits, R;     // R: rows per CTA (a multiple of 16)
@@ -159,7 +160,9 @@ __global__ void __launch_bounds__(kBpThreads, MT <= 2 ? 2 : 1) bitplane_w1a_kern
         const int n = n0 + row;
         int32_t qs = 0;
         for (int c = 0; c < kQsumParts; ++c) qs += p.qsum[(size_t)t * kQsumParts + c];
-        const int32_t acc = 2 * tile_acc[o] - qs;
+        const int32_t zp = p.zp ? p.zp[t] : 0;
+        const int32_t acc = 2 * tile_acc[o] - qs - (p.zp ? zp * p.rowsum[n] : 0);
+        qs -= p.K * zp;
         if (p.acc_debug) p.acc_debug[(size_t)t * p.N + n] = acc;
         if (p.out) {
             const float sc = p.scales[t];
@@ -220,6 +223,7 @@ int launch_gemm_bitplane(const GemmArgs& a, cudaStream_t stream) {
     if (sms <= 0) return BWLA_ERR_CUDA;
     BitplaneParams p{};
     p.codes = a.codes; p.scales = a.scales; p.qsum = a.qsum; p.packed = a.packed; p.alpha = a.alpha; p.mu = a.mu;
+    p.zp = a.zp; p.rowsum = a.rowsum;
     p.U = (const __nv_bfloat16*)a.U; p.Thl = (const __nv_bfloat16*)a.Thl; p.r = a.r; p.lr_cols = lowrank_cols(a.r);
     p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug;
     p.M = (int)a.M; p.N = (int)a.N; p.K = (int)a.K; p.bits = a.bits;

@@ -42,6 +42,9 @@ __global__ void __launch_bounds__(128) gemm_simple_kernel(GemmArgs a) {
 #pragma unroll
         for (int i = 0; i < kTokTile; ++i) v = (lane == i) ? acc[i] : v;
         const int64_t t = t0 + lane;
+        // asymmetric codes: the zero point leaves through the row's sign sum (exact in int32)
+        const int32_t zp = a.zp ? a.zp[t] : 0;
+        if (a.zp) v -= zp * a.rowsum[n];
         if (a.acc_debug) a.acc_debug[t * a.N + n] = v;
         if (a.out) {
             const float sc = a.scales[t];
@@ -61,6 +64,7 @@ __global__ void __launch_bounds__(128) gemm_simple_kernel(GemmArgs a) {
             if (a.mu) {
                 int32_t qs = 0;
                 for (int c = 0; c < kQsumParts; ++c) qs += a.qsum[t * kQsumParts + c];
+                qs -= (int32_t)a.K * zp;
                 y = fmaf(__fmul_rn(a.mu[n], sc), (float)qs, y);
             }
             ((__nv_bfloat16*)a.out)[t * a.ldo + n] = __float2bfloat16_rn(y);

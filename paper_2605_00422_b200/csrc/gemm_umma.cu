@@ -55,6 +55,8 @@ struct UmmaParams {
     const int32_t* qsum;         // [M][kQsumParts] partial sums
     const float* alpha;          // [N]
     const float* mu;             // [N] or NULL
+    const int32_t* zp;           // [M] zero points of asymmetric codes, or NULL
+    const int32_t* rowsum;       // [N] sum_k sign(n,k); read only when zp is given
     const __nv_bfloat16* U;      // [N][r] or NULL
     __nv_bfloat16* out;          // [M][ldo] or NULL
     int64_t ldo;
@@ -87,8 +89,8 @@ struct UmmaCfg {
     static constexpr int bars_off = t_off + 3 * sub_bytes;
     static constexpr int n_bars = 2 * WS + 2 * BS + 2 * AS + 4;
     static constexpr int misc_off = bars_off + n_bars * 8;            // tmem slot, abort flag
-    static constexpr int tok_off = misc_off + 16;                      // scales[N_TOK], qsum[N_TOK]
-    static constexpr int used = tok_off + 8 * N_TOK;
+    static constexpr int tok_off = misc_off + 16;                      // scales[N_TOK], qsum[N_TOK], zero points[N_TOK]
+    static constexpr int used = tok_off + 12 * N_TOK;
     static constexpr int total = used + 1024;                          // + slack for 1024-byte alignment
     static constexpr int red_bytes = 2 * N_TOK * kRowsPerCta * 4;
     static constexpr bool can_split = red_bytes <= u_off;
@@ -98,10 +100,12 @@ struct UmmaCfg {
     static_assert(N_TOK * kRowsPerCta * 2 <= u_off, "output tile does not fit the stage memory");
 };
 
-// One output value from its two accumulators (mu_sc is zero when the layer has no row shift).
-__device__ __forceinline__ float finish_value(int32_t d, float l, float alpha_sc, float mu_sc, int32_t qs) {
-    const int32_t acc = -(d >> 6) - qs;
-    return fmaf(mu_sc, (float)qs, __fmul_rn(alpha_sc, (float)acc) + l);
+// One output value from its two accumulators (mu_sc is zero when the layer has no row shift).  zr = zero point of the
+// token x sign sum of the row, kz = K x zero point (both zero for symmetric codes): a code stands for scale * (code -
+// zero point), and the zero point's share of the sums is taken out in exact integer arithmetic.
+__device__ __forceinline__ float finish_value(int32_t d, float l, float alpha_sc, float mu_sc, int32_t qs, int32_t zr, int32_t kz) {
+    const int32_t acc = -(d >> 6) - qs - zr;
+    return fmaf(mu_sc, (float)(qs - kz), __fmul_rn(alpha_sc, (float)acc) + l);
 }
 
 template <int N_TOK, int WS, int BS, int TMEM_COLS, int NISS, int EW>
@@ -133,6 +137,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::misc_off + 4);
     float* scale_s = reinterpret_cast<float*>(smem + L::tok_off);
     int32_t* qsum_s = reinterpret_cast<int32_t*>(smem + L::tok_off + 4 * N_TOK);
+    int32_t* zp_s = reinterpret_cast<int32_t*>(smem + L::tok_off + 8 * N_TOK);
     // after the K loop the stage memory is free:
     int32_t* red_i = reinterpret_cast<int32_t*>(smem);                                 // [N_TOK][128] partial sums
     float* red_f = reinterpret_cast<float*>(smem + N_TOK * kRowsPerCta * 4);           // [N_TOK][128] low-rank term
@@ -207,6 +212,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 qs = a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w;
             }
             qsum_s[i] = qs;
+            zp_s[i] = (p.zp && t < p.M) ? p.zp[t] : 0;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(s_full);
@@ -313,6 +319,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         // this row's weight scale and shift do not depend on the preceding kernel: fetched now, used in the epilogue
         float alpha_row = n0 + row < p.N ? __ldg(p.alpha + n0 + row) : 0.f;
         float mu_row = (p.mu && n0 + row < p.N) ? __ldg(p.mu + n0 + row) : 0.f;
+        const int32_t rs_row = (p.zp && n0 + row < p.N) ? __ldg(p.rowsum + n0 + row) : 0;
         // pinned in registers: left alone, the compiler re-issues the global loads where the values are used
         asm volatile("" : "+f"(alpha_row), "+f"(mu_row));
         if (lowrank_here) {
@@ -422,21 +429,22 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 }
                 // the chunk's scales and code sums go to registers first: the tile stores below may alias them as far as
                 // the compiler knows, and a load behind every store would serialise the loop
-                float sc[16]; int32_t qs[16];
+                float sc[16]; int32_t qs[16], zp[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) { sc[j] = scale_s[16 * c + j]; qs[j] = qsum_s[16 * c + j]; }
+                for (int j = 0; j < 16; ++j) { sc[j] = scale_s[16 * c + j]; qs[j] = qsum_s[16 * c + j]; zp[j] = zp_s[16 * c + j]; }
                 // branch-free per element (rows beyond N and tokens beyond M produce values nobody stores):
                 // a branch per element costs more than the arithmetic it would skip
                 if (dbg && valid_row) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (t0 + 16 * c + j < M_) dbg[(int64_t)(t0 + 16 * c + j) * N_ + n] = -((int32_t)v[j] >> 6) - qs[j];
+                        if (t0 + 16 * c + j < M_) dbg[(int64_t)(t0 + 16 * c + j) * N_ + n] = -((int32_t)v[j] >> 6) - qs[j] - zp[j] * rs_row;
                 }
                 if (single) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const float lr = lowrank_here ? __uint_as_float(l[j]) : 0.f;
-                        const float y = finish_value((int32_t)v[j], lr, __fmul_rn(alpha_n, sc[j]), __fmul_rn(mu_n, sc[j]), qs[j]);
+                        const float y = finish_value((int32_t)v[j], lr, __fmul_rn(alpha_n, sc[j]), __fmul_rn(mu_n, sc[j]), qs[j],
+                                                     zp[j] * rs_row, p.K * zp[j]);
                         otile[(16 * c + j) * kRowsPerCta + row] = __float2bfloat16_rn(y);      // [token][row]
                     }
                 } else if (L::can_split) {
@@ -500,9 +508,10 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 for (int j = 0; j < 4; ++j) {
                     float y = 0.f;
                     if (n + j < p.N) {
+                        const int32_t zr = p.zp ? zp_s[tt] * p.rowsum[n + j] : 0;
                         y = finish_value(d[j], l4[j], __fmul_rn(p.alpha[n + j], scale_s[tt]),
-                                         p.mu ? __fmul_rn(p.mu[n + j], scale_s[tt]) : 0.f, qsum_s[tt]);
-                        if (p.acc_debug) p.acc_debug[(int64_t)(t0 + tt) * p.N + n + j] = -(d[j] >> 6) - qsum_s[tt];
+                                         p.mu ? __fmul_rn(p.mu[n + j], scale_s[tt]) : 0.f, qsum_s[tt], zr, p.K * zp_s[tt]);
+                        if (p.acc_debug) p.acc_debug[(int64_t)(t0 + tt) * p.N + n + j] = -(d[j] >> 6) - qsum_s[tt] - zr;
                     }
                     y4[j] = __float2bfloat16_rn(y);
                 }
@@ -563,7 +572,8 @@ static int launch_umma_t(const CUtensorMap& wm, const CUtensorMap& bm, const CUt
 
 bool umma_supports(int64_t M, int64_t K, int64_t N, int r, int bits) {
     // the tensor core sums -128 * code over the set sign bits: |D| <= 128 * K * qmax must fit the int32 accumulator
-    const int64_t qmax = ((int64_t)1 << (bits - 1)) - 1;
+    // (asymmetric codes reach -2^(b-1), one step further than the symmetric ones)
+    const int64_t qmax = (int64_t)1 << (bits - 1);
     return M > 0 && N > 0 && K % 128 == 0 && 128 * K * qmax < ((int64_t)1 << 31) && r <= kLowrankPad &&
            M * N < (int64_t)1 << 31 && M < (int64_t)1 << 30 && encode_tiled_fn() != nullptr;
 }
@@ -636,7 +646,7 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
 
     UmmaParams p{};
     p.M = M; p.N = N; p.K = K; p.total_units = units; p.splits = split; p.r = a.r;
-    p.scales = a.scales; p.qsum = a.qsum; p.alpha = a.alpha; p.mu = a.mu; p.U = (const __nv_bfloat16*)a.U;
+    p.scales = a.scales; p.qsum = a.qsum; p.alpha = a.alpha; p.mu = a.mu; p.zp = a.zp; p.rowsum = a.rowsum; p.U = (const __nv_bfloat16*)a.U;
     p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug; p.status = a.status;
 
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);

@@ -168,7 +168,7 @@ int launch_prepare_okt(const OktGeom& g, const float* P1, const float* P2, void*
 struct OktKernelParams {
     OktGeom g;
     int64_t M;
-    int bits;
+    int bits, asym;
     int n_problems;
     int clusters_per_problem;       // cluster i of a problem takes tokens i, i + clusters_per_problem, ...
     int rot_first, rot_ctas;        // rotation CTAs are blocks [rot_first, rot_first + rot_ctas)
@@ -251,8 +251,10 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 10) + 1;
     int* red_sum = reinterpret_cast<int*>(bars + 11);
-    float* red_max = reinterpret_cast<float*>(bars + 12);        // [kOktAluWarps]
-    float* slots = red_max + kOktAluWarps;                       // [2][8] absmax per CTA of the cluster, by token parity
+    float* red_max = reinterpret_cast<float*>(bars + 12);        // [16] largest value (symmetric: largest magnitude) per ALU warp
+    float* slots = red_max + 16;                                 // [2][8] the same per CTA of the cluster, by token parity
+    float* red_min = slots + 16;                                 // [16], [2][8]: smallest value (asymmetric quantiser only)
+    float* slots_min = red_min + 16;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int D = g.dt_count * g.cs_count;
@@ -397,6 +399,7 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
         const bool quarter_valid = q * 32 < rows;      // warp-uniform: a quarter without valid lanes only keeps the protocol
         const int d = d0 + lane_d;
         const int qmax = (1 << (p.bits - 1)) - 1;
+        const bool asym = p.asym != 0;
         const int chunks_b = n1p >> 4, chunks_d = ncols >> 4;
         bool failed = false;
         bool dep_waited = false;
@@ -437,7 +440,7 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             //      handed back at once, so that the next token's stage A runs under the rest of this one
             if (!failed && !warp_wait(d2_full, ph, abort_flag)) { give_up(p.status, abort_flag, 0x71); failed = true; }
             uint32_t yv[kOktChunksD][16];
-            float amax = 0.f;
+            float amax = 0.f, vmin = 0.f;                       // asymmetric: amax holds the largest value, zero included
             if (!failed && quarter_valid) {
                 tc_fence_after();
 #pragma unroll
@@ -456,33 +459,52 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                         const int cols_left = g.n1 - (c0 + 16 * ch);
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
-                            if (lane_valid && i < cols_left) amax = fmaxf(amax, fabsf(__uint_as_float(yv[j][i])));
+                            if (lane_valid && i < cols_left) {
+                                const float v = __uint_as_float(yv[j][i]);
+                                amax = fmaxf(amax, asym ? v : fabsf(v));
+                                vmin = fminf(vmin, v);
+                            }
                     }
                 }
             }
             amax = warp_max(amax);
-            if (lane == 0) red_max[warp - 2] = amax;
+            vmin = -warp_max(-vmin);
+            if (lane == 0) { red_max[warp - 2] = amax; red_min[warp - 2] = vmin; }
             // one decision for all ALU warps: a warp that gave up must not leave the others alone at a barrier
             if (alu_barrier_or(failed || *abort_flag != 0)) break;
-            amax = 0.f;
+            amax = 0.f; vmin = 0.f;
 #pragma unroll
-            for (int wi = 0; wi < kOktAluWarps; ++wi) amax = fmaxf(amax, red_max[wi]);
+            for (int wi = 0; wi < kOktAluWarps; ++wi) { amax = fmaxf(amax, red_max[wi]); vmin = fminf(vmin, red_min[wi]); }
             if (D > 1) {
                 const int par = it & 1;
                 if (e < D) {
                     // this CTA's absmax into slot [par][rank] of CTA e, then one arrival on that CTA's barrier
                     st_shared_cluster_u32(map_shared_rank(smem_u32(slots + par * 8 + rank), (uint32_t)e), __float_as_uint(amax));
+                    st_shared_cluster_u32(map_shared_rank(smem_u32(slots_min + par * 8 + rank), (uint32_t)e), __float_as_uint(vmin));
                     mbar_arrive_remote(map_shared_rank(smem_u32(&xbar[par]), (uint32_t)e));
                 }
                 if (!warp_wait_cluster(&xbar[par], (uint32_t)((it >> 1) & 1), abort_flag)) { give_up(p.status, abort_flag, 0x72); failed = true; }
                 if (!failed) {
-                    amax = 0.f;
-                    for (int c = 0; c < D; ++c) amax = fmaxf(amax, slots[par * 8 + c]);
+                    amax = 0.f; vmin = 0.f;
+                    for (int c = 0; c < D; ++c) { amax = fmaxf(amax, slots[par * 8 + c]); vmin = fminf(vmin, slots_min[par * 8 + c]); }
                 }
             }
-            float inv, scale;
-            if (amax == 0.f) { inv = 0.f; scale = 1.f; }
-            else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
+            // symmetric: codes in [-qmax, qmax] around zero.  Asymmetric (Sec. 4.1): u = rne(y * inv) + zero in [0, 2^b - 1]
+            // with an integer zero point; what is stored is u - 2^(b-1) (+ the caller's bias), so that it fits int8.
+            float inv, scale, zero_f = 0.f, lo_c = -(float)qmax, hi_c = (float)qmax, half_f = 0.f;
+            if (!asym) {
+                if (amax == 0.f) { inv = 0.f; scale = 1.f; }
+                else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
+            } else {
+                const float levels = (float)((1 << p.bits) - 1);
+                const float range = __fsub_rn(amax, vmin);
+                if (range == 0.f) { inv = 0.f; scale = 1.f; }
+                else { inv = __fdiv_rn(levels, range); scale = __fdiv_rn(range, levels); }
+                const float tz = __fmul_rn(-vmin, inv);
+                zero_f = fminf(fmaxf(__fadd_rn(__fadd_rn(tz, 12582912.f), -12582912.f), 0.f), levels);
+                lo_c = 0.f; hi_c = levels; half_f = (float)(1 << (p.bits - 1));
+            }
+            const float store_shift = (float)pr.code_bias - half_f;
             // nothing is stored to global memory before the preceding kernel of the stream has completed
             if (!dep_waited) { griddep_wait(); dep_waited = true; }
             // ---- codes.  Rounding to nearest-even by adding 1.5 * 2^23 (the code is then the low byte of the sum's bit
@@ -493,7 +515,6 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             int8_t* ct = pr.codes + t * (int64_t)g.K;
             if (!failed && quarter_valid) {
                 const bool interleave = pr.codes_layout != 0;
-                const float fq = (float)qmax;
 #pragma unroll
                 for (int j = 0; j < kOktChunksD; ++j) {
                     const int ch = part + j * kOktAluPerQuarter;
@@ -503,11 +524,12 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                         uint32_t code[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            // products beyond +-qmax only come from rounding of the reciprocal: clamp, then round
-                            const float tq = fminf(fmaxf(__fmul_rn(__uint_as_float(yv[j][i]), inv), -fq), fq);
-                            const float magic = __fadd_rn(tq, 12582912.f);
-                            fsum += (lane_valid && i < cols_left) ? __fadd_rn(magic, -12582912.f) : 0.f;
-                            code[i] = __float_as_uint(magic);
+                            // round (adding 1.5 * 2^23 leaves the nearest-even integer in the low mantissa bits), shift by the
+                            // zero point, clamp (products beyond the range only come from rounding of the reciprocal)
+                            const float rq = __fadd_rn(__fadd_rn(__fmul_rn(__uint_as_float(yv[j][i]), inv), 12582912.f), -12582912.f);
+                            const float u = fminf(fmaxf(rq + zero_f, lo_c), hi_c);
+                            fsum += (lane_valid && i < cols_left) ? u - half_f : 0.f;
+                            code[i] = __float_as_uint(__fadd_rn(u + store_shift, 12582912.f));
                         }
                         // one simple guarded store per element, so that the compiler predicates it instead of branching
                         if (stage) {
@@ -566,7 +588,10 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                     if (rank == 0)
                         for (int c = D; c < kQsumParts; ++c) pr.qsum[t * kQsumParts + c] = 0;
                 }
-                if (rank == 0) pr.scales[t] = scale;
+                if (rank == 0) {
+                    pr.scales[t] = scale;
+                    if (pr.zp) pr.zp[t] = (int)(zero_f + store_shift);
+                }
             }
             if (e == 0) *red_sum = 0;
         }
@@ -592,14 +617,14 @@ bool okt_accepts_x(const void* x, int64_t ldx) {
     return (reinterpret_cast<uintptr_t>(x) & 15) == 0 && ldx % 8 == 0 && encode_tiled_fn() != nullptr;
 }
 
-int launch_okt(const OktGeom& g, const void* x, int64_t M, int64_t ldx, int bits, int n_problems,
+int launch_okt(const OktGeom& g, const void* x, int64_t M, int64_t ldx, int bits, int asym, int n_problems,
                const OktProblem* problems, const OktLowrank* lowrank, uint32_t* status, cudaStream_t stream) {
     if (M == 0 || n_problems == 0) return BWLA_OK;
     if (n_problems > kOktMaxProblems || M >= ((int64_t)1 << 31)) return BWLA_ERR_INVALID_ARG;
     const int sms = sm_count();
     if (sms <= 0) return BWLA_ERR_CUDA;
     OktKernelParams p{};
-    p.g = g; p.M = M; p.bits = bits; p.n_problems = n_problems; p.status = status;
+    p.g = g; p.M = M; p.bits = bits; p.asym = asym; p.n_problems = n_problems; p.status = status;
     const int D = g.dt_count * g.cs_count;
     size_t smem = (size_t)g.smem_bytes;
     int lr_total = 0;

@@ -29,6 +29,26 @@ __global__ void __launch_bounds__(256) pack_signs_kernel(const T* __restrict__ w
     }
 }
 
+// One warp per row: the number of +1 weights minus the number of -1 weights.
+__global__ void __launch_bounds__(256) row_sums_kernel(const uint32_t* __restrict__ packed, int64_t N, int64_t words,
+                                                       int32_t* __restrict__ rowsum) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= N) return;
+    int ones = 0;
+    for (int64_t w = lane; w < words; w += 32) ones += __popc(packed[row * words + w]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ones += __shfl_xor_sync(0xFFFFFFFFu, ones, o);
+    if (lane == 0) rowsum[row] = 2 * ones - (int32_t)(words * 32);
+}
+
+int launch_row_sums(const uint32_t* packed, int64_t N, int64_t K, int32_t* rowsum, cudaStream_t stream) {
+    if (N == 0) return BWLA_OK;
+    ProfScope prof(kProfPack, stream);
+    row_sums_kernel<<<(unsigned)((N + 7) / 8), 256, 0, stream>>>(packed, N, K / 32, rowsum);
+    return after_launch();
+}
+
 int launch_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw, uint32_t* packed,
                       cudaStream_t stream) {
     const int64_t words = K / 32;

@@ -312,11 +312,11 @@ def test_a_set_status_word_is_reported_cleared_and_the_next_call_is_clean(bwla):
 
 
 def test_accumulator_range_guard_of_the_tensor_core_path(bwla):
-    """The tensor core sums -128 * code over the set sign bits; where 128 * K * qmax could leave int32 the shape must
-    go to the simple kernel."""
-    assert bwla.bwla_chosen_path(16, 132096, 1024, 0, 8) == bwla.BWLA_PATH_I8      # 128 * K * 127 < 2^31
-    assert bwla.bwla_chosen_path(16, 132224, 1024, 0, 8) == bwla.BWLA_PATH_SIMPLE  # ... > 2^31
-    assert bwla.bwla_chosen_path(16, 132224, 1024, 0, 6) == bwla.BWLA_PATH_I8      # qmax = 31 leaves room
+    """The tensor core sums -128 * code over the set sign bits; where 128 * K * 2^(b-1) could leave int32 the shape
+    must go to the simple kernel."""
+    assert bwla.bwla_chosen_path(16, 130944, 1024, 0, 8) == bwla.BWLA_PATH_I8      # 128 * K * 128 < 2^31
+    assert bwla.bwla_chosen_path(16, 131072, 1024, 0, 8) == bwla.BWLA_PATH_SIMPLE  # ... = 2^31
+    assert bwla.bwla_chosen_path(16, 131072, 1024, 0, 6) == bwla.BWLA_PATH_I8      # 6-bit codes leave room
 
 
 def test_empty_batch_and_argument_errors(bwla):

@@ -116,3 +116,79 @@ def test_grouped_layers_match_the_oracle_layer_by_layer(bwla, idxs, M):
     assert bwla.bwla_check_status(ws) == 0
     for a, b in zip(outs, outs2):
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+# ------------------------------------------------------------------------------------------------
+# per-token asymmetric quantiser (the paper's stated setting, Sec. 4.1)
+# ------------------------------------------------------------------------------------------------
+def _check_asym_codes(u, s, z, Y, bits):
+    """GPU codes / scales / zero points against the oracle's fp64 definition: what a code stands for, u - z, must agree
+    except at flagged near-ties (+-1); where the zero point itself sat on a rounding boundary the two may be shifted
+    against each other, which only shows at the clamped ends of the range."""
+    ref = oracle.quantize_asym(Y, bits, "f64")
+    L = (1 << bits) - 1
+    window = oracle.near_tie_window_asym(bits)
+    r_gpu = u.astype(np.int32) - z.astype(np.int32)[:, None]
+    r_ref = ref["codes"].astype(np.int32) - ref["zeros"].astype(np.int32)[:, None]
+    bad = r_gpu != r_ref
+    assert np.all(np.abs(r_gpu - r_ref)[bad] == 1), "a code differs from the oracle by more than one step"
+    zero_moved = z != ref["zeros"]
+    assert np.all(ref["dist_zero"][zero_moved] <= window), "a zero point differs away from a rounding boundary"
+    at_clamp = (ref["codes"] == 0) | (ref["codes"] == L) | (u == 0) | (u == L)
+    excused = (ref["dist"] <= window) | (zero_moved[:, None] & at_clamp)
+    assert not (bad & ~excused).any(), f"{int((bad & ~excused).sum())} code mismatches outside the near-tie window"
+    assert np.all(np.abs(s.astype(np.float64) - ref["scales"]) <= 2e-6 * ref["scales"])
+    return {"mismatches": int(bad.sum()), "near_ties": int((ref["dist"] <= window).sum()), "zero_moved": int(zero_moved.sum())}
+
+
+@pytest.mark.parametrize("n1,n2,M,bits", [(32, 32, 16, 6), (64, 80, 9, 6), (64, 80, 200, 8), (86, 128, 4, 4), (160, 160, 5, 6),
+                                         (160, 160, 80, 8), (4, 8, 5, 4)])
+def test_asymmetric_quantiser_stages_b_and_c(bwla, n1, n2, M, bits):
+    K = n1 * n2
+    shape = gen.small_shape(K, 32, n1, n2, 0, shape_id=n1 * 1000 + n2)
+    lay = gen.make_layer(0, shape, bits)
+    xb = gen.make_activations(0, shape, M)
+    xb[0] = gen.bf16_bits_from_f32(np.abs(gen.f32_from_bf16_bits(xb[0])))      # a row whose mean is far from zero
+    if M > 2:
+        xb[2] = 0                                                              # an all-zero row
+    L = _layer_for_rotation(bwla, lay, shape, bits)
+    u, s, z, y = bwla.bwla_layer_rotate_quant_asym(L, H.bf16_to_dev(xb), want_y=True)
+    torch.cuda.synchronize()
+    u, s, z, y = u.cpu().numpy(), s.cpu().numpy(), z.cpu().numpy(), y.cpu().numpy().astype(np.float64)
+    # (B) the oracle's quantiser with the fp32 decision rule on the GPU's own Y: bit for bit
+    q32 = oracle.quantize_asym(y, bits, "f32")
+    assert np.array_equal(q32["codes"], u) and np.array_equal(q32["zeros"], z) and np.array_equal(q32["scales"], s)
+    # (C) against the fp64 definition on the oracle's rotation
+    rep = _check_asym_codes(u, s, z, oracle.rotate(xb, lay.P1, lay.P2), bits)
+    print(f"\\n[asym {n1}x{n2} M={M} b={bits}] {rep}")
+
+
+@pytest.mark.parametrize("idxs,M,bits,path", [((0, 1, 2), 16, 6, None), ((4, 5), 3, 8, None), ((6,), 16, 6, None), ((3,), 130, 6, None),
+                                              ((1,), 2, 6, "bitplane"), ((1,), 5, 8, "simple")])
+def test_asymmetric_layers_match_the_oracle(bwla, idxs, M, bits, path):
+    shapes = [gen.CONFIG_SHAPES[2][i] for i in idxs]
+    lays = [gen.make_layer(2, sh, bits, direct_words=True, with_mu=(i == 0)) for i, sh in enumerate(shapes)]
+    xb = gen.make_activations(2, shapes[0], M)
+    xb[0] = gen.bf16_bits_from_f32(np.abs(gen.f32_from_bf16_bits(xb[0])))
+    dls = [H.DeviceLayer(l, bwla) for l in lays]
+    layers = [bwla.Layer(d.P1, d.P2, bits, d.packed, d.alpha, d.U, d.V, d.mu, asymmetric=True) for d in dls]
+    if path:
+        bwla.bwla_force_path({"bitplane": bwla.BWLA_PATH_BITPLANE, "simple": bwla.BWLA_PATH_SIMPLE}[path])
+    try:
+        ws = bwla.new_group_workspace(layers, M)
+        outs = bwla.bwla_w1ax_linear_group(layers, H.bf16_to_dev(xb), workspace=ws)
+        assert bwla.bwla_check_status(ws) == 0
+    finally:
+        bwla.bwla_force_path(bwla.BWLA_PATH_AUTO)
+    for lay, d, out in zip(lays, dls, outs):
+        ref = oracle.linear_asym(xb, lay.P1, lay.P2, bits, d.packed_host, lay.alpha, lay.U, lay.V, lay.mu)
+        # a code one step off at a near-tie moves the token's outputs by (|alpha| + |mu|) * s_t: the standalone entry
+        # gives this layer's codes (same kernel, same arithmetic)
+        u, s, z, _ = bwla.bwla_layer_rotate_quant_asym(layers[lays.index(lay)], H.bf16_to_dev(xb))
+        r_gpu = u.cpu().numpy().astype(np.int32) - z.cpu().numpy().astype(np.int32)[:, None]
+        r_ref = ref["codes"].astype(np.int32) - ref["zeros"].astype(np.int32)[:, None]
+        flips = np.abs(r_gpu - r_ref).sum(axis=1).astype(np.float64)
+        per_row = np.abs(lay.alpha.astype(np.float64)) + (0.0 if lay.mu is None else np.abs(lay.mu.astype(np.float64)))
+        slack = flips[:, None] * per_row[None, :] * ref["scales"].astype(np.float64)[:, None]
+        rep = H.check_output(H.bf16_to_host(out), ref["y"], step_slack=slack)
+        assert rep["rel_l2"] <= 2e-3
