@@ -77,15 +77,19 @@ bool okt_geometry(int n1, int n2, OktGeom* out) {
     g.atom2 = pick_atom(n2, &g.n2p);
     g.atom1 = pick_atom(n1, &g.n1p);
     g.dt_count = n2 > 128 ? 2 : 1;
-    g.dt_rows = g.dt_count == 1 ? n2 : round_up_int((n2 + 1) / 2, 8);
     g.x_bytes = g.n1p * g.n2p * 2;
-    g.p2t_bytes = 3 * g.dt_rows * g.n2p * 2;
     int tc = 32;
     while (tc < (5 * g.n1p + 1) / 2) tc *= 2;
     if (tc > 512) return false;
     g.tmem_cols = tc;
     const int chunks = g.n1p / 16;
+    // Two lane tiles: the boundary on a multiple of 32 rows when that fits (every CTA then owns whole groups of 32 codes
+    // and stores them wide), else on a multiple of 8.
+    for (int align = (g.dt_count == 2 && n2 % 32 == 0) ? 32 : 8; align >= 8; align = (align == 32 ? 8 : 0))
     for (int cs = 1; cs <= 4; cs *= 2) {
+        g.dt_rows = g.dt_count == 1 ? n2 : round_up_int((n2 + 1) / 2, align);
+        if (g.dt_count == 2 && g.dt_rows >= n2) continue;
+        g.p2t_bytes = 3 * g.dt_rows * g.n2p * 2;
         const int per = (chunks + cs - 1) / cs;
         if (cs > 1 && (cs - 1) * per >= chunks) continue;       // a slab would be empty
         g.cs_count = cs;
@@ -95,7 +99,9 @@ bool okt_geometry(int n1, int n2, OktGeom* out) {
         g.p1t_off = round_up_int(g.p2t_bytes, 1024);
         g.x_off = g.p1t_off + round_up_int(g.p1t_bytes, 1024);
         // one CTA per token: the codes are put together in shared memory and leave as 128-bit stores
-        g.stage_bytes = (g.dt_count == 1 && cs == 1) ? round_up_int(g.K, 16) : 0;
+        // the codes a CTA produces for a token are put together in shared memory and leave as wide stores: the whole
+        // token when one CTA owns it, else the CTA's (column slab) x (lane tile) block, one run of dt_rows bytes per column
+        g.stage_bytes = (g.dt_count == 1 && cs == 1) ? round_up_int(g.K, 16) : round_up_int(g.cs_cols * g.dt_rows, 16);
         g.stage_off = g.x_off + round_up_int(g.x_bytes, 1024);
         g.bar_off = g.stage_off + round_up_int(g.stage_bytes, 1024);
         int total = g.bar_off + kOktBarBytes;
@@ -532,18 +538,13 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                             code[i] = __float_as_uint(__fadd_rn(u + store_shift, 12582912.f));
                         }
                         // one simple guarded store per element, so that the compiler predicates it instead of branching
-                        if (stage) {
-                            int8_t* dst = stage + k0;
+                        {
+                            // whole token: natural position k; part of a token: [column of the slab][lane of the tile]
+                            int8_t* dst = stage + (D == 1 ? k0 : 16 * ch * rows + lane_d);
+                            const int step = D == 1 ? g.n2 : rows;
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
-                                if (lane_valid && i < cols_left) dst[i * g.n2] = (int8_t)code[i];
-                        } else {
-                            const int word_sel = (k0 & 7) << 2;
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int k = k0 + i * g.n2;
-                                if (lane_valid && i < cols_left) ct[interleave ? ((k & ~31) | word_sel | ((k >> 3) & 3)) : k] = (int8_t)code[i];
-                            }
+                                if (lane_valid && i < cols_left) dst[i * step] = (int8_t)code[i];
                         }
                         if (pr.y_debug) {
                             float* yt = pr.y_debug + t * (int64_t)g.K + k0;
@@ -558,27 +559,53 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             local_sum = warp_sum(local_sum);
             if (lane == 0 && local_sum != 0) atomicAdd(red_sum, local_sum);
             alu_barrier();
-            if (stage && !failed) {
-                // The token's codes leave as 128-bit stores, one group of 32 per thread and step (K is a multiple of 32).
-                // Interleaved order: output word j of a group holds k = j, j + 8, j + 16, j + 24, i.e. byte j & 3 of the
-                // natural words j >> 2, 2 + (j >> 2), 4 + (j >> 2), 6 + (j >> 2).
+            if (!failed) {
+                // The codes leave as wide stores, one group of 32 consecutive k per thread and step.  Interleaved order:
+                // output word j of a group holds k = j, j + 8, j + 16, j + 24, i.e. byte j & 3 of the natural words j >> 2,
+                // 2 + (j >> 2), 4 + (j >> 2), 6 + (j >> 2).
                 const bool interleave = pr.codes_layout != 0;
-                for (int gi = e; gi < (g.K >> 5); gi += kOktAluThreads) {
-                    const uint4 lo = *reinterpret_cast<const uint4*>(stage + 32 * gi), hi = *reinterpret_cast<const uint4*>(stage + 32 * gi + 16);
-                    uint4 o0 = lo, o1 = hi;
-                    if (interleave) {
-                        const uint32_t n[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-                        uint32_t o[8];
+                auto put_group = [&](const int8_t* src, int8_t* dst) {       // src 8-byte aligned, dst 32-byte aligned
+                    const uint2* s2 = reinterpret_cast<const uint2*>(src);
+                    const uint2 a0 = s2[0], a1 = s2[1], a2 = s2[2], a3 = s2[3];
+                    const uint32_t n[8] = {a0.x, a0.y, a1.x, a1.y, a2.x, a2.y, a3.x, a3.y};
+                    uint32_t o[8];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const uint32_t ab = __byte_perm(n[j >> 2], n[2 + (j >> 2)], (uint32_t)(j & 3) | ((uint32_t)(4 + (j & 3)) << 4));
-                            const uint32_t cd = __byte_perm(n[4 + (j >> 2)], n[6 + (j >> 2)], (uint32_t)(j & 3) | ((uint32_t)(4 + (j & 3)) << 4));
-                            o[j] = __byte_perm(ab, cd, 0x5410);
-                        }
-                        o0 = make_uint4(o[0], o[1], o[2], o[3]); o1 = make_uint4(o[4], o[5], o[6], o[7]);
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t sel = (uint32_t)(j & 3) | ((uint32_t)(4 + (j & 3)) << 4);
+                        o[j] = interleave ? __byte_perm(__byte_perm(n[j >> 2], n[2 + (j >> 2)], sel),
+                                                        __byte_perm(n[4 + (j >> 2)], n[6 + (j >> 2)], sel), 0x5410)
+                                          : n[j];
                     }
-                    uint4* out = reinterpret_cast<uint4*>(ct + 32 * gi);
-                    out[0] = o0; out[1] = o1;
+                    uint4* out = reinterpret_cast<uint4*>(dst);
+                    out[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                    out[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                };
+                if (D == 1) {
+                    for (int gi = e; gi < (g.K >> 5); gi += kOktAluThreads) put_group(stage + 32 * gi, ct + 32 * gi);
+                } else {
+                    // this CTA's block: for every column c of the slab a run of `rows` codes at k = c * n2 + d0.  Whole
+                    // groups of 32 inside a run go out as above; the ends of a run share their group with a neighbouring
+                    // CTA and go out byte by byte.
+                    const int cols_here = min(ncols, g.n1 - c0);
+                    const int groups_per_run = (rows >> 5) + 2;
+                    for (int item = e; item < cols_here * groups_per_run; item += kOktAluThreads) {
+                        const int cl = item / groups_per_run, gi = item - cl * groups_per_run;
+                        const int k_begin = (c0 + cl) * g.n2 + d0, k_end = k_begin + rows;
+                        const int g_lo = (k_begin + 31) & ~31, g_hi = k_end & ~31;      // whole groups: [g_lo, g_hi)
+                        const int8_t* run = stage + cl * rows - k_begin;                 // run[k] for k in [k_begin, k_end)
+                        int b0, b1;                                                      // byte-wise part of this item
+                        if (gi == 0) { b0 = k_begin; b1 = min(g_lo, k_end); }
+                        else if (gi == groups_per_run - 1) { b0 = max(g_hi, g_lo); b1 = k_end; if (g_hi < g_lo) b0 = b1; }
+                        else {
+                            const int gk = g_lo + 32 * (gi - 1);
+                            if (gk + 32 <= g_hi) put_group(run + gk, ct + gk);
+                            b0 = b1 = 0;
+                        }
+                        for (int k = b0; k < b1; ++k) {
+                            const int kl = k & 31;
+                            ct[interleave ? ((k & ~31) | ((kl & 7) << 2) | (kl >> 3)) : k] = run[k];
+                        }
+                    }
                 }
             }
             if (e == 0 && !failed) {
