@@ -320,6 +320,82 @@ def cublas_bf16_context(shapes, layers, Ms, device, torch, distinct=8, reps=3):
     return out
 
 
+def run_per_shape(args):
+    """Every shape of workload configs 1-3 at its token counts and bit widths, one linear at a time: whole call (CUDA
+    events around a graph of calls over layers with distinct weights) and kernel-only times (events around each launch),
+    for the chosen contraction path and, up to four tokens, for the other one.  Prints a markdown table; not part of the
+    one-line benchmark contract."""
+    import torch
+    from paper_2605_00422_b200 import bwla
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    NL = 6                                            # layers with distinct sign words per shape (cold weights)
+    rows = []
+    print("| config | shape | bits | M | path | whole call us | prologue us | contraction us | GB/s (call bytes) | TOPS (2MKN) | "
+          "% of measured HBM | % of 2x burst bf16 | other path us |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for cfg in (1, 2, 3):
+        for sh in gen.CONFIG_SHAPES[cfg]:
+            for bits in gen.CONFIG_BITS[cfg]:
+                g = torch.Generator(device=device)
+                g.manual_seed(1000 * cfg + sh.shape_id)
+                P1 = torch.from_numpy(gen.orthogonal_f32(sh.n1, gen._rng(cfg, 0, sh.shape_id, gen.T_P1))).to(device)
+                P2 = torch.from_numpy(gen.orthogonal_f32(sh.n2, gen._rng(cfg, 0, sh.shape_id, gen.T_P2))).to(device)
+                alpha = torch.exp(-4.0 + 0.3 * torch.randn(sh.N, device=device, generator=g))
+                U = (0.01 * torch.randn(sh.N, sh.r, device=device, generator=g)).to(torch.bfloat16)
+                V = (0.01 * torch.randn(sh.r, sh.K, device=device, generator=g)).to(torch.bfloat16)
+                layers = []
+                for _ in range(NL):
+                    pk = torch.randint(-2 ** 31, 2 ** 31, (sh.N, sh.K // 32), dtype=torch.int64, device=device, generator=g).to(torch.int32)
+                    layers.append(bwla.Layer(P1, P2, bits, pk, alpha, U, V))
+                for M in gen.CONFIG_TOKENS[cfg]:
+                    x = student_t_activations(M, sh.K, device, torch, 99 + M)
+                    out = [torch.empty(M, sh.N, dtype=torch.bfloat16, device=device)]
+                    ws = torch.zeros(bwla.bwla_group_workspace_bytes([layers[0]], M), dtype=torch.uint8, device=device)
+
+                    def measure(path):
+                        bwla.bwla_force_path(path)
+                        try:
+                            run = lambda: [bwla.bwla_w1ax_linear_group([L], x, outs=out, workspace=ws) for L in layers]
+                            run()
+                            torch.cuda.synchronize()
+                            gr = torch.cuda.CUDAGraph()
+                            with torch.cuda.graph(gr):
+                                run()
+                            reps = 5 if M <= 512 else 2
+                            gr.replay()
+                            torch.cuda.synchronize()
+                            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                            e0.record()
+                            for _ in range(reps):
+                                gr.replay()
+                            e1.record()
+                            torch.cuda.synchronize()
+                            whole = e0.elapsed_time(e1) / reps / NL * 1e3
+                            bwla.bwla_profile_enable(True)
+                            run()
+                            prof = bwla.bwla_profile_collect()
+                            bwla.bwla_profile_enable(False)
+                            return whole, prof["prologue"][0] / NL * 1e3, prof["contraction"][0] / NL * 1e3
+                        finally:
+                            bwla.bwla_force_path(bwla.BWLA_PATH_AUTO)
+
+                    chosen = bwla.bwla_chosen_path(M, sh.K, sh.N, sh.r, bits)
+                    whole, pro, con = measure(bwla.BWLA_PATH_AUTO)
+                    other = ""
+                    if M <= 4:
+                        alt = bwla.BWLA_PATH_BITPLANE if chosen == bwla.BWLA_PATH_I8 else bwla.BWLA_PATH_I8
+                        other = "%.1f (%s)" % (measure(alt)[0], {2: "bit-plane", 3: "tcgen05"}[alt])
+                    gbs = call_bytes(sh, M) / (whole * 1e-6) / 1e9
+                    tops = call_ops(sh, M) / (whole * 1e-6) / 1e12
+                    name = {1: "simple", 2: "bit-plane", 3: "tcgen05 i8"}[chosen]
+                    print(f"| {cfg} | {sh.name} {sh.K}->{sh.N} | {bits} | {M} | {name} | {whole:.1f} | {pro:.1f} | {con:.1f} | {gbs:.0f} | "
+                          f"{tops:.1f} | {100 * gbs / peaks['hbm_gbs']:.1f} | {100 * tops / (2 * peaks['bf16_tflops']):.1f} | {other} |", flush=True)
+                del layers
+                torch.cuda.empty_cache()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -434,7 +510,11 @@ def run_ours(args):
                 "traffic": measured_traffic("decode", k_bytes / k_n) if k_n else None,
                 "launches_per_step": k_n, "avg_launch_us": (k_ms / k_n * 1e3) if k_n else None,
                 "algorithmic_bytes_per_launch": (k_bytes / k_n) if k_n else None,
-                "algorithmic_bytes_per_step": k_bytes}
+                "algorithmic_bytes_per_step": k_bytes,
+                # the same launches charged with the whole call's algorithmic bytes (sign bits, U and V, alpha, Kronecker
+                # factors, activations in, outputs out) instead of what the contraction kernel itself reads and writes
+                "achieved_with_call_bytes": (step_bytes / (k_ms * 1e-3) / 1e9) if k_ms > 0 else None,
+                "whole_step_frac": value / world / peaks["hbm_gbs"]}
     del graph
     spot = oracle_spot_check(stack, xs, M, bwla, torch) if (rank == 0 and not args.no_cpu_baseline) else None
 
@@ -450,6 +530,44 @@ def run_ours(args):
         decode_other[f"M{Mo}"] = {"value": world * bytes_o / (ms_o * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms_o,
                                   "status": bwla.bwla_check_status(ws_o)}
         del graph_o
+
+    # both contraction paths at one and four tokens (the bit-plane kernel takes at most four); AUTO picks per shape
+    decode_paths = {}
+    if not args.skip_extras:
+        for Mo in (1, 4):
+            xs_o, outs_o, ws_o = make_io(Mo)
+            for name, path in (("bitplane", bwla.BWLA_PATH_BITPLANE), ("i8", bwla.BWLA_PATH_I8)):
+                bwla.bwla_force_path(path)
+                try:
+                    graph_o, _ = capture(xs_o, outs_o, ws_o)
+                    ms_o = timed(graph_o.replay, 5, 3) / 5
+                finally:
+                    bwla.bwla_force_path(bwla.BWLA_PATH_AUTO)
+                bytes_o = args.layers * sum(call_bytes(sh, Mo) for sh in shapes)
+                decode_paths[f"M{Mo}_{name}"] = {"ms_per_step": ms_o, "value": world * bytes_o / (ms_o * 1e-3) / 1e9, "unit": "GB/s",
+                                                 "status": bwla.bwla_check_status(ws_o)}
+                del graph_o
+        decode_paths["M8"] = "the bit-plane kernel takes at most four tokens; see decode_other_batches for the tcgen05 path"
+        decode_paths["chosen"] = {f"M{Mo}": {sh.name: bwla.bwla_chosen_path(Mo, sh.K, sh.N, sh.r, BITS) for sh in shapes} for Mo in (1, 4, 8, 16)}
+
+    # the operating point of the paper's end-to-end figure (Sec. 4.4): W1A8 at batch 4, decode
+    w1a8 = None
+    if not args.skip_extras:
+        for row in stack:
+            for lin in row:
+                lin.layer = bwla.Layer(lin.P1, lin.P2, 8, lin.packed, lin.alpha, lin.U, lin.V)
+        torch.cuda.synchronize()
+        xs_8, outs_8, ws_8 = make_io(4)
+        graph_8, _ = capture(xs_8, outs_8, ws_8)
+        ms_8 = timed(graph_8.replay, 5, 3) / 5
+        bytes_8 = args.layers * sum(call_bytes(sh, 4) for sh in shapes)
+        w1a8 = {"workload": "same stack, 8-bit codes, 4 tokens (batch 4 decode)", "ms_per_step": ms_8,
+                "value": world * bytes_8 / (ms_8 * 1e-3) / 1e9, "unit": "GB/s", "status": bwla.bwla_check_status(ws_8)}
+        del graph_8
+        for row in stack:
+            for lin in row:
+                lin.layer = bwla.Layer(lin.P1, lin.P2, BITS, lin.packed, lin.alpha, lin.U, lin.V)
+        torch.cuda.synchronize()
 
     # ------------------------------ prefill ------------------------------
     prefill = None
@@ -523,7 +641,7 @@ def run_ours(args):
             "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
             "kernel_ms_per_step": {k: round(v[0], 4) for k, v in prof.items()},
             "cpu_baseline": cpu, "decode_other_batches": decode_other, "prefill": prefill, "device_status": status,
-            "parity_spot_check": spot, "cublas_bf16_context": cublas,
+            "parity_spot_check": spot, "cublas_bf16_context": cublas, "decode_paths": decode_paths, "w1a8_batch4": w1a8,
         }
         print(json.dumps(line))
     if world > 1:
@@ -543,9 +661,13 @@ def main():
     ap.add_argument("--prefill-layers", type=int, default=0, help="layers in the prefill step (0 = all)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cublas", action="store_true", help="skip the cuBLAS bf16 context measurement")
+    ap.add_argument("--skip-extras", action="store_true", help="skip the forced-path and W1A8 batch-4 decode steps")
+    ap.add_argument("--per-shape", action="store_true", help="time every shape of workload configs 1-3 on its own and print a table")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.per_shape:
+        run_per_shape(args)
     else:
         run_ours(args)
 

@@ -205,5 +205,8 @@ int launch_gemm_bitplane(const GemmArgs& a, cudaStream_t stream);
 // tcgen05 path with the fused epilogue.  codes_interleaved: int8 [M][K] in the interleaved order.
 bool umma_supports(int64_t M, int64_t K, int64_t N, int r, int bits);
 int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream);
+// More than 64 tokens: the same contraction in CTAs that stay on their SM and take tiles of 128 rows x 128 tokens in turn.
+bool umma_persistent_supports(int64_t M, int64_t K, int64_t N, int r);
+int launch_gemm_umma_persistent(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream);
 
 }  // namespace bwla

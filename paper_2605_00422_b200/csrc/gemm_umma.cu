@@ -606,6 +606,7 @@ static int choose_wide_splits(int tiles, int units, int narrow_splits, int sms) 
 // codes_interleaved: int8 [M][K] in the interleaved order.  a.Thl: bf16 [3][M][64], T = hi + mid + lo.
 int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream) {
     const int M = (int)a.M, N = (int)a.N, K = (int)a.K;
+    if (umma_persistent_supports(a.M, a.K, a.N, a.r)) return launch_gemm_umma_persistent(a, codes_interleaved, stream);
     const int n_tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
     const int row_tiles = (N + kRowsPerCta - 1) / kRowsPerCta;
     const int tok_tiles = (M + n_tok - 1) / n_tok;
