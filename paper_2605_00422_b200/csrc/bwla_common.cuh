@@ -141,8 +141,7 @@ struct OktGeom {
     int dt_count, dt_rows;  // tiles of the rows d of P2^T (= tensor-memory lanes) and rows per tile (a multiple of 8)
     int cs_count, cs_cols;  // slabs of the rows c of P1^T (= output columns) and columns per slab (a multiple of 16)
     int p2t_bytes, p1t_bytes, x_bytes;      // one tile of P2^T terms, one slab of P1^T terms, one token's X tile
-    int p1t_off, x_off, stage_off, bar_off; // shared-memory offsets (P2^T tile at 0)
-    int stage_bytes;                        // room for one token's codes when one CTA owns the whole token, else 0
+    int p1t_off, x_off, bar_off;            // shared-memory offsets (P2^T tile at 0)
     int tmem_cols, smem_bytes;
 };
 constexpr int kOktMaxProblems = 4;          // linears that share one x and are rotated by one launch

@@ -83,8 +83,8 @@ bool okt_geometry(int n1, int n2, OktGeom* out) {
     if (tc > 512) return false;
     g.tmem_cols = tc;
     const int chunks = g.n1p / 16;
-    // Two lane tiles: the boundary on a multiple of 32 rows when that fits (every CTA then owns whole groups of 32 codes
-    // and stores them wide), else on a multiple of 8.
+    // Two lane tiles: the boundary on a multiple of 32 rows when that fits (a warp's 32 code bytes of a column then fill
+    // one whole 32-byte sector), else on a multiple of 8.
     for (int align = (g.dt_count == 2 && n2 % 32 == 0) ? 32 : 8; align >= 8; align = (align == 32 ? 8 : 0))
     for (int cs = 1; cs <= 4; cs *= 2) {
         g.dt_rows = g.dt_count == 1 ? n2 : round_up_int((n2 + 1) / 2, align);
@@ -98,12 +98,7 @@ bool okt_geometry(int n1, int n2, OktGeom* out) {
         g.p1t_bytes = 3 * g.cs_cols * g.n1p * 2;
         g.p1t_off = round_up_int(g.p2t_bytes, 1024);
         g.x_off = g.p1t_off + round_up_int(g.p1t_bytes, 1024);
-        // one CTA per token: the codes are put together in shared memory and leave as 128-bit stores
-        // the codes a CTA produces for a token are put together in shared memory and leave as wide stores: the whole
-        // token when one CTA owns it, else the CTA's (column slab) x (lane tile) block, one run of dt_rows bytes per column
-        g.stage_bytes = (g.dt_count == 1 && cs == 1) ? round_up_int(g.K, 16) : round_up_int(g.cs_cols * g.dt_rows, 16);
-        g.stage_off = g.x_off + round_up_int(g.x_bytes, 1024);
-        g.bar_off = g.stage_off + round_up_int(g.stage_bytes, 1024);
+        g.bar_off = g.x_off + round_up_int(g.x_bytes, 1024);
         int total = g.bar_off + kOktBarBytes;
         // the MMAs of stage A read 128 rows of every block of P2^T terms, whatever the tile's row count: what lies
         // behind the last block must still be this CTA's shared memory
@@ -221,6 +216,36 @@ __device__ __forceinline__ bool warp_wait_cluster(uint64_t* bar, uint32_t parity
     return false;
 }
 
+// One term of a contraction: `atoms` K-atoms of STEPS k-steps (16 elements, 32 bytes = 2 descriptor units) each, both
+// operands in shared memory, blocks of blk_a / blk_b descriptor units per K-atom.  `clear` starts the accumulator afresh.
+template <int STEPS>
+__device__ __forceinline__ void issue_term_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t blk_a, uint32_t b_lo, uint32_t b_hi,
+                                              uint32_t blk_b, int atoms, uint32_t idesc, bool clear) {
+    if (clear) ptx::mma_f16_ss_words<false>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc);
+    else ptx::mma_f16_ss_words<true>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc);
+#pragma unroll
+    for (int s = 1; s < STEPS; ++s) ptx::mma_f16_ss_words<true>(d_tmem, a_lo + 2u * s, a_hi, b_lo + 2u * s, b_hi, idesc);
+    for (int at = 1; at < atoms; ++at) {
+        a_lo += blk_a; b_lo += blk_b;
+#pragma unroll
+        for (int s = 0; s < STEPS; ++s) ptx::mma_f16_ss_words<true>(d_tmem, a_lo + 2u * s, a_hi, b_lo + 2u * s, b_hi, idesc);
+    }
+}
+// The same with the A operand in tensor memory: 8 columns (16 bf16) per k-step.
+template <int STEPS>
+__device__ __forceinline__ void issue_term_ts(uint32_t d_tmem, uint32_t a_col, uint32_t b_lo, uint32_t b_hi, uint32_t blk_b, int atoms,
+                                              uint32_t idesc, bool clear) {
+    if (clear) ptx::mma_f16_ts_words<false>(d_tmem, a_col, b_lo, b_hi, idesc);
+    else ptx::mma_f16_ts_words<true>(d_tmem, a_col, b_lo, b_hi, idesc);
+#pragma unroll
+    for (int s = 1; s < STEPS; ++s) ptx::mma_f16_ts_words<true>(d_tmem, a_col + 8u * s, b_lo + 2u * s, b_hi, idesc);
+    for (int at = 1; at < atoms; ++at) {
+        a_col += 8u * STEPS; b_lo += blk_b;
+#pragma unroll
+        for (int s = 0; s < STEPS; ++s) ptx::mma_f16_ts_words<true>(d_tmem, a_col + 8u * s, b_lo + 2u * s, b_hi, idesc);
+    }
+}
+
 __global__ void __launch_bounds__(kOktThreads, 1)
 okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams p) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -291,7 +316,7 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
         for (int off = 0; off < g.p1t_bytes; off += 16384)
             tma_bulk_g2s(p1t + off, src1 + off, (uint32_t)min(16384, g.p1t_bytes - off), const_full);
         *abort_flag = 0;
-        *red_sum = 0;
+        red_sum[0] = 0; red_sum[1] = 0;
         mbar_init(x_full, 1);
         mbar_init(x_empty, 1);
         mbar_init(d1_full, 1);
@@ -355,8 +380,8 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             const uint32_t blk_x = (uint32_t)(n1p * g.atom2) >> 4;            // one K-atom block of X
             const uint32_t blk_p1 = (uint32_t)(g.cs_cols * g.atom1) >> 4;     // one (term, K-atom) block of P1^T
             const int steps2 = g.atom2 / 32, steps1 = g.atom1 / 32;           // MMAs (K = 16) per K-atom: 1, 2 or 4
-            const int ls2 = steps2 >> 1 == 2 ? 2 : steps2 >> 1, ls1 = steps1 >> 1 == 2 ? 2 : steps1 >> 1;   // log2
-            const int nk2 = atoms2 * steps2, nk1 = atoms1 * steps1;           // k-steps per term
+            const uint32_t lo_p2 = (uint32_t)dP2, hi_p2 = (uint32_t)(dP2 >> 32), lo_x = (uint32_t)dX, hi_x = (uint32_t)(dX >> 32),
+                           lo_p1 = (uint32_t)dP1, hi_p1 = (uint32_t)(dP1 >> 32);
             bool ok = wait_or_abort(const_full, 0, abort_flag);
             if (!ok) give_up(p.status, abort_flag, 0x61);
             for (int it = 0; it < ntok && ok; ++it) {
@@ -365,14 +390,11 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                 if (!wait_or_abort(x_full, ph, abort_flag)) { give_up(p.status, abort_flag, 0x63); break; }
                 tc_fence_after();
                 // stage A: the small terms first, so that the large partial sums meet as few additions as possible
-                // k-step q of a term lies in K-atom q >> ls (blocks blk apart), 32 bytes (2 units) per step inside the atom
                 for (int h = 2; h >= 0; --h) {
-                    const uint64_t da = dP2 + (uint64_t)((uint32_t)(h * atoms2) * blk_a);
-#pragma unroll 4
-                    for (int q = 0; q < nk2; ++q) {
-                        const uint32_t at = (uint32_t)(q >> ls2), in = (uint32_t)(q & (steps2 - 1)) << 1;
-                        mma_f16_ss(tm_d, da + (at * blk_a + in), dX + (at * blk_x + in), idesc_a, (h == 2 && q == 0) ? 0u : 1u);
-                    }
+                    const uint32_t a_lo = lo_p2 + (uint32_t)(h * atoms2) * blk_a;
+                    if (steps2 == 4) issue_term_ss<4>(tm_d, a_lo, hi_p2, blk_a, lo_x, hi_x, blk_x, atoms2, idesc_a, h == 2);
+                    else if (steps2 == 2) issue_term_ss<2>(tm_d, a_lo, hi_p2, blk_a, lo_x, hi_x, blk_x, atoms2, idesc_a, h == 2);
+                    else issue_term_ss<1>(tm_d, a_lo, hi_p2, blk_a, lo_x, hi_x, blk_x, atoms2, idesc_a, h == 2);
                 }
                 tc_commit(x_empty);
                 tc_commit(d1_full);
@@ -384,12 +406,10 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                     constexpr int hz_of[6] = {2, 0, 1, 1, 0, 0};
                     constexpr int hp_of[6] = {0, 2, 1, 0, 1, 0};
                     const uint32_t a_col = tm_a2 + (uint32_t)(hz_of[pair] * (n1p >> 1));
-                    const uint64_t db = dP1 + (uint64_t)((uint32_t)(hp_of[pair] * atoms1) * blk_p1);
-#pragma unroll 4
-                    for (int q = 0; q < nk1; ++q) {
-                        const uint32_t at = (uint32_t)(q >> ls1), in = (uint32_t)(q & (steps1 - 1)) << 1;
-                        mma_f16_ts(tm_d, a_col + 8u * q, db + (at * blk_p1 + in), idesc_c, (pair == 0 && q == 0) ? 0u : 1u);
-                    }
+                    const uint32_t b_lo = lo_p1 + (uint32_t)(hp_of[pair] * atoms1) * blk_p1;
+                    if (steps1 == 4) issue_term_ts<4>(tm_d, a_col, b_lo, hi_p1, blk_p1, atoms1, idesc_c, pair == 0);
+                    else if (steps1 == 2) issue_term_ts<2>(tm_d, a_col, b_lo, hi_p1, blk_p1, atoms1, idesc_c, pair == 0);
+                    else issue_term_ts<1>(tm_d, a_col, b_lo, hi_p1, blk_p1, atoms1, idesc_c, pair == 0);
                 }
                 tc_commit(d2_full);
             }
@@ -409,44 +429,68 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
         const int chunks_b = n1p >> 4, chunks_d = ncols >> 4;
         bool failed = false;
         bool dep_waited = false;
-        int8_t* stage = g.stage_bytes ? reinterpret_cast<int8_t*>(smem + g.stage_off) : nullptr;
+        // Stage B of one token: every chunk's read is requested while the one before it is split and written back.
+        auto stage_b = [&](uint32_t phb) {
+            if (!failed && !warp_wait(d1_full, phb, abort_flag)) { give_up(p.status, abort_flag, 0x70); failed = true; }
+            if (failed) return;
+            tc_fence_after();
+            if (quarter_valid) {
+                uint32_t v[16];
+                int ch = part;
+                if (ch < chunks_b) tmem_ld_32x16(tm_d + lane_addr + 16 * ch, v);
+                while (ch < chunks_b) {
+                    tc_wait_ld();
+                    float f[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(v[i]);
+                    const int nxt = ch + kOktAluPerQuarter;
+                    if (nxt < chunks_b) tmem_ld_32x16(tm_d + lane_addr + 16 * nxt, v);
+                    uint32_t th[8], tmid[8], tl[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) split3_pair(f[2 * i], f[2 * i + 1], th[i], tmid[i], tl[i]);
+                    tmem_st_32x8(tm_a2 + lane_addr + 8 * ch, th);
+                    tmem_st_32x8(tm_a2 + lane_addr + (n1p >> 1) + 8 * ch, tmid);
+                    tmem_st_32x8(tm_a2 + lane_addr + n1p + 8 * ch, tl);
+                    ch = nxt;
+                }
+                tc_wait_st();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(a2_full);
+        };
+        // The ALU warps run one stage ahead of themselves: stage B of token it + 1 sits in the middle of stage D of token
+        // it (after its accumulator has gone to registers and its absmax has been sent off), so that the second
+        // contraction of the next token, and the exchange of the absmax inside a cluster, run under the rounding and
+        // the stores of this one.
+        // every CTA of the cluster leaves its own part of the token's code sum; the consumer adds the parts
+        auto put_qsum = [&](int64_t tq, int parq) {
+            if (pr.qsum) {
+                pr.qsum[tq * kQsumParts + rank] = red_sum[parq];
+                if (rank == 0)
+                    for (int c = D; c < kQsumParts; ++c) pr.qsum[tq * kQsumParts + c] = 0;
+            }
+            red_sum[parq] = 0;
+        };
+        // Where element k of a token is stored: at k, or (interleaved layout) inside each group of 32 at byte 4 (k % 8) +
+        // (k % 32) / 8.  The codes go straight to global memory, one byte per lane: the 32 lanes of a warp fill one
+        // 32-byte sector per column (two halves where n2 is not a multiple of 32).  16 columns on, and 4 columns on,
+        // the position inside the group repeats (n2 is a multiple of 8), so four offsets per thread cover every column.
+        const bool interleave = pr.codes_layout != 0;
+        int off[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int k = (c0 + 16 * part) * g.n2 + d + r * g.n2, kl = k & 31;
+            off[r] = (interleave ? ((k & ~31) | ((kl & 7) << 2) | (kl >> 3)) : k) - r * g.n2;
+        }
+        if (ntok > 0) stage_b(0u);
         for (int it = 0; it < ntok; ++it) {
             const uint32_t ph = (uint32_t)(it & 1);
             const int64_t t = tok0 + (int64_t)it * p.clusters_per_problem;
-            // ---- stage B: every chunk's read is requested while the one before it is split and written back
-            if (!failed && !warp_wait(d1_full, ph, abort_flag)) { give_up(p.status, abort_flag, 0x70); failed = true; }
-            if (!failed) {
-                tc_fence_after();
-                if (quarter_valid) {
-                    uint32_t v[16];
-                    int ch = part;
-                    if (ch < chunks_b) tmem_ld_32x16(tm_d + lane_addr + 16 * ch, v);
-                    while (ch < chunks_b) {
-                        tc_wait_ld();
-                        float f[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) f[i] = __uint_as_float(v[i]);
-                        const int nxt = ch + kOktAluPerQuarter;
-                        if (nxt < chunks_b) tmem_ld_32x16(tm_d + lane_addr + 16 * nxt, v);
-                        uint32_t th[8], tmid[8], tl[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) split3_pair(f[2 * i], f[2 * i + 1], th[i], tmid[i], tl[i]);
-                        tmem_st_32x8(tm_a2 + lane_addr + 8 * ch, th);
-                        tmem_st_32x8(tm_a2 + lane_addr + (n1p >> 1) + 8 * ch, tmid);
-                        tmem_st_32x8(tm_a2 + lane_addr + n1p + 8 * ch, tl);
-                        ch = nxt;
-                    }
-                    tc_wait_st();
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(a2_full);
-            }
-            // ---- stage D: this warp's chunks of Y^T go to registers (both reads in flight at once) and the accumulator is
-            //      handed back at once, so that the next token's stage A runs under the rest of this one
+            // ---- stage D: this warp's chunks of Y^T go to registers (all reads in flight at once) and the accumulator is
+            //      handed back at once: the next token's stage A runs under the reduction below
             if (!failed && !warp_wait(d2_full, ph, abort_flag)) { give_up(p.status, abort_flag, 0x71); failed = true; }
             uint32_t yv[kOktChunksD][16];
-            float amax = 0.f, vmin = 0.f;                       // asymmetric: amax holds the largest value, zero included
             if (!failed && quarter_valid) {
                 tc_fence_after();
 #pragma unroll
@@ -457,39 +501,52 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             tc_fence_before();
             __syncwarp();
             if (lane == 0 && !failed) mbar_arrive(d_free);
+            // Columns beyond n1 are exact zeros (the padding rows of P1^T are), which changes neither reduction: the
+            // largest magnitude is at least zero and the asymmetric range contains zero by definition.  Lanes beyond the
+            // tile's rows hold anything and are masked once, after the loops.
+            float amax = 0.f, vmin = 0.f;                       // asymmetric: amax holds the largest value, zero included
             if (!failed && quarter_valid) {
+                float m0 = 0.f, m1 = 0.f, l0 = 0.f, l1 = 0.f;  // two chains each
 #pragma unroll
                 for (int j = 0; j < kOktChunksD; ++j) {
-                    const int ch = part + j * kOktAluPerQuarter;
-                    if (ch < chunks_d) {
-                        const int cols_left = g.n1 - (c0 + 16 * ch);
+                    if (part + j * kOktAluPerQuarter < chunks_d) {
+                        if (!asym) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            if (lane_valid && i < cols_left) {
-                                const float v = __uint_as_float(yv[j][i]);
-                                amax = fmaxf(amax, asym ? v : fabsf(v));
-                                vmin = fminf(vmin, v);
+                            for (int i = 0; i < 16; i += 2) {
+                                m0 = fmaxf(m0, fabsf(__uint_as_float(yv[j][i])));
+                                m1 = fmaxf(m1, fabsf(__uint_as_float(yv[j][i + 1])));
                             }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; i += 2) {
+                                const float a = __uint_as_float(yv[j][i]), c = __uint_as_float(yv[j][i + 1]);
+                                m0 = fmaxf(m0, a); m1 = fmaxf(m1, c);
+                                l0 = fminf(l0, a); l1 = fminf(l1, c);
+                            }
+                        }
                     }
                 }
+                if (lane_valid) { amax = fmaxf(m0, m1); vmin = fminf(l0, l1); }
             }
             amax = warp_max(amax);
-            vmin = -warp_max(-vmin);
+            if (asym) vmin = -warp_max(-vmin);
             if (lane == 0) { red_max[warp - 2] = amax; red_min[warp - 2] = vmin; }
             // one decision for all ALU warps: a warp that gave up must not leave the others alone at a barrier
             if (alu_barrier_or(failed || *abort_flag != 0)) break;
+            if (e == 0 && it > 0) put_qsum(t - p.clusters_per_problem, (it - 1) & 1);
             amax = 0.f; vmin = 0.f;
 #pragma unroll
             for (int wi = 0; wi < kOktAluWarps; ++wi) { amax = fmaxf(amax, red_max[wi]); vmin = fminf(vmin, red_min[wi]); }
+            const int par = it & 1;
+            if (D > 1 && e < D) {
+                // this CTA's absmax into slot [par][rank] of CTA e, then one arrival on that CTA's barrier
+                st_shared_cluster_u32(map_shared_rank(smem_u32(slots + par * 8 + rank), (uint32_t)e), __float_as_uint(amax));
+                st_shared_cluster_u32(map_shared_rank(smem_u32(slots_min + par * 8 + rank), (uint32_t)e), __float_as_uint(vmin));
+                mbar_arrive_remote(map_shared_rank(smem_u32(&xbar[par]), (uint32_t)e));
+            }
+            if (it + 1 < ntok) stage_b(ph ^ 1u);
             if (D > 1) {
-                const int par = it & 1;
-                if (e < D) {
-                    // this CTA's absmax into slot [par][rank] of CTA e, then one arrival on that CTA's barrier
-                    st_shared_cluster_u32(map_shared_rank(smem_u32(slots + par * 8 + rank), (uint32_t)e), __float_as_uint(amax));
-                    st_shared_cluster_u32(map_shared_rank(smem_u32(slots_min + par * 8 + rank), (uint32_t)e), __float_as_uint(vmin));
-                    mbar_arrive_remote(map_shared_rank(smem_u32(&xbar[par]), (uint32_t)e));
-                }
-                if (!warp_wait_cluster(&xbar[par], (uint32_t)((it >> 1) & 1), abort_flag)) { give_up(p.status, abort_flag, 0x72); failed = true; }
+                if (!failed && !warp_wait_cluster(&xbar[par], (uint32_t)((it >> 1) & 1), abort_flag)) { give_up(p.status, abort_flag, 0x72); failed = true; }
                 if (!failed) {
                     amax = 0.f; vmin = 0.f;
                     for (int c = 0; c < D; ++c) { amax = fmaxf(amax, slots[par * 8 + c]); vmin = fminf(vmin, slots_min[par * 8 + c]); }
@@ -513,38 +570,51 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             const float store_shift = (float)pr.code_bias - half_f;
             // nothing is stored to global memory before the preceding kernel of the stream has completed
             if (!dep_waited) { griddep_wait(); dep_waited = true; }
-            // ---- codes.  Rounding to nearest-even by adding 1.5 * 2^23 (the code is then the low byte of the sum's bit
-            //      pattern), clamping in fp32 before it: no float-to-integer conversions, which are slow instructions.
+            // ---- codes.  With B = 1.5 * 2^23 + an even integer, fl(v + B) = B + rne(v) for |v| < 2^22: one addition
+            //      rounds to nearest-even (the sum's ulp is 1, and ties go to an even sum, hence to an even rne(v)) and
+            //      leaves the integer in the low mantissa bits; no float-to-integer conversions, which are slow
+            //      instructions.  Everything added to the rounded product (zero point, shift of the stored code) goes
+            //      into B except its parity bit, which is added to the bit pattern.  The clamp acts on the sum (products
+            //      beyond the range only come from rounding of the reciprocal and of the zero point).  The stored byte
+            //      is the low byte of the pattern, and the patterns themselves are summed for the code sum: every one
+            //      is 0x4B400000 + the stored code.
             //      A CTA that owns the whole token collects the codes in shared memory in natural order (a warp writes 32
             //      consecutive bytes per column) and reorders them on the way out.
-            float fsum = 0.f;
+            const int shift_i = (int)(zero_f + store_shift);                 // small integer, exact
+            const uint32_t odd = (uint32_t)(shift_i & 1);
+            const float bias_even = 12582912.f + (float)(shift_i - (int)odd);
+            const float lo_b = 12582912.f + (lo_c + store_shift) - (float)odd, hi_b = 12582912.f + (hi_c + store_shift) - (float)odd;
+            uint32_t usum = 0u;
+            int counted = 0;
             int8_t* ct = pr.codes + t * (int64_t)g.K;
             if (!failed && quarter_valid) {
-                const bool interleave = pr.codes_layout != 0;
 #pragma unroll
                 for (int j = 0; j < kOktChunksD; ++j) {
                     const int ch = part + j * kOktAluPerQuarter;
-                    if (ch < chunks_d) {
-                        const int cols_left = g.n1 - (c0 + 16 * ch);
+                    const int cols_left = g.n1 - (c0 + 16 * ch);             // warp-uniform
+                    if (ch < chunks_d && cols_left > 0) {
                         const int k0 = (c0 + 16 * ch) * g.n2 + d;
-                        uint32_t code[16];
+                        int8_t* const cb = ct + (int64_t)(16 * kOktAluPerQuarter * j) * g.n2;
+                        if (cols_left >= 16) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            // round (adding 1.5 * 2^23 leaves the nearest-even integer in the low mantissa bits), shift by the
-                            // zero point, clamp (products beyond the range only come from rounding of the reciprocal)
-                            const float rq = __fadd_rn(__fadd_rn(__fmul_rn(__uint_as_float(yv[j][i]), inv), 12582912.f), -12582912.f);
-                            const float u = fminf(fmaxf(rq + zero_f, lo_c), hi_c);
-                            fsum += (lane_valid && i < cols_left) ? u - half_f : 0.f;
-                            code[i] = __float_as_uint(__fadd_rn(u + store_shift, 12582912.f));
-                        }
-                        // one simple guarded store per element, so that the compiler predicates it instead of branching
-                        {
-                            // whole token: natural position k; part of a token: [column of the slab][lane of the tile]
-                            int8_t* dst = stage + (D == 1 ? k0 : 16 * ch * rows + lane_d);
-                            const int step = D == 1 ? g.n2 : rows;
+                            for (int i = 0; i < 16; ++i) {
+                                const float sv = fminf(fmaxf(__fadd_rn(__fmul_rn(__uint_as_float(yv[j][i]), inv), bias_even), lo_b), hi_b);
+                                const uint32_t w = __float_as_uint(sv) + odd;
+                                usum += w;
+                                if (lane_valid) cb[off[i & 3] + i * g.n2] = (int8_t)w;
+                            }
+                            counted += 16;
+                        } else {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                if (lane_valid && i < cols_left) dst[i * step] = (int8_t)code[i];
+                            for (int i = 0; i < 16; ++i) {
+                                const float sv = fminf(fmaxf(__fadd_rn(__fmul_rn(__uint_as_float(yv[j][i]), inv), bias_even), lo_b), hi_b);
+                                const uint32_t w = __float_as_uint(sv) + odd;
+                                if (i < cols_left) {
+                                    usum += w;
+                                    if (lane_valid) cb[off[i & 3] + i * g.n2] = (int8_t)w;
+                                }
+                            }
+                            counted += cols_left;
                         }
                         if (pr.y_debug) {
                             float* yt = pr.y_debug + t * (int64_t)g.K + k0;
@@ -555,73 +625,19 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                     }
                 }
             }
-            int local_sum = (int)fsum;                            // a sum of at most 48 integers below 128: exact in fp32
+            // sum of (stored code - the caller's bias) over this lane's elements, in wrap-around arithmetic; the CTA's sum
+            // is collected in red_sum[par] and leaves after the next token's barrier (or the one behind the loop)
+            int local_sum = lane_valid ? (int)(usum - (uint32_t)counted * (0x4B400000u + (uint32_t)pr.code_bias)) : 0;
             local_sum = warp_sum(local_sum);
-            if (lane == 0 && local_sum != 0) atomicAdd(red_sum, local_sum);
-            alu_barrier();
-            if (!failed) {
-                // The codes leave as wide stores, one group of 32 consecutive k per thread and step.  Interleaved order:
-                // output word j of a group holds k = j, j + 8, j + 16, j + 24, i.e. byte j & 3 of the natural words j >> 2,
-                // 2 + (j >> 2), 4 + (j >> 2), 6 + (j >> 2).
-                const bool interleave = pr.codes_layout != 0;
-                auto put_group = [&](const int8_t* src, int8_t* dst) {       // src 8-byte aligned, dst 32-byte aligned
-                    const uint2* s2 = reinterpret_cast<const uint2*>(src);
-                    const uint2 a0 = s2[0], a1 = s2[1], a2 = s2[2], a3 = s2[3];
-                    const uint32_t n[8] = {a0.x, a0.y, a1.x, a1.y, a2.x, a2.y, a3.x, a3.y};
-                    uint32_t o[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t sel = (uint32_t)(j & 3) | ((uint32_t)(4 + (j & 3)) << 4);
-                        o[j] = interleave ? __byte_perm(__byte_perm(n[j >> 2], n[2 + (j >> 2)], sel),
-                                                        __byte_perm(n[4 + (j >> 2)], n[6 + (j >> 2)], sel), 0x5410)
-                                          : n[j];
-                    }
-                    uint4* out = reinterpret_cast<uint4*>(dst);
-                    out[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                    out[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                };
-                if (D == 1) {
-                    for (int gi = e; gi < (g.K >> 5); gi += kOktAluThreads) put_group(stage + 32 * gi, ct + 32 * gi);
-                } else {
-                    // this CTA's block: for every column c of the slab a run of `rows` codes at k = c * n2 + d0.  Whole
-                    // groups of 32 inside a run go out as above; the ends of a run share their group with a neighbouring
-                    // CTA and go out byte by byte.
-                    const int cols_here = min(ncols, g.n1 - c0);
-                    const int groups_per_run = (rows >> 5) + 2;
-                    for (int item = e; item < cols_here * groups_per_run; item += kOktAluThreads) {
-                        const int cl = item / groups_per_run, gi = item - cl * groups_per_run;
-                        const int k_begin = (c0 + cl) * g.n2 + d0, k_end = k_begin + rows;
-                        const int g_lo = (k_begin + 31) & ~31, g_hi = k_end & ~31;      // whole groups: [g_lo, g_hi)
-                        const int8_t* run = stage + cl * rows - k_begin;                 // run[k] for k in [k_begin, k_end)
-                        int b0, b1;                                                      // byte-wise part of this item
-                        if (gi == 0) { b0 = k_begin; b1 = min(g_lo, k_end); }
-                        else if (gi == groups_per_run - 1) { b0 = max(g_hi, g_lo); b1 = k_end; if (g_hi < g_lo) b0 = b1; }
-                        else {
-                            const int gk = g_lo + 32 * (gi - 1);
-                            if (gk + 32 <= g_hi) put_group(run + gk, ct + gk);
-                            b0 = b1 = 0;
-                        }
-                        for (int k = b0; k < b1; ++k) {
-                            const int kl = k & 31;
-                            ct[interleave ? ((k & ~31) | ((kl & 7) << 2) | (kl >> 3)) : k] = run[k];
-                        }
-                    }
-                }
+            if (lane == 0 && local_sum != 0 && !failed) atomicAdd(&red_sum[par], local_sum);
+            if (e == 0 && !failed && rank == 0) {
+                pr.scales[t] = scale;
+                if (pr.zp) pr.zp[t] = shift_i;
             }
-            if (e == 0 && !failed) {
-                // every CTA of the cluster leaves its own part of the token's code sum; the consumer adds the parts
-                if (pr.qsum) {
-                    pr.qsum[t * kQsumParts + rank] = *red_sum;
-                    if (rank == 0)
-                        for (int c = D; c < kQsumParts; ++c) pr.qsum[t * kQsumParts + c] = 0;
-                }
-                if (rank == 0) {
-                    pr.scales[t] = scale;
-                    if (pr.zp) pr.zp[t] = (int)(zero_f + store_shift);
-                }
-            }
-            if (e == 0) *red_sum = 0;
         }
+        // the last token's code sum
+        if (!alu_barrier_or(failed || *abort_flag != 0) && e == 0 && ntok > 0)
+            put_qsum(tok0 + (int64_t)(ntok - 1) * p.clusters_per_problem, (ntok - 1) & 1);
     }
     tc_fence_before();
     __syncthreads();
