@@ -5,6 +5,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <algorithm>
+
 #include "bwla.h"
 
 namespace bwla {
@@ -83,6 +85,15 @@ constexpr int kLrCounterWord = 4;
 
 __host__ __device__ inline int lowrank_cols(int r) { return r > kLowrankPad ? (r + 1) / 2 * 2 : kLowrankPad; }
 
+// T = V x for many tokens on the tensor cores (lowrank_umma.cu): whether it takes the problem, the bytes of partial sums
+// it needs in the workspace (0: none), and the launch for the problems of one group (all share x, M, K; every entry of
+// `lowrank` has V, Thl and, where partial sums are needed, lr_part set).
+struct OktLowrank;
+bool lowrank_umma_supports(int64_t M, int64_t K, int r);
+size_t lowrank_umma_part_bytes(int64_t M, int64_t K, int r);
+int launch_lowrank_umma(const void* x, int64_t M, int64_t K, int64_t ldx, int n_problems, const OktLowrank* lowrank,
+                        uint32_t* status, cudaStream_t stream);
+
 struct Workspace {
     size_t status, scales, zp, qsum, T, lr_part, codes, prep, total;
 };
@@ -100,7 +111,8 @@ inline Workspace workspace_layout(int64_t M, int64_t K, int64_t N, int r, int bi
     w.qsum = off;   off += align_up((size_t)M * 4 * kQsumParts, 256);
     const size_t lr_cols = (size_t)lowrank_cols(r);
     w.T = off;      off += align_up((size_t)M * lr_cols * 6, 256);     // bf16 [3][M][cols]
-    w.lr_part = off; off += r > 0 ? align_up((size_t)kLrKSplitMax * 16 * lr_cols * 4, 256) : 0;   // fp32 [KS][16][cols]
+    // partial sums of T: fp32 [KS][16][cols] for the few-token blocks, [tile][part][cols][128] for the tensor-core kernel
+    w.lr_part = off; off += r > 0 ? align_up(std::max((size_t)kLrKSplitMax * 16 * lr_cols * 4, lowrank_umma_part_bytes(M, K, r)), 256) : 0;
     w.codes = off;  off += align_up((size_t)M * (size_t)K, 256);
     w.prep = off;   off += with_prepared ? kOktPreparedMax : 0;
     (void)N; (void)bits;

@@ -671,10 +671,28 @@ int launch_okt(const OktGeom& g, const void* x, int64_t M, int64_t ldx, int bits
     const int D = g.dt_count * g.cs_count;
     size_t smem = (size_t)g.smem_bytes;
     int lr_total = 0;
+    // Many tokens: T = V x of all problems goes first, as a launch of its own on the tensor cores.  Every kernel of the
+    // chain waits for its predecessor before it ends, so the contraction still finds T complete.
+    bool lr_done[kOktMaxProblems] = {};
+    if (lowrank) {
+        OktLowrank batch[kOktMaxProblems];
+        int nb = 0;
+        for (int i = 0; i < n_problems; ++i)
+            if (lowrank[i].V && lowrank[i].r > 0 && lowrank[i].Thl && lowrank_umma_supports(M, g.K, lowrank[i].r) &&
+                (reinterpret_cast<uintptr_t>(lowrank[i].V) & 15) == 0 &&
+                (lowrank[i].lr_part || lowrank_umma_part_bytes(M, g.K, lowrank[i].r) == 0)) {
+                batch[nb++] = lowrank[i];
+                lr_done[i] = true;
+            }
+        if (nb > 0) {
+            int st = launch_lowrank_umma(x, M, g.K, ldx, nb, batch, status, stream);
+            if (st != BWLA_OK) return st;
+        }
+    }
     for (int i = 0; i < n_problems; ++i) {
         p.prob[i] = problems[i];
         p.lr_begin[i] = lr_total;
-        if (lowrank && lowrank[i].V && lowrank[i].r > 0 && lowrank[i].Thl) {
+        if (lowrank && !lr_done[i] && lowrank[i].V && lowrank[i].r > 0 && lowrank[i].Thl) {
             PrologueParams& lp = p.lr[i];
             lp.x = (const __nv_bfloat16*)x; lp.M = M; lp.K = g.K; lp.ldx = ldx;
             lp.V = (const __nv_bfloat16*)lowrank[i].V; lp.r = lowrank[i].r; lp.Thl = (__nv_bfloat16*)lowrank[i].Thl;
