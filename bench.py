@@ -34,8 +34,8 @@ from paper_2605_00422_b200 import inputs as gen  # noqa: E402
 # the hash of the kernel source the capture was taken from.  The ratio scales the average launch of the step; when the
 # kernel source has changed since, the figure is dropped (null).
 NCU_TRAFFIC = {
-    "decode": {"dram_bytes": 19921408, "algorithmic_bytes": 20670592,          # gate_proj launch, M = 16
-               "kernel_sha256": "8fdb1b724e6e02c96fb9ec3913a706469829eb71127ca3db28cab207383e01eb"},
+    "decode": {"dram_bytes": 19881984, "algorithmic_bytes": 20216896,          # gate_proj launch, M = 8
+               "kernel_sha256": "752765d413035336f74e818bfc69bd111d18a2b0ae11326877688097b5047279"},
 }
 
 METRIC = "W1A6 linear: decode HBM GB/s & prefill INT8 TOPS vs B200 roofline, Qwen3-32B"
@@ -336,7 +336,11 @@ def run_per_shape(args):
           "% of measured HBM | % of 2x burst bf16 | other path us |")
     print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for cfg in (1, 2, 3):
+        if args.cfg and cfg != args.cfg:
+            continue
         for sh in gen.CONFIG_SHAPES[cfg]:
+            if args.shape and sh.name != args.shape:
+                continue
             for bits in gen.CONFIG_BITS[cfg]:
                 g = torch.Generator(device=device)
                 g.manual_seed(1000 * cfg + sh.shape_id)
@@ -350,6 +354,8 @@ def run_per_shape(args):
                     pk = torch.randint(-2 ** 31, 2 ** 31, (sh.N, sh.K // 32), dtype=torch.int64, device=device, generator=g).to(torch.int32)
                     layers.append(bwla.Layer(P1, P2, bits, pk, alpha, U, V))
                 for M in gen.CONFIG_TOKENS[cfg]:
+                    if args.m and M != args.m:
+                        continue
                     x = student_t_activations(M, sh.K, device, torch, 99 + M)
                     out = [torch.empty(M, sh.N, dtype=torch.bfloat16, device=device)]
                     ws = torch.zeros(bwla.bwla_group_workspace_bytes([layers[0]], M), dtype=torch.uint8, device=device)
@@ -591,7 +597,7 @@ def run_ours(args):
         i8_peak = 2.0 * peaks["bf16_tflops"]
         prefill = {"metric": "prefill INT8 TOPS (2*M*K*N of the contraction / whole-step time)", "value": tops,
                    "unit": "TOPS", "M": Mp, "layers": Lp, "steps": steps_p, "ms_per_step": ms_p / steps_p, "clocks": clocks_p,
-                   "roofline": {"bound": "tensor", "kernel": "umma_w1a_kernel, prefill stack", "achieved": k_tops,
+                   "roofline": {"bound": "tensor", "kernel": "umma_w1a_persistent_kernel (tcgen05 kind::i8 contraction), prefill stack", "achieved": k_tops,
                                 "peak": i8_peak, "peak_source": peaks["source"] + " bf16 burst x 2 (int8:bf16 nominal ratio)",
                                 "unit": "TOP/s", "frac": (k_tops / i8_peak) if k_tops else None, "traffic": None,
                                 "frac_of_sustained": (k_tops / (2.0 * peaks["bf16_tflops_sustained"])) if k_tops else None,
@@ -663,6 +669,9 @@ def main():
     ap.add_argument("--no-cublas", action="store_true", help="skip the cuBLAS bf16 context measurement")
     ap.add_argument("--skip-extras", action="store_true", help="skip the forced-path and W1A8 batch-4 decode steps")
     ap.add_argument("--per-shape", action="store_true", help="time every shape of workload configs 1-3 on its own and print a table")
+    ap.add_argument("--shape", default=None, help="with --per-shape: only the shape of this name (e.g. q_gate)")
+    ap.add_argument("--cfg", type=int, default=0, help="with --per-shape: only this workload config (1, 2 or 3)")
+    ap.add_argument("--m", type=int, default=0, help="with --per-shape: only this token count")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
