@@ -141,6 +141,47 @@ void bwla_oracle_rotate(const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
     }
 }
 
+/*
+ * Final binarisation in the rotated coordinates (Alg. 2, last step, with Eq. 1-3): X = W_res R with R = P1 (x) P2,
+ * i.e. every row of W_res = W - M goes through the same map as an activation row, X_n = flatten(P1^T reshape(w_n) P2);
+ * then per output row n: mu_n = mean_k X_nk, alpha_n = mean_k |X_nk - mu_n|, bit_nk = (X_nk - mu_n > 0).
+ * (The centring matrix H of Alg. 2 is the subtraction of the row mean; the mean is kept as the row shift of Eq. 4.)
+ * W_res is fp32 [N][K], widened exactly.  X (fp64 [N][K]) is returned for the tests' near-zero window.
+ */
+void bwla_oracle_binarize(const float* W, int64_t N, int64_t K, const float* P1, int64_t n1, const float* P2, int64_t n2,
+                          double* X, double* mu, double* alpha, uint32_t* packed) {
+    int64_t words = K / 32;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t n = 0; n < N; ++n) {
+        double* Z = (double*)malloc(sizeof(double) * (size_t)K);
+        const float* w = W + n * K;
+        for (int64_t a = 0; a < n1; ++a)
+            for (int64_t d = 0; d < n2; ++d) {
+                double s = 0.0;
+                for (int64_t b = 0; b < n2; ++b) s += (double)w[a * n2 + b] * (double)P2[b * n2 + d];
+                Z[a * n2 + d] = s;
+            }
+        double* x = X + n * K;
+        for (int64_t c = 0; c < n1; ++c)
+            for (int64_t d = 0; d < n2; ++d) {
+                double s = 0.0;
+                for (int64_t a = 0; a < n1; ++a) s += (double)P1[a * n1 + c] * Z[a * n2 + d];
+                x[c * n2 + d] = s;
+            }
+        free(Z);
+        double m = 0.0;
+        for (int64_t k = 0; k < K; ++k) m += x[k];
+        m /= (double)K;
+        double dsum = 0.0;
+        for (int64_t k = 0; k < K; ++k) dsum += fabs(x[k] - m);
+        mu[n] = m;
+        alpha[n] = dsum / (double)K;
+        for (int64_t wd = 0; wd < words; ++wd) packed[n * words + wd] = 0u;
+        for (int64_t k = 0; k < K; ++k)
+            if (x[k] - m > 0.0) packed[n * words + (k >> 5)] |= (1u << (k & 31));
+    }
+}
+
 static double round_half_even(double t) {
     double f = floor(t);
     double d = t - f;

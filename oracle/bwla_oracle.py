@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "libbwla_oracle.so")
 __all__ = [
     "build", "num_threads", "kron_factor", "row_stats", "pack_signs", "pack_signs_bf16", "unpack_signs",
     "rotate", "quantize", "gemm", "lowrank", "epilogue", "linear", "bf16_round", "near_tie_window",
-    "quantize_asym", "gemm_asym", "linear_asym", "near_tie_window_asym",
+    "quantize_asym", "gemm_asym", "linear_asym", "near_tie_window_asym", "binarize",
 ]
 
 
@@ -111,6 +111,23 @@ def rotate(x_bits: np.ndarray, P1: np.ndarray, P2: np.ndarray) -> np.ndarray:
     Y = np.empty((M, K), np.float64)
     _L().bwla_oracle_rotate(_p(x_bits), i64(M), i64(K), i64(K), _p(P1), i64(n1), _p(P2), i64(n2), _p(Y))
     return Y
+
+
+def binarize(W: np.ndarray, P1: np.ndarray, P2: np.ndarray) -> Dict[str, np.ndarray]:
+    """Alg. 2, last step: rows of W_res (fp32 [N][K]) rotated, then Eq. 1-3 per row.  Returns X (fp64), mu, alpha,
+    packed."""
+    W = _c(W, np.float32)
+    P1 = _c(P1, np.float32)
+    P2 = _c(P2, np.float32)
+    N, K = W.shape
+    n1, n2 = P1.shape[0], P2.shape[0]
+    assert n1 * n2 == K and K % 32 == 0
+    X = np.empty((N, K), np.float64)
+    mu = np.empty(N, np.float64)
+    alpha = np.empty(N, np.float64)
+    packed = np.empty((N, K // 32), np.uint32)
+    _L().bwla_oracle_binarize(_p(W), i64(N), i64(K), _p(P1), i64(n1), _p(P2), i64(n2), _p(X), _p(mu), _p(alpha), _p(packed))
+    return {"X": X, "mu": mu, "alpha": alpha, "packed": packed}
 
 
 def quantize(Y: np.ndarray, bits: int, decision: str = "f64") -> Dict[str, np.ndarray]:

@@ -418,3 +418,60 @@ def test_asymmetric_layer_approaches_the_unquantised_product_with_more_bits():
         errs[bits] = (np.linalg.norm(ya - exact), np.linalg.norm(ys - exact))
     assert errs[6][0] < 0.4 * errs[4][0] and errs[8][0] < 0.4 * errs[6][0]
     assert all(errs[b][0] <= 1.05 * errs[b][1] for b in errs)
+
+
+# ----------------------------------------------------------------------------------------------
+# Final binarisation in the rotated coordinates (Alg. 2, last step; Eq. 1-3)
+# ----------------------------------------------------------------------------------------------
+def test_binarisation_recovers_rows_that_are_binary_in_the_rotated_coordinates():
+    """W_res = (mu + c * s) R^T with balanced signs: the rotated rows are mu + c s exactly (up to rounding), so the
+    oracle must return those signs, c and mu.  A rotation by R^T instead of R, or swapped factors, scrambles the rows."""
+    n1, n2, N = 4, 8, 6
+    K = n1 * n2
+    rng = np.random.default_rng(77)
+    P1, P2 = _orth(n1, 1), _orth(n2, 2)
+    R = np.kron(P1.astype(np.float64), P2.astype(np.float64))
+    s = np.tile(np.array([1.0, -1.0]), K // 2)[None, :].repeat(N, 0)
+    for n in range(N):
+        rng.shuffle(s[n])                                       # balanced: mean(s) = 0
+    c = rng.uniform(0.5, 2.0, N)
+    mu = rng.uniform(-0.3, 0.3, N)
+    X = mu[:, None] + c[:, None] * s
+    W = (X @ R.T).astype(np.float32)                            # W R = X up to the fp32 rounding of W
+    out = oracle.binarize(W, P1, P2)
+    np.testing.assert_allclose(out["X"], X, atol=5e-6)
+    np.testing.assert_allclose(out["mu"], mu, atol=2e-6)
+    np.testing.assert_allclose(out["alpha"], c, atol=2e-6)
+    assert np.array_equal(oracle.unpack_signs(out["packed"], K), s.astype(np.int8))
+
+
+def test_binarisation_with_identity_factors_is_equation_1_on_the_rows_themselves():
+    rng = np.random.default_rng(5)
+    N, n1, n2 = 5, 2, 16
+    K = n1 * n2
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    out = oracle.binarize(W, np.eye(n1, dtype=np.float32), np.eye(n2, dtype=np.float32))
+    assert np.array_equal(out["X"], W.astype(np.float64))
+    # a hand-written row: values 1, 2, 3, 6 repeated -> mean 3, mean |x - 3| = (2 + 1 + 0 + 3) / 4 = 1.5, signs - - - +
+    row = np.tile(np.array([1.0, 2.0, 3.0, 6.0], np.float32), K // 4)[None, :]
+    o2 = oracle.binarize(row, np.eye(n1, dtype=np.float32), np.eye(n2, dtype=np.float32))
+    assert o2["mu"][0] == 3.0 and o2["alpha"][0] == 1.5
+    assert np.array_equal(oracle.unpack_signs(o2["packed"], K)[0], np.tile(np.array([-1, -1, -1, 1], np.int8), K // 4))
+
+
+def test_binarisation_scale_minimises_the_reconstruction_error_of_the_rotated_row():
+    """For the signs and the shift the oracle returns, alpha = mean |x - mu| is the least-squares scale (1-D scan), and
+    the rotation keeps the row norms (orthogonal factors)."""
+    n1, n2, N = 8, 8, 4
+    rng = np.random.default_rng(9)
+    P1, P2 = _orth(n1, 3), _orth(n2, 4)
+    W = rng.standard_normal((N, n1 * n2)).astype(np.float32)
+    out = oracle.binarize(W, P1, P2)
+    np.testing.assert_allclose(np.linalg.norm(out["X"], axis=1), np.linalg.norm(W.astype(np.float64), axis=1), rtol=1e-6)
+    s = oracle.unpack_signs(out["packed"], n1 * n2).astype(np.float64)
+    for n in range(N):
+        x = out["X"][n] - out["mu"][n]
+        grid = out["alpha"][n] * np.linspace(0.5, 1.5, 2001)
+        errs = [np.sum((x - a * s[n]) ** 2) for a in grid]
+        assert abs(grid[int(np.argmin(errs))] - out["alpha"][n]) <= out["alpha"][n] * 1e-3
+        assert abs(np.mean(x)) < 1e-12
