@@ -400,6 +400,14 @@ int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const voi
             if (st != BWLA_OK) return st;
         }
     }
+    // Several contractions that all go to the small-batch tensor-core kernel run beside one another (GemmArgs::dep_mode).
+    bool siblings = count > 1 && M <= 64;
+    for (int i = 0; i < count; ++i) siblings = siblings && path[i] == BWLA_PATH_I8;
+    // each sibling plans for its share of the SMs (by row tiles) when all of them fit the device at once
+    int64_t tiles_total = 0;
+    for (int i = 0; i < count; ++i) tiles_total += (layers[i]->N + 127) / 128;
+    const int sms_all = sm_count();
+    const bool share = siblings && tiles_total <= sms_all;
     for (int i = 0; i < count; ++i) {
         const bwla_layer* L = layers[i];
         GemmArgs g{};
@@ -408,6 +416,8 @@ int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const voi
         g.zp = L->asym ? (int32_t*)(wbase[i] + ws[i].zp) : nullptr; g.rowsum = L->rowsum;
         g.Thl = L->r > 0 ? wbase[i] + ws[i].T : nullptr; g.U = L->U; g.r = L->r; g.out = outs[i]; g.ldo = ldos[i];
         g.acc_debug = nullptr; g.status = status;
+        g.dep_mode = siblings ? (i == 0 ? kDepHead : kDepSibling) : kDepChain;
+        g.sm_budget = share ? (int)(((int64_t)sms_all * ((L->N + 127) / 128)) / tiles_total) : 0;
         st = run_contraction(path[i], g, (int8_t*)(wbase[i] + ws[i].codes), s);
         if (st != BWLA_OK) return st;
     }

@@ -204,7 +204,14 @@ struct GemmArgs {
     int64_t ldo;
     int32_t* acc_debug;       // [M][N] or NULL
     uint32_t* status;         // workspace status words
+    // Contractions of a group that read the results of the same preceding kernel (the rotation launch): the first one
+    // (kDepHead) lets the next kernel of the stream start only once it has itself seen that kernel complete, so the
+    // others (kDepSibling) need not wait for their predecessor, a sibling, before they read: they run beside it.
+    // kDepChain: the ordinary chain (wait for the predecessor before reading its results).
+    int dep_mode;
+    int sm_budget;            // SMs this launch should plan for (0: all): siblings share the device
 };
+enum { kDepChain = 0, kDepHead = 1, kDepSibling = 2 };
 
 int launch_gemm_simple(const GemmArgs& a, cudaStream_t stream);
 

@@ -34,6 +34,8 @@
 // in-flight copies land, still takes part in the cluster barriers, frees its tensor memory and returns.
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "bwla_common.cuh"
 #include "umma_ptx.cuh"
 #include "umma_wait.cuh"
@@ -61,6 +63,7 @@ struct UmmaParams {
     __nv_bfloat16* out;          // [M][ldo] or NULL
     int64_t ldo;
     int32_t* acc_debug;          // [M][N] or NULL
+    int dep_mode;                // kDepChain / kDepHead / kDepSibling (bwla_common.cuh)
     uint32_t* status;
 };
 
@@ -176,8 +179,11 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_base_slot;
-    // the next kernel of the stream may start its own independent preamble now
-    griddep_launch_dependents();
+    // The next kernel of the stream may start its own independent preamble now.  The head of a group of sibling
+    // contractions holds this back until it has seen the kernel before it complete (warp 1 below): whoever starts after
+    // that may read that kernel's results without waiting for anything.
+    const bool dep_wait = p.dep_mode != kDepSibling;   // a sibling's inputs are complete before it starts
+    if (p.dep_mode != kDepHead) griddep_launch_dependents();
 
     if (warp == 0) {
         // ---------------- packed sign words: HBM -> shared memory (independent of the preceding kernel) ----------------
@@ -190,7 +196,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 // A stage that is not free yet is released by the expansion, which in the end waits for the preceding
                 // kernel's codes: the bounded wait starts counting once that kernel has finished.
                 if (!mbar_test_wait(&w_empty[ws], wph ^ 1)) {
-                    griddep_wait();
+                    if (dep_wait) griddep_wait();
                     if (!wait_or_abort(&w_empty[ws], wph ^ 1, abort_flag)) { give_up(p.status, abort_flag, 0x10); break; }
                 }
                 mbar_expect_tx(&w_full[ws], L::w_bytes);
@@ -201,7 +207,8 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
         }
     } else if (warp == 1) {
         // ---------------- per-token scales, T and the activation codes: L2 -> shared memory ----------------
-        griddep_wait();                           // all of them come from the preceding kernel
+        if (dep_wait) griddep_wait();             // all of them come from the preceding kernel
+        if (p.dep_mode == kDepHead && lane == 0) griddep_launch_dependents();
         for (int i = lane; i < N_TOK; i += 32) {
             const int t = t0 + i;
             scale_s[i] = t < p.M ? p.scales[t] : 0.f;
@@ -248,7 +255,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t idesc_lr = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
             bool ok = true;
-            griddep_wait();                           // everything this thread waits for follows the preceding kernel
+            if (dep_wait) griddep_wait();             // everything this thread waits for follows the preceding kernel
             if (iss == 0 && lowrank_here) {
                 if (!wait_or_abort(u_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x32); ok = false; }
                 if (ok && !wait_or_abort(t_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x33); ok = false; }
@@ -373,7 +380,7 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                 // An operand stage that is still taken frees up only when MMAs have run, and those need the codes of the
                 // preceding kernel: the bounded wait starts counting once that kernel has finished.
                 if (!__all_sync(0xFFFFFFFFu, mbar_test_wait(&a_empty[as], aph ^ 1u))) {
-                    griddep_wait();
+                    if (dep_wait) griddep_wait();
                     if (!warp_wait(&a_empty[as], aph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x41); ok = false; }
                 }
                 if (ok) {
@@ -393,8 +400,9 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (lane == 0) mbar_arrive(&w_empty[ws]);
             if (++ws == WS) { ws = 0; wph ^= 1u; }
         }
-        // the stores of the epilogue come after the preceding kernel; the per-token scales and code sums it wrote were
-        // staged in shared memory by warp 1 while the K loop ran
+        // the stores of the epilogue come after the preceding kernel (for a sibling: this is the wait every kernel of the
+        // chain executes before it ends); the per-token scales and code sums were staged in shared memory by warp 1
+        // while the K loop ran
         griddep_wait();
         if (!warp_wait(s_full, 0, abort_flag)) { give_up(p.status, abort_flag, 0x51); ok = false; }
         if (ok) {
@@ -613,8 +621,10 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
     const int units = (K + kUnitK - 1) / kUnitK;
     const int sms = sm_count();
     if (sms <= 0) return BWLA_ERR_CUDA;
-    int split = choose_splits(row_tiles * tok_tiles, units, n_tok <= 64, sms);
-    const int wide_split = n_tok <= 32 ? choose_wide_splits(row_tiles * tok_tiles, units, split, sms) : 0;
+    // siblings that run beside one another plan for their share of the SMs
+    const int plan_sms = a.sm_budget > 0 ? std::max(std::min(sms, a.sm_budget), row_tiles * tok_tiles) : sms;
+    int split = choose_splits(row_tiles * tok_tiles, units, n_tok <= 64, plan_sms);
+    const int wide_split = n_tok <= 32 ? choose_wide_splits(row_tiles * tok_tiles, units, split, plan_sms) : 0;
     if (wide_split) split = wide_split;
 
     CUtensorMap wm, bm, tm;
@@ -648,7 +658,7 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
     UmmaParams p{};
     p.M = M; p.N = N; p.K = K; p.total_units = units; p.splits = split; p.r = a.r;
     p.scales = a.scales; p.qsum = a.qsum; p.alpha = a.alpha; p.mu = a.mu; p.zp = a.zp; p.rowsum = a.rowsum; p.U = (const __nv_bfloat16*)a.U;
-    p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug; p.status = a.status;
+    p.out = (__nv_bfloat16*)a.out; p.ldo = a.ldo; p.acc_debug = a.acc_debug; p.status = a.status; p.dep_mode = a.dep_mode;
 
     dim3 grid((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     switch (n_tok) {
