@@ -67,6 +67,26 @@ int bwla_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw,
                     uint32_t* packed, void* stream);
 
 /*
+ * Final binarisation in the rotated coordinates, offline, once per layer.   (Alg. 2, last step; Eq. 1-3)
+ * Every row of W_res = W - M (the weights less the PSP low-rank part) goes through the same map as an activation row,
+ * X_n = flatten(P1^T reshape(w_n, n1 x n2) P2); then mu[n] = mean_k X[n][k], alpha[n] = mean_k |X[n][k] - mu[n]|,
+ * packed bit (n, k) = (X[n][k] - mu[n] > 0).  The outputs are what bwla_w1ax_linear / bwla_layer_create take.
+ *   w_res  device, [N][ldw] fp32 (dtype 0) or bf16 (dtype 1), ldw >= K
+ *   P1, P2 device, fp32, 16-byte aligned; n1*n2 == K, K a positive multiple of 32
+ *   packed device, uint32 [N][K/32]; alpha, mu device, fp32 [N]; all written in full
+ *   workspace: 256-byte aligned device scratch of bwla_binarize_workspace_bytes(K) bytes (0 for an invalid K); the call
+ *     clears its status words itself.
+ * The rotation runs on the tensor-core kernel (fp32 rows as three bf16 terms, three passes); its error is below 1e-6 of
+ * a row's largest rotated magnitude, so a sign can differ from the exact one only where |X - mu| is below that.
+ * Factor sizes that kernel does not take (n2 % 8 != 0, n2 > 256, n1 > 192) return BWLA_ERR_UNSUPPORTED.
+ * N == 0 is a no-op.  Asynchronous on `stream`; bwla_check_status(workspace, stream) reports a device-side timeout.
+ */
+size_t bwla_binarize_workspace_bytes(int64_t K);
+int bwla_binarize_rows(const void* w_res, int dtype, int64_t N, int64_t K, int64_t ldw, const float* P1, int n1,
+                       const float* P2, int n2, uint32_t* packed, float* alpha, float* mu, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
+/*
  * Online OKT + per-token symmetric quantisation.   (Sec. 3.1 Kronecker evaluation; Sec. 4.1 per-token)
  *   x_bf16 device, bf16 [M][ldx], ldx >= K
  *   P1     device, fp32 [n1][n1];  P2 device, fp32 [n2][n2];  n1*n2 == K

@@ -37,7 +37,8 @@ EXPORTS = [
     "bwla_status_string", "bwla_profile_enable", "bwla_profile_collect", "bwla_w1ax_linear_static",
     "bwla_workspace_section", "bwla_force_rotation", "bwla_layer_prepared_bytes", "bwla_layer_create",
     "bwla_layer_destroy", "bwla_layer_rotate_quant", "bwla_group_workspace_bytes", "bwla_w1ax_linear_group",
-    "bwla_layer_set_activation_quant", "bwla_layer_rotate_quant_asym",
+    "bwla_layer_set_activation_quant", "bwla_layer_rotate_quant_asym", "bwla_binarize_workspace_bytes",
+    "bwla_binarize_rows",
 ]
 
 
@@ -55,6 +56,9 @@ def _load() -> C.CDLL:
     i64, vp, ci, sz = C.c_int64, C.c_void_p, C.c_int, C.c_size_t
     lib.bwla_pack_signs.argtypes = [vp, ci, i64, i64, i64, vp, vp]
     lib.bwla_rotate_quant_act.argtypes = [vp, i64, i64, i64, vp, ci, vp, ci, ci, vp, vp, vp]
+    lib.bwla_binarize_workspace_bytes.argtypes = [i64]
+    lib.bwla_binarize_workspace_bytes.restype = sz
+    lib.bwla_binarize_rows.argtypes = [vp, ci, i64, i64, i64, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
     lib.bwla_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
     lib.bwla_workspace_bytes.restype = sz
     lib.bwla_w1ax_linear.argtypes = [vp, i64, i64, i64, vp, ci, vp, ci, ci, vp, vp, vp, vp, vp, ci, vp, i64, i64,
@@ -169,6 +173,31 @@ def bwla_pack_signs(w: torch.Tensor, packed: Optional[torch.Tensor] = None) -> t
                               _ptr(packed), _stream())
     _check(st, "bwla_pack_signs")
     return packed
+
+
+def bwla_binarize_workspace_bytes(K: int) -> int:
+    return int(_lib.bwla_binarize_workspace_bytes(K))
+
+
+def bwla_binarize_rows(w_res: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, workspace: Optional[torch.Tensor] = None):
+    """w_res: fp32 or bf16 [N][K] (row stride >= K) -> (packed int32 [N][K/32], alpha fp32 [N], mu fp32 [N]) of the rows
+    rotated by P1 (x) P2 (Alg. 2, last step)."""
+    if w_res.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("w_res must be fp32 or bf16")
+    _need(w_res, w_res.dtype, "w_res", 2)
+    _need(P1, torch.float32, "P1", 2)
+    _need(P2, torch.float32, "P2", 2)
+    N, K = w_res.shape
+    packed = torch.empty((N, K // 32), dtype=torch.int32, device=w_res.device)
+    alpha = torch.empty(N, dtype=torch.float32, device=w_res.device)
+    mu = torch.empty(N, dtype=torch.float32, device=w_res.device)
+    if workspace is None:
+        workspace = torch.zeros(bwla_binarize_workspace_bytes(K), dtype=torch.uint8, device=w_res.device)
+    st = _lib.bwla_binarize_rows(_ptr(w_res), 0 if w_res.dtype == torch.float32 else 1, N, K, w_res.stride(0) if N > 0 else K,
+                                 _ptr(P1), P1.shape[0], _ptr(P2), P2.shape[0], _ptr(packed), _ptr(alpha), _ptr(mu),
+                                 _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "bwla_binarize_rows")
+    return packed, alpha, mu
 
 
 def bwla_rotate_quant_act(x: torch.Tensor, P1: torch.Tensor, P2: torch.Tensor, bits: int,

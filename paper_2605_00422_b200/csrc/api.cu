@@ -111,6 +111,26 @@ int bwla_pack_signs(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw,
     return launch_pack_signs(w, dtype, N, K, ldw, packed, (cudaStream_t)stream);
 }
 
+size_t bwla_binarize_workspace_bytes(int64_t K) {
+    if (K <= 0 || K % 32 != 0 || K > 25600) return 0;
+    return binarize_workspace_bytes(K);
+}
+
+int bwla_binarize_rows(const void* w_res, int dtype, int64_t N, int64_t K, int64_t ldw, const float* P1, int n1,
+                       const float* P2, int n2, uint32_t* packed, float* alpha, float* mu, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    g_launch_count = 0;
+    if (N < 0 || !valid_rotation_dims(K, n1, n2) || ldw < K || (dtype != BWLA_DTYPE_F32 && dtype != BWLA_DTYPE_BF16))
+        return BWLA_ERR_INVALID_ARG;
+    if (N == 0) return BWLA_OK;
+    if (!w_res || !P1 || !P2 || !packed || !alpha || !mu) return BWLA_ERR_INVALID_ARG;
+    if (((uintptr_t)P1 & 15) || ((uintptr_t)P2 & 15)) return BWLA_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < bwla_binarize_workspace_bytes(K)) return BWLA_ERR_WORKSPACE;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+    return launch_binarize(w_res, dtype, N, K, ldw, P1, n1, P2, n2, packed, alpha, mu, workspace, (cudaStream_t)stream);
+}
+
 int bwla_rotate_quant_act(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* P1, int n1,
                           const float* P2, int n2, int bits, int8_t* codes, float* scales, void* stream) {
     g_launch_count = 0;

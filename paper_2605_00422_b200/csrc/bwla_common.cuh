@@ -213,6 +213,11 @@ struct GemmArgs {
 };
 enum { kDepChain = 0, kDepHead = 1, kDepSibling = 2 };
 
+// Final binarisation of weight rows in the rotated coordinates (binarize.cu).
+size_t binarize_workspace_bytes(int64_t K);
+int launch_binarize(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw, const float* P1, int n1, const float* P2, int n2,
+                    uint32_t* packed, float* alpha, float* mu, void* workspace, cudaStream_t stream);
+
 int launch_gemm_simple(const GemmArgs& a, cudaStream_t stream);
 
 // One to four tokens: activation bit-planes against the packed sign words (and + popc), weights never expanded.

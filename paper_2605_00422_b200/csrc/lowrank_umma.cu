@@ -214,9 +214,19 @@ __global__ void __launch_bounds__(lru::kTok) lowrank_reduce_kernel(const LrUmmaP
     const int64_t t = (int64_t)tile * kTok + threadIdx.x;
     float s[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     const float* src = p.part[pi] + (size_t)tile * p.ks * (kCols * kTok) + (size_t)(8 * cg) * kTok + threadIdx.x;
-    for (int k = 0; k < p.ks; ++k) {
+    // all loads of four parts are in flight before the first addition (the loop is a chain of L2 latencies otherwise);
+    // the additions keep the order of the parts
+    for (int k0 = 0; k0 < p.ks; k0 += 4) {
+        float v[4][8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) s[c] += __ldcg(src + (size_t)k * (kCols * kTok) + c * kTok);
+        for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                v[kk][c] = k0 + kk < p.ks ? __ldcg(src + (size_t)(k0 + kk) * (kCols * kTok) + c * kTok) : 0.f;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) s[c] += v[kk][c];
     }
     if (t < p.M) store_terms(p.Thl[pi], p.M, t, 8 * cg, s);
 }

@@ -528,8 +528,10 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                 }
                 if (lane_valid) { amax = fmaxf(m0, m1); vmin = fminf(l0, l1); }
             }
-            amax = warp_max(amax);
-            if (asym) vmin = -warp_max(-vmin);
+            // both are non-negative here (NaNs aside), so their bit patterns order like the values: one warp-wide integer
+            // reduction each instead of five shuffle steps
+            amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(fmaxf(amax, 0.f))));
+            if (asym) vmin = -__uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(fmaxf(-vmin, 0.f))));
             if (lane == 0) { red_max[warp - 2] = amax; red_min[warp - 2] = vmin; }
             // one decision for all ALU warps: a warp that gave up must not leave the others alone at a barrier
             if (alu_barrier_or(failed || *abort_flag != 0)) break;
@@ -544,6 +546,24 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                 st_shared_cluster_u32(map_shared_rank(smem_u32(slots_min + par * 8 + rank), (uint32_t)e), __float_as_uint(vmin));
                 mbar_arrive_remote(map_shared_rank(smem_u32(&xbar[par]), (uint32_t)e));
             }
+            // symmetric: codes in [-qmax, qmax] around zero.  Asymmetric (Sec. 4.1): u = rne(y * inv) + zero in [0, 2^b - 1]
+            // with an integer zero point; what is stored is u - 2^(b-1) (+ the caller's bias), so that it fits int8.
+            float inv = 0.f, scale = 1.f, zero_f = 0.f, lo_c = -(float)qmax, hi_c = (float)qmax, half_f = 0.f;
+            auto set_scales = [&]() {
+                if (!asym) {
+                    if (amax != 0.f) { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
+                } else {
+                    const float levels = (float)((1 << p.bits) - 1);
+                    const float range = __fsub_rn(amax, vmin);
+                    if (range != 0.f) { inv = __fdiv_rn(levels, range); scale = __fdiv_rn(range, levels); }
+                    const float tz = __fmul_rn(-vmin, inv);
+                    zero_f = fminf(fmaxf(__fadd_rn(__fadd_rn(tz, 12582912.f), -12582912.f), 0.f), levels);
+                    lo_c = 0.f; hi_c = levels; half_f = (float)(1 << (p.bits - 1));
+                }
+            };
+            // (a CTA that owns its token alone has the absmax now: the divisions go in front of stage B, which still
+            // waits for the next token's stage A at this point)
+            if (D == 1) set_scales();
             if (it + 1 < ntok) stage_b(ph ^ 1u);
             if (D > 1) {
                 if (!failed && !warp_wait_cluster(&xbar[par], (uint32_t)((it >> 1) & 1), abort_flag)) { give_up(p.status, abort_flag, 0x72); failed = true; }
@@ -551,21 +571,7 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
                     amax = 0.f; vmin = 0.f;
                     for (int c = 0; c < D; ++c) { amax = fmaxf(amax, slots[par * 8 + c]); vmin = fminf(vmin, slots_min[par * 8 + c]); }
                 }
-            }
-            // symmetric: codes in [-qmax, qmax] around zero.  Asymmetric (Sec. 4.1): u = rne(y * inv) + zero in [0, 2^b - 1]
-            // with an integer zero point; what is stored is u - 2^(b-1) (+ the caller's bias), so that it fits int8.
-            float inv, scale, zero_f = 0.f, lo_c = -(float)qmax, hi_c = (float)qmax, half_f = 0.f;
-            if (!asym) {
-                if (amax == 0.f) { inv = 0.f; scale = 1.f; }
-                else { inv = __fdiv_rn((float)qmax, amax); scale = __fdiv_rn(amax, (float)qmax); }
-            } else {
-                const float levels = (float)((1 << p.bits) - 1);
-                const float range = __fsub_rn(amax, vmin);
-                if (range == 0.f) { inv = 0.f; scale = 1.f; }
-                else { inv = __fdiv_rn(levels, range); scale = __fdiv_rn(range, levels); }
-                const float tz = __fmul_rn(-vmin, inv);
-                zero_f = fminf(fmaxf(__fadd_rn(__fadd_rn(tz, 12582912.f), -12582912.f), 0.f), levels);
-                lo_c = 0.f; hi_c = levels; half_f = (float)(1 << (p.bits - 1));
+                set_scales();
             }
             const float store_shift = (float)pr.code_bias - half_f;
             // nothing is stored to global memory before the preceding kernel of the stream has completed
@@ -578,8 +584,6 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             //      beyond the range only come from rounding of the reciprocal and of the zero point).  The stored byte
             //      is the low byte of the pattern, and the patterns themselves are summed for the code sum: every one
             //      is 0x4B400000 + the stored code.
-            //      A CTA that owns the whole token collects the codes in shared memory in natural order (a warp writes 32
-            //      consecutive bytes per column) and reorders them on the way out.
             const int shift_i = (int)(zero_f + store_shift);                 // small integer, exact
             const uint32_t odd = (uint32_t)(shift_i & 1);
             const float bias_even = 12582912.f + (float)(shift_i - (int)odd);
@@ -628,7 +632,7 @@ okt_umma_kernel(const __grid_constant__ CUtensorMap x_map, const OktKernelParams
             // sum of (stored code - the caller's bias) over this lane's elements, in wrap-around arithmetic; the CTA's sum
             // is collected in red_sum[par] and leaves after the next token's barrier (or the one behind the loop)
             int local_sum = lane_valid ? (int)(usum - (uint32_t)counted * (0x4B400000u + (uint32_t)pr.code_bias)) : 0;
-            local_sum = warp_sum(local_sum);
+            local_sum = __reduce_add_sync(0xFFFFFFFFu, local_sum);
             if (lane == 0 && local_sum != 0 && !failed) atomicAdd(&red_sum[par], local_sum);
             if (e == 0 && !failed && rank == 0) {
                 pr.scales[t] = scale;
