@@ -383,7 +383,9 @@ int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const voi
     cudaStream_t s = (cudaStream_t)stream;
     const bwla_layer* L0 = layers[0];
     char* base = (char*)workspace;
-    uint32_t* status = (uint32_t*)base;                  // the status word of the whole call: the first layer's
+    // The status words of the whole call are the first layer's: only those 256 bytes start at zero.  Layer i keeps its
+    // arrival counters for split sums of T in words 4 + 8 i .. 11 + 8 i of them.
+    uint32_t* status = (uint32_t*)base;
     Workspace ws[kOktMaxProblems];
     char* wbase[kOktMaxProblems];
     int path[kOktMaxProblems];
@@ -406,7 +408,7 @@ int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const voi
                                L->asym ? (int32_t*)(wbase[i] + ws[i].zp) : nullptr, 0,
                                (float*)(wbase[i] + ws[i].scales), (int32_t*)(wbase[i] + ws[i].qsum), nullptr};
             lr[i] = OktLowrank{L->V, L->r, wbase[i] + ws[i].T, L->r > 0 ? (float*)(wbase[i] + ws[i].lr_part) : nullptr,
-                               (uint32_t*)(wbase[i] + ws[i].status) + kLrCounterWord};
+                               status + 8 * i + kLrCounterWord};
         }
         st = launch_okt(L0->geom, x_bf16, M, ldx, L0->bits, L0->asym, count, pr, lr, status, s);
         if (st != BWLA_OK) return st;
@@ -416,7 +418,7 @@ int bwla_w1ax_linear_group(const bwla_layer* const* layers, int count, const voi
             st = launch_prologue(x_bf16, M, L->K, ldx, L->P1, L->n1, L->P2, L->n2, L->bits, (int8_t*)(wbase[i] + ws[i].codes),
                                  path[i] == BWLA_PATH_I8 ? 1 : 0, (float*)(wbase[i] + ws[i].scales),
                                  (int32_t*)(wbase[i] + ws[i].qsum), L->V, L->r, wbase[i] + ws[i].T,
-                                 L->r > 0 ? (float*)(wbase[i] + ws[i].lr_part) : nullptr, (uint32_t*)(wbase[i] + ws[i].status), s);
+                                 L->r > 0 ? (float*)(wbase[i] + ws[i].lr_part) : nullptr, status + 8 * i, s);
             if (st != BWLA_OK) return st;
         }
     }

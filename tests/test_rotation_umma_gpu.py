@@ -192,3 +192,22 @@ def test_asymmetric_layers_match_the_oracle(bwla, idxs, M, bits, path):
         slack = flips[:, None] * per_row[None, :] * ref["scales"].astype(np.float64)[:, None]
         rep = H.check_output(H.bf16_to_host(out), ref["y"], step_slack=slack)
         assert rep["rel_l2"] <= 2e-3
+
+
+def test_group_workspace_needs_only_its_first_256_bytes_zeroed(bwla):
+    """The arrival counters of every layer's split sums of T live in the first status block: a workspace that is garbage
+    behind its first 256 bytes gives the same outputs as a zero-filled one (K = 25600 and 8192 split K at 16 tokens)."""
+    for idxs in ((6,), (3,), (0, 1, 2)):
+        shapes = [gen.CONFIG_SHAPES[2][i] for i in idxs]
+        lays = [gen.make_layer(2, sh, 6, direct_words=True) for sh in shapes]
+        dls = [H.DeviceLayer(l, bwla) for l in lays]
+        layers = [bwla.Layer(d.P1, d.P2, 6, d.packed, d.alpha, d.U, d.V) for d in dls]
+        x = H.bf16_to_dev(gen.make_activations(2, shapes[0], 16))
+        clean = bwla.new_group_workspace(layers, 16)
+        outs_a = bwla.bwla_w1ax_linear_group(layers, x, workspace=clean)
+        dirty = torch.randint(0, 256, (clean.numel(),), dtype=torch.uint8, device="cuda")
+        dirty[:256] = 0
+        outs_b = bwla.bwla_w1ax_linear_group(layers, x, workspace=dirty)
+        assert bwla.bwla_check_status(dirty) == 0
+        for a, b in zip(outs_a, outs_b):
+            assert torch.equal(a, b)
