@@ -5,7 +5,7 @@
 //   D2[n][t] = sum_j U[n][j] * T[t][j]                                        (PSP low-rank term, Sec. 3.2)
 //   out[t][n] = bf16(alpha[n] * s_t * acc + D2 [+ mu[n] * s_t * sum_k q[t][k]])   (Eq. 4 on the accumulator)
 //
-// One CTA owns 128 output rows x up to 128 tokens x a slice of K; the CTAs that share a tile and split K form a
+// One CTA owns 128 output rows x up to 64 tokens x a slice of K; the CTAs that share a tile and split K form a
 // thread-block cluster and add their partial sums through distributed shared memory, so nothing but the bf16
 // result is written to global memory.  Inside a CTA:
 //   * warp 0 streams packed sign words by TMA (128 rows x 128 bytes = 1024 weights per row, 128B-swizzled); these
@@ -615,7 +615,8 @@ static int choose_wide_splits(int tiles, int units, int narrow_splits, int sms) 
 int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStream_t stream) {
     const int M = (int)a.M, N = (int)a.N, K = (int)a.K;
     if (umma_persistent_supports(a.M, a.K, a.N, a.r)) return launch_gemm_umma_persistent(a, codes_interleaved, stream);
-    const int n_tok = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128;
+    if (M > 64) return BWLA_ERR_UNSUPPORTED;                  // (every such problem this path takes went to the persistent kernel)
+    const int n_tok = M <= 16 ? 16 : M <= 32 ? 32 : 64;
     const int row_tiles = (N + kRowsPerCta - 1) / kRowsPerCta;
     const int tok_tiles = (M + n_tok - 1) / n_tok;
     const int units = (K + kUnitK - 1) / kUnitK;
@@ -669,8 +670,8 @@ int launch_gemm_umma(const GemmArgs& a, const int8_t* codes_interleaved, cudaStr
         // a grid larger than the SM count would run in two waves with one CTA per SM: two smaller CTAs per SM instead
         case 64: return grid.x * grid.y * grid.z > (unsigned)sms ? launch_umma_t<64, 2, 2, 256, 1, 2>(wm, bm, tm, p, grid, stream)
                                                        : launch_umma_t<64, 4, 3, 512, 2, 4>(wm, bm, tm, p, grid, stream);
-        default: return launch_umma_t<128, 2, 6, 512, 1, 4>(wm, bm, tm, p, grid, stream);
     }
+    return BWLA_ERR_UNSUPPORTED;
 }
 
 }  // namespace bwla
