@@ -211,3 +211,32 @@ def test_group_workspace_needs_only_its_first_256_bytes_zeroed(bwla):
         assert bwla.bwla_check_status(dirty) == 0
         for a, b in zip(outs_a, outs_b):
             assert torch.equal(a, b)
+
+
+def test_outputs_of_one_group_feed_the_next_group_without_synchronisation(bwla):
+    """q/k/v run beside one another (the siblings of a group do not wait for each other); the next group reads q's
+    output as its x right behind them on the same stream.  The result must not depend on host synchronisation."""
+    M = 16
+    sq, sk, sv, so = (gen.CONFIG_SHAPES[2][i] for i in (0, 1, 2, 3))
+    assert sq.N == so.K
+    lays = [gen.make_layer(2, sh, 6, direct_words=True) for sh in (sq, sk, sv, so)]
+    dls = [H.DeviceLayer(l, bwla) for l in lays]
+    L = [bwla.Layer(d.P1, d.P2, 6, d.packed, d.alpha, d.U, d.V) for d in dls]
+    x = H.bf16_to_dev(gen.make_activations(2, sq, M))
+    ws1 = bwla.new_group_workspace(L[:3], M)
+    ws2 = bwla.new_group_workspace(L[3:], M)
+
+    def run(sync):
+        outs = bwla.bwla_w1ax_linear_group(L[:3], x, workspace=ws1)
+        if sync:
+            torch.cuda.synchronize()
+        y = bwla.bwla_w1ax_linear_group(L[3:], outs[0], workspace=ws2)[0]
+        torch.cuda.synchronize()
+        return [o.clone() for o in outs] + [y.clone()]
+
+    want = run(True)
+    for _ in range(5):
+        got = run(False)
+        for a, b in zip(want, got):
+            assert torch.equal(a, b)
+    assert bwla.bwla_check_status(ws1) == 0 and bwla.bwla_check_status(ws2) == 0
