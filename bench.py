@@ -333,8 +333,8 @@ def run_per_shape(args):
     NL = 6                                            # layers with distinct sign words per shape (cold weights)
     rows = []
     print("| config | shape | bits | M | path | whole call us | prologue us | contraction us | GB/s (call bytes) | TOPS (2MKN) | "
-          "% of measured HBM | % of 2x burst bf16 | other path us |")
-    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
+          "% of measured HBM | % of 8 TB/s | % of 2x burst bf16 | % of 4.5 POP/s | other path us |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for cfg in (1, 2, 3):
         if args.cfg and cfg != args.cfg:
             continue
@@ -397,7 +397,8 @@ def run_per_shape(args):
                     tops = call_ops(sh, M) / (whole * 1e-6) / 1e12
                     name = {1: "simple", 2: "bit-plane", 3: "tcgen05 i8"}[chosen]
                     print(f"| {cfg} | {sh.name} {sh.K}->{sh.N} | {bits} | {M} | {name} | {whole:.1f} | {pro:.1f} | {con:.1f} | {gbs:.0f} | "
-                          f"{tops:.1f} | {100 * gbs / peaks['hbm_gbs']:.1f} | {100 * tops / (2 * peaks['bf16_tflops']):.1f} | {other} |", flush=True)
+                          f"{tops:.1f} | {100 * gbs / peaks['hbm_gbs']:.1f} | {100 * gbs / 8000.0:.1f} | "
+                          f"{100 * tops / (2 * peaks['bf16_tflops']):.1f} | {100 * tops / 4500.0:.1f} | {other} |", flush=True)
                 del layers
                 torch.cuda.empty_cache()
 

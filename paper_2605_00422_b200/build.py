@@ -49,16 +49,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 def build_microbench() -> str:
-    """The instruction-rate probes (a stand-alone program; not part of the library)."""
-    src = os.path.join(_HERE, "microbench", "issue_rates.cu")
-    out = os.path.join(_HERE, "microbench", "issue_rates")
+    """The instruction-rate probes (stand-alone programs; not part of the library)."""
     nvcc = os.environ.get("NVCC", "nvcc")
-    res = subprocess.run([nvcc, "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a", "-o", out, src],
-                         capture_output=True, text=True)
-    if res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-        raise RuntimeError("nvcc failed building the microbenchmark")
-    return out
+    outs = []
+    for name in ("issue_rates", "umma_rates"):
+        src = os.path.join(_HERE, "microbench", name + ".cu")
+        out = os.path.join(_HERE, "microbench", name)
+        res = subprocess.run([nvcc, "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a", "-I", INCLUDE,
+                              "-I", CSRC, "-o", out, src], capture_output=True, text=True)
+        if res.returncode != 0:
+            sys.stderr.write(res.stdout + res.stderr)
+            raise RuntimeError("nvcc failed building the microbenchmark " + name)
+        outs.append(out)
+    return " ".join(outs)
 
 
 if __name__ == "__main__":
