@@ -27,7 +27,8 @@ __device__ __forceinline__ void mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 
-// KIND 0: i8, A in tensor memory; 1: i8, A in shared memory; 2: f16 (bf16 operands), shared; 3: f16, A in tensor memory
+// KIND 0: i8, A in tensor memory; 1: i8, A in shared memory; 2: f16 (bf16 operands), shared; 3: f16, A in tensor memory;
+// 4: i8, A in shared memory, M = 64
 template <int KIND>
 __global__ void __launch_bounds__(128, 1) probe(int n_cols, int count, long long* issue_cycles, long long* total_cycles,
                                                 uint32_t* status) {
@@ -52,15 +53,16 @@ __global__ void __launch_bounds__(128, 1) probe(int n_cols, int count, long long
     tc_fence_after();
     const uint32_t tmem_base = *slot;
     if (threadIdx.x == 0) {
-        const uint32_t fmt = KIND < 2 ? (2u << 4) : (1u << 4);           // D = s32 / f32
-        const uint32_t idesc = fmt | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((128u >> 4) << 24);
+        const uint32_t fmt = (KIND < 2 || KIND == 4) ? (2u << 4) : (1u << 4);           // D = s32 / f32
+        const uint32_t m_rows = KIND == 4 ? 64u : 128u;
+        const uint32_t idesc = fmt | (1u << 7) | (1u << 10) | ((uint32_t)(n_cols >> 3) << 17) | ((m_rows >> 4) << 24);
         const uint32_t a_addr = smem_u32(smem), b_addr = a_addr + kABytes;
         const long long t0 = clock64();
         for (int i = 0; i < count; ++i) {
             const uint32_t j = (uint32_t)i & 3u;
             const uint64_t db = smem_desc_sw128(b_addr, 32 * j);
             if (KIND == 0) mma_i8_ts(tmem_base, tmem_base + 256 + 8 * j, db, idesc, i ? 1u : 0u);
-            else if (KIND == 1) mma_i8_ss(tmem_base, smem_desc_sw128(a_addr, 32 * j), db, idesc, i ? 1u : 0u);
+            else if (KIND == 1 || KIND == 4) mma_i8_ss(tmem_base, smem_desc_sw128(a_addr, 32 * j), db, idesc, i ? 1u : 0u);
             else if (KIND == 2) mma_f16_ss(tmem_base, smem_desc_sw128(a_addr, 32 * j), db, idesc, i ? 1u : 0u);
             else mma_f16_ts(tmem_base, tmem_base + 256 + 8 * j, db, idesc, i ? 1u : 0u);
         }
@@ -80,7 +82,7 @@ __global__ void __launch_bounds__(128, 1) probe(int n_cols, int count, long long
 }
 
 template <int KIND>
-static int run(const char* name, int k_per_mma, const int* ns, int n_ns, int sms, double ghz, long long* d_issue, long long* d_total,
+static int run(const char* name, int m_rows, int k_per_mma, const int* ns, int n_ns, int sms, double ghz, long long* d_issue, long long* d_total,
                uint32_t* d_status) {
     cudaFuncSetAttribute(probe<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     const int count = 4096;
@@ -99,7 +101,7 @@ static int run(const char* name, int k_per_mma, const int* ns, int n_ns, int sms
         double issue = 0, total = 0;
         for (int i = 0; i < sms; ++i) { issue += (double)h[i]; total += (double)h[sms + i]; }
         issue /= (double)sms * count; total /= (double)sms * count;
-        const double ops = 2.0 * 128 * n * k_per_mma;
+        const double ops = 2.0 * m_rows * n * k_per_mma;
         printf("| %s | %d | %.1f | %.1f | %.0f |\n", name, n, total, issue, ops * sms * ghz / total / 1e3);
     }
     delete[] h;
@@ -118,14 +120,16 @@ int main() {
     cudaMalloc(&d_total, sizeof(long long) * sms);
     cudaMalloc(&d_status, 256);
     cudaMemset(d_status, 0, 256);
-    printf("%s, %d SMs, %.3f GHz (attribute clock), 4096 MMAs (M = 128) per SM, all SMs at once\n", prop.name, sms, ghz);
+    printf("%s, %d SMs, %.3f GHz (attribute clock), 4096 MMAs (M = 128 unless stated) per SM, all SMs at once\n", prop.name, sms, ghz);
     printf("| instruction | N | cycles per MMA (complete) | cycles per MMA (issue loop) | device Tera-op/s at that rate |\n|---|---|---|---|---|\n");
     const int n_i8[] = {16, 32, 64, 128, 256};
     const int n_f16[] = {16, 64, 80, 128, 160, 256};
     int rc = 0;
-    rc |= run<0>("kind::i8, K = 32, A in tensor memory", 32, n_i8, 5, sms, ghz, d_issue, d_total, d_status);
-    rc |= run<1>("kind::i8, K = 32, A in shared memory", 32, n_i8, 5, sms, ghz, d_issue, d_total, d_status);
-    rc |= run<2>("kind::f16 (bf16), K = 16, A in shared memory", 16, n_f16, 6, sms, ghz, d_issue, d_total, d_status);
-    rc |= run<3>("kind::f16 (bf16), K = 16, A in tensor memory", 16, n_f16, 6, sms, ghz, d_issue, d_total, d_status);
+    rc |= run<0>("kind::i8, K = 32, A in tensor memory", 128, 32, n_i8, 5, sms, ghz, d_issue, d_total, d_status);
+    rc |= run<1>("kind::i8, K = 32, A in shared memory", 128, 32, n_i8, 5, sms, ghz, d_issue, d_total, d_status);
+    rc |= run<2>("kind::f16 (bf16), K = 16, A in shared memory", 128, 16, n_f16, 6, sms, ghz, d_issue, d_total, d_status);
+    rc |= run<3>("kind::f16 (bf16), K = 16, A in tensor memory", 128, 16, n_f16, 6, sms, ghz, d_issue, d_total, d_status);
+    const int n_m64[] = {64, 128, 256};
+    rc |= run<4>("kind::i8, K = 32, A in shared memory, M = 64", 64, 32, n_m64, 3, sms, ghz, d_issue, d_total, d_status);
     return rc;
 }
