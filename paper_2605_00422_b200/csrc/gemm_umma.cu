@@ -206,33 +206,19 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);   // let copies in flight land
         }
     } else if (warp == 1) {
-        // ---------------- per-token scales, T and the activation codes: L2 -> shared memory ----------------
-        if (dep_wait) griddep_wait();             // all of them come from the preceding kernel
-        if (p.dep_mode == kDepHead && lane == 0) griddep_launch_dependents();
-        for (int i = lane; i < N_TOK; i += 32) {
-            const int t = t0 + i;
-            scale_s[i] = t < p.M ? p.scales[t] : 0.f;
-            int32_t qs = 0;
-            if (t < p.M) {
-                const int4* parts = reinterpret_cast<const int4*>(p.qsum + (size_t)t * kQsumParts);
-                const int4 a = parts[0], b = parts[1];
-                qs = a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w;
-            }
-            qsum_s[i] = qs;
-            zp_s[i] = (p.zp && t < p.M) ? p.zp[t] : 0;
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(s_full);
-        if (elect_one()) {
+        // ---------------- T and the activation codes: L2 -> shared memory ----------------
+        // The first copies leave right behind the dependency: everything that can be done before it is (descriptor
+        // prefetch), everything else that follows it (the per-token scalars: warp 5; the look at the status word) comes
+        // after them or elsewhere.  The K loop cannot start before the first codes have landed.
+        if (lane == 0) {
             tma_prefetch_desc(&b_map);
             if (lowrank_here) tma_prefetch_desc(&t_map);
-            if (p.status && *reinterpret_cast<volatile uint32_t*>(p.status) != 0) *abort_flag = 1;   // the call already failed
-            if (lowrank_here && !*abort_flag) {
-                mbar_expect_tx(t_full, 3 * L::sub_bytes);
-                for (int h = 0; h < 3; ++h) tma_load_3d(tbuf + h * L::sub_bytes, &t_map, 0, t0, h, t_full);
-            }
+        }
+        if (dep_wait) griddep_wait();             // all of them come from the preceding kernel
+        if (p.dep_mode == kDepHead && lane == 0) griddep_launch_dependents();
+        if (elect_one()) {
             int bs = 0; uint32_t bph = 0;
-            bool ok = true;
+            bool ok = true, first = true;
             for (int u = unit_begin; u < unit_end && ok && !*abort_flag; ++u) {
                 const int ns = sub_count(u);
                 for (int s0 = 0; s0 < ns; s0 += SUBS) {
@@ -242,6 +228,14 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
                     for (int s = 0; s < cnt; ++s)
                         tma_load_2d(bbuf + bs * L::b_bytes + s * L::sub_bytes, &b_map, (u * 8 + s0 + s) * kBlockK, t0, &b_full[bs]);
                     if (++bs == BS) { bs = 0; bph ^= 1; }
+                    if (first) {
+                        first = false;
+                        if (lowrank_here) {
+                            mbar_expect_tx(t_full, 3 * L::sub_bytes);
+                            for (int h = 0; h < 3; ++h) tma_load_3d(tbuf + h * L::sub_bytes, &t_map, 0, t0, h, t_full);
+                        }
+                        if (p.status && *reinterpret_cast<volatile uint32_t*>(p.status) != 0) *abort_flag = 1;   // the call already failed
+                    }
                 }
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);
@@ -249,7 +243,25 @@ umma_w1a_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     } else if (warp < 6) {
         // ---------------- MMA issue: thread `iss` takes k-blocks kb = iss, iss + NISS, ... ----------------
         const int iss = warp - 2;
-        if (iss < NISS && elect_one()) {
+        static_assert(NISS <= 3, "warp 5 stages the per-token scalars");
+        if (warp == 5) {
+            // ---------------- per-token scales, code sums and zero points into shared memory ----------------
+            if (dep_wait) griddep_wait();             // they come from the preceding kernel (a sibling's are complete)
+            for (int i = lane; i < N_TOK; i += 32) {
+                const int t = t0 + i;
+                scale_s[i] = t < p.M ? p.scales[t] : 0.f;
+                int32_t qs = 0;
+                if (t < p.M) {
+                    const int4* parts = reinterpret_cast<const int4*>(p.qsum + (size_t)t * kQsumParts);
+                    const int4 a = parts[0], b = parts[1];
+                    qs = a.x + a.y + a.z + a.w + b.x + b.y + b.z + b.w;
+                }
+                qsum_s[i] = qs;
+                zp_s[i] = (p.zp && t < p.M) ? p.zp[t] : 0;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_full);
+        } else if (iss < NISS && elect_one()) {
             // instruction descriptors: D = s32, A = s8 (tensor memory, K-major), B = s8 (shared, K-major), M = 128;
             // and D = f32, A = B = bf16 (shared, K-major), M = 128
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TOK >> 3) << 17) | ((128u >> 4) << 24);
