@@ -35,7 +35,7 @@ from paper_2605_00422_b200 import inputs as gen  # noqa: E402
 # kernel source has changed since, the figure is dropped (null).
 NCU_TRAFFIC = {
     "decode": {"dram_bytes": 19881728, "algorithmic_bytes": 20216896,          # gate_proj launch, M = 8
-               "kernel_sha256": "e901d8e8f5e1190cdd51048be2f8220b89abe89ee1cddcc774e99525850802f7"},
+               "kernel_sha256": "c8b8ebb137de23f31e5bfe57756a613fbc1113d2d736c5cef58e013ed50bad3e"},
 }
 
 METRIC = "W1A6 linear: decode HBM GB/s & prefill INT8 TOPS vs B200 roofline, Qwen3-32B"
