@@ -389,6 +389,34 @@ void bwla_oracle_epilogue(const int64_t* acc, const float* scales, const float* 
         }
 }
 
+/*
+ * The weight-only operating point, W1A16 (Table 1, upper half: binarised weights, 16-bit activations): the rotated
+ * activation is not quantised to integers but kept as a 16-bit value, here bf16 (round to nearest even of the fp64
+ * rotation), and meets the signs directly:
+ *   yhat = bf16(Y),  acc[t][n] = sum_k s[n][k] * yhat[t][k],  y[t][n] = alpha[n] * acc[t][n] + L[t][n] (+ mu[n] * sum_k yhat[t][k]).
+ * Y (fp64 [M][K]) comes from bwla_oracle_rotate, L (fp64 [M][N], may be NULL) from bwla_oracle_lowrank.
+ */
+void bwla_oracle_a16(const double* Y, int64_t M, int64_t K, const uint32_t* packed, const float* alpha, const float* mu,
+                     const double* L, int64_t N, uint16_t* yhat, double* acc, double* y) {
+    int64_t words = K / 32;
+    for (int64_t i = 0; i < M * K; ++i) yhat[i] = f64_to_bf16(Y[i]);
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t t = 0; t < M; ++t) {
+            double a = 0.0, sum = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                double v = bf16_to_f64(yhat[t * K + k]);
+                a += ((packed[n * words + (k >> 5)] >> (k & 31)) & 1u) ? v : -v;
+                sum += v;
+            }
+            acc[t * N + n] = a;
+            double out = (double)alpha[n] * a;
+            if (L) out += L[t * N + n];
+            if (mu) out += (double)mu[n] * sum;
+            y[t * N + n] = out;
+        }
+}
+
 /* The whole layer, steps in order.  Optional outputs may be NULL.  Returns 0, or 1 if an accumulator leaves int32. */
 int bwla_oracle_linear(const uint16_t* x, int64_t M, int64_t K, int64_t ldx,
                        const float* P1, int64_t n1, const float* P2, int64_t n2, int bits, int decision,

@@ -20,7 +20,7 @@ _LIB = os.path.join(_HERE, "libbwla_oracle.so")
 __all__ = [
     "build", "num_threads", "kron_factor", "row_stats", "pack_signs", "pack_signs_bf16", "unpack_signs",
     "rotate", "quantize", "gemm", "lowrank", "epilogue", "linear", "bf16_round", "near_tie_window",
-    "quantize_asym", "gemm_asym", "linear_asym", "near_tie_window_asym", "binarize",
+    "quantize_asym", "gemm_asym", "linear_asym", "near_tie_window_asym", "binarize", "linear_a16",
 ]
 
 
@@ -239,6 +239,26 @@ def bf16_round(y: np.ndarray) -> np.ndarray:
     out = np.empty(y.shape, np.uint16)
     _L().bwla_oracle_bf16_round(_p(y), i64(y.size), _p(out))
     return out
+
+
+def linear_a16(x_bits, P1, P2, packed, alpha, U_bits=None, V_bits=None, mu=None) -> Dict[str, np.ndarray]:
+    """The weight-only layer (W1A16): rotated activations kept in bf16.  Returns y (fp64), Y (rotated, fp64), yhat (bf16
+    bits), acc (fp64)."""
+    x_bits = _c(x_bits, np.uint16)
+    packed = _c(packed, np.uint32)
+    alpha = _c(alpha, np.float32)
+    M, K = x_bits.shape
+    N = packed.shape[0]
+    assert packed.shape[1] * 32 == K and alpha.shape == (N,)
+    Y = rotate(x_bits, P1, P2)
+    L = lowrank(x_bits, U_bits, V_bits) if U_bits is not None else None
+    if mu is not None:
+        mu = _c(mu, np.float32)
+    yhat = np.empty((M, K), np.uint16)
+    acc = np.empty((M, N), np.float64)
+    y = np.empty((M, N), np.float64)
+    _L().bwla_oracle_a16(_p(Y), i64(M), i64(K), _p(packed), _p(alpha), _p(mu), _p(L), i64(N), _p(yhat), _p(acc), _p(y))
+    return {"y": y, "Y": Y, "yhat": yhat, "acc": acc}
 
 
 def linear(x_bits, P1, P2, bits, packed, alpha, U_bits=None, V_bits=None, mu=None,

@@ -475,3 +475,50 @@ def test_binarisation_scale_minimises_the_reconstruction_error_of_the_rotated_ro
         errs = [np.sum((x - a * s[n]) ** 2) for a in grid]
         assert abs(grid[int(np.argmin(errs))] - out["alpha"][n]) <= out["alpha"][n] * 1e-3
         assert abs(np.mean(x)) < 1e-12
+
+
+# ----------------------------------------------------------------------------------------------
+# W1A16: the weight-only operating point (Table 1, upper half)
+# ----------------------------------------------------------------------------------------------
+def test_a16_with_identity_factors_is_the_plain_signed_sum_of_the_activations():
+    """P = I: the rotated activation is x itself, which is bf16 already, so nothing is rounded and the layer is
+    alpha * (S x) with S the +-1 matrix, written here with an independent dense product."""
+    n1, n2, N, M = 4, 16, 24, 5
+    K = n1 * n2
+    rng = np.random.default_rng(21)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    packed = oracle.pack_signs(W)
+    S = np.where(W > 0, 1.0, -1.0)
+    alpha = rng.uniform(0.5, 2.0, N).astype(np.float32)
+    mu = rng.uniform(-0.1, 0.1, N).astype(np.float32)
+    xb = _bf16(rng.standard_normal((M, K)))
+    x = gen.f32_from_bf16_bits(xb).astype(np.float64)
+    out = oracle.linear_a16(xb, np.eye(n1, dtype=np.float32), np.eye(n2, dtype=np.float32), packed, alpha, mu=mu)
+    assert np.array_equal(gen.f32_from_bf16_bits(out["yhat"]).astype(np.float64), x)
+    want = (x @ S.T) * alpha.astype(np.float64)[None, :] + x.sum(axis=1)[:, None] * mu.astype(np.float64)[None, :]
+    np.testing.assert_allclose(out["y"], want, rtol=0, atol=1e-12 * np.abs(want).max())
+
+
+def test_a16_error_is_the_bf16_rounding_of_the_rotated_activation_and_below_the_8_bit_layer():
+    n1, n2, N, M, r = 8, 16, 64, 12, 8
+    K = n1 * n2
+    rng = np.random.default_rng(22)
+    P1, P2 = _orth(n1, 5), _orth(n2, 6)
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    packed = oracle.pack_signs(W)
+    S = np.where(W > 0, 1.0, -1.0)
+    alpha = rng.uniform(0.5, 2.0, N).astype(np.float32)
+    U = _bf16(0.05 * rng.standard_normal((N, r)))
+    V = _bf16(0.05 * rng.standard_normal((r, K)))
+    xb = _bf16(rng.standard_normal((M, K)))
+    a16 = oracle.linear_a16(xb, P1, P2, packed, alpha, U, V)
+    a8 = oracle.linear(xb, P1, P2, 8, packed, alpha, U, V)
+    exact = (a16["Y"] @ S.T) * alpha.astype(np.float64)[None, :] + oracle.lowrank(xb, U, V)
+    e16 = np.linalg.norm(a16["y"] - exact) / np.linalg.norm(exact)
+    e8 = np.linalg.norm(a8["y"] - exact) / np.linalg.norm(exact)
+    assert e16 < e8 < 2e-2
+    # every rotated value moved by at most half a bf16 step, so every output by at most alpha * sum_k 2^-9 |Y_k|
+    bound = alpha.astype(np.float64)[None, :] * (np.abs(a16["Y"]).sum(axis=1) * 2.0 ** -9)[:, None]
+    assert np.all(np.abs(a16["y"] - exact) <= bound + 1e-12)
+    # and the rounding itself is the bf16 rounding the rest of the oracle uses
+    assert np.array_equal(a16["yhat"], oracle.bf16_round(a16["Y"]))
