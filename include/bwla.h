@@ -203,6 +203,22 @@ int bwla_layer_rotate_quant(const bwla_layer* layer, const void* x_bf16, int64_t
 enum { BWLA_ACT_SYMMETRIC = 0, BWLA_ACT_ASYMMETRIC = 1 };
 int bwla_layer_set_activation_quant(bwla_layer* layer, int mode);
 
+/*
+ * The weight-only operating point, W1A16 (Table 1, upper half: binarised weights, 16-bit activations), on a prepared
+ * layer: the rotated activation Y = P1^T X P2 (Sec. 3.1) is rounded to bf16 instead of being quantised to integer codes,
+ *   out[t][n] = bf16( alpha[n] * sum_k sign[n][k] * bf16(Y[t][k]) + U (V x_t) [+ mu[n] * sum_k bf16(Y[t][k])] ),
+ * a bf16 contraction on the tensor cores with fp32 accumulation (partial sums of 128 values of k are added in rounded
+ * fp32).  The layer's activation bit width and quantiser mode are not used.
+ *   x_bf16 device, bf16 [M][ldx], 16-byte aligned, ldx >= K and a multiple of 8; out_bf16 device, bf16 [M][ldo], ldo >= N
+ *   workspace: 256-byte aligned device scratch of bwla_w1a16_workspace_bytes(layer, M) bytes (about 7 bytes per
+ *     activation value); its first 256 bytes must be zero before the first call; bwla_check_status reads it.
+ * Needs K % 64 == 0, r <= 64 and factor sizes the tensor-core rotation takes, else BWLA_ERR_UNSUPPORTED.  M == 0 is a
+ * no-op.  Asynchronous on `stream`.
+ */
+size_t bwla_w1a16_workspace_bytes(const bwla_layer* layer, int64_t M);
+int bwla_layer_w1a16_linear(const bwla_layer* layer, const void* x_bf16, int64_t M, int64_t ldx, void* out_bf16,
+                            int64_t ldo, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The asymmetric quantiser alone: codes device uint8 [M][K] (u), scales device fp32 [M], zeros device int32 [M] (z),
  * y_f32 device fp32 [M][K] or NULL. */
 int bwla_layer_rotate_quant_asym(const bwla_layer* layer, const void* x_bf16, int64_t M, int64_t ldx,

@@ -38,7 +38,7 @@ EXPORTS = [
     "bwla_workspace_section", "bwla_force_rotation", "bwla_layer_prepared_bytes", "bwla_layer_create",
     "bwla_layer_destroy", "bwla_layer_rotate_quant", "bwla_group_workspace_bytes", "bwla_w1ax_linear_group",
     "bwla_layer_set_activation_quant", "bwla_layer_rotate_quant_asym", "bwla_binarize_workspace_bytes",
-    "bwla_binarize_rows",
+    "bwla_binarize_rows", "bwla_w1a16_workspace_bytes", "bwla_layer_w1a16_linear",
 ]
 
 
@@ -85,6 +85,9 @@ def _load() -> C.CDLL:
     lib.bwla_layer_set_activation_quant.restype = ci
     lib.bwla_layer_rotate_quant_asym.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
     lib.bwla_layer_rotate_quant_asym.restype = ci
+    lib.bwla_w1a16_workspace_bytes.argtypes = [vp, i64]
+    lib.bwla_w1a16_workspace_bytes.restype = sz
+    lib.bwla_layer_w1a16_linear.argtypes = [vp, vp, i64, i64, vp, i64, vp, sz, vp]
     lib.bwla_group_workspace_bytes.argtypes = [C.POINTER(vp), ci, i64]
     lib.bwla_group_workspace_bytes.restype = sz
     lib.bwla_w1ax_linear_group.argtypes = [C.POINTER(vp), ci, vp, i64, i64, C.POINTER(vp), C.POINTER(i64), vp, sz, vp]
@@ -310,6 +313,26 @@ class Layer:
         if h is not None and h.value and _lib is not None:      # (_lib is None while the interpreter shuts down)
             _lib.bwla_layer_destroy(h)
             self.handle = C.c_void_p()
+
+
+def bwla_w1a16_workspace_bytes(layer: Layer, M: int) -> int:
+    return int(_lib.bwla_w1a16_workspace_bytes(layer.handle, M))
+
+
+def bwla_layer_w1a16_linear(layer: Layer, x: torch.Tensor, out: Optional[torch.Tensor] = None,
+                            workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The weight-only layer (W1A16): bf16 x [M][K] -> bf16 out [M][N], rotated activations kept in bf16."""
+    _need(x, torch.bfloat16, "x", 2)
+    M = x.shape[0]
+    if out is None:
+        out = torch.empty((M, layer.N), dtype=torch.bfloat16, device=x.device)
+    _need(out, torch.bfloat16, "out", 2)
+    if workspace is None:
+        workspace = torch.zeros(max(256, bwla_w1a16_workspace_bytes(layer, M)), dtype=torch.uint8, device=x.device)
+    st = _lib.bwla_layer_w1a16_linear(layer.handle, _ptr(x), M, x.stride(0) if M > 0 else layer.K, _ptr(out),
+                                      out.stride(0) if M > 0 else layer.N, _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "bwla_layer_w1a16_linear")
+    return out
 
 
 def bwla_layer_prepared_bytes(K: int, N: int, n1: int, n2: int, r: int) -> int:

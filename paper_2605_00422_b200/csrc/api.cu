@@ -349,6 +349,53 @@ int bwla_layer_rotate_quant(const bwla_layer* L, const void* x_bf16, int64_t M, 
                            nullptr, nullptr, nullptr, (cudaStream_t)stream);
 }
 
+struct A16Workspace { size_t status, Y, yhat, ysum, codes, scales, T, lr_part, total; };
+static A16Workspace a16_layout(const bwla_layer* L, int64_t M) {
+    A16Workspace w{};
+    size_t off = 0;
+    w.status = off; off += kStatusBytes;
+    w.Y = off;      off += align_up((size_t)M * (size_t)L->K * 4, 256);
+    w.yhat = off;   off += align_up((size_t)M * (size_t)L->K * 2, 256);
+    w.ysum = off;   off += align_up((size_t)M * 4, 256);
+    w.codes = off;  off += align_up((size_t)M * (size_t)L->K, 256);
+    w.scales = off; off += align_up((size_t)M * 4, 256);
+    const size_t lr_cols = (size_t)lowrank_cols(L->r);
+    w.T = off;      off += align_up((size_t)M * lr_cols * 6, 256);
+    w.lr_part = off; off += L->r > 0 ? align_up(std::max((size_t)kLrKSplitMax * 16 * lr_cols * 4, lowrank_umma_part_bytes(M, L->K, L->r)), 256) : 0;
+    w.total = off;
+    return w;
+}
+
+size_t bwla_w1a16_workspace_bytes(const bwla_layer* layer, int64_t M) {
+    if (!layer || M < 0) return 0;
+    return a16_layout(layer, M).total;
+}
+
+int bwla_layer_w1a16_linear(const bwla_layer* L, const void* x_bf16, int64_t M, int64_t ldx, void* out_bf16, int64_t ldo,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+    g_launch_count = 0;
+    if (!L || M < 0 || ldx < L->K || ldo < L->N) return BWLA_ERR_INVALID_ARG;
+    if (M == 0) return BWLA_OK;
+    if (!x_bf16 || !out_bf16) return BWLA_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < bwla_w1a16_workspace_bytes(L, M)) return BWLA_ERR_WORKSPACE;
+    int st = check_device();
+    if (st != BWLA_OK) return st;
+    if (!L->okt || !okt_accepts_x(x_bf16, ldx) || !a16_supports(M, L->K, L->N, L->r)) return BWLA_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)stream;
+    const A16Workspace w = a16_layout(L, M);
+    char* base = (char*)workspace;
+    uint32_t* status = (uint32_t*)(base + w.status);
+    // the rotation hands out Y in fp32 (its int8 codes, quantised at 8 bits, are a by-product nobody reads here)
+    OktProblem pr{L->prepared, (int8_t*)(base + w.codes), 0, nullptr, 0, (float*)(base + w.scales), nullptr, (float*)(base + w.Y)};
+    OktLowrank lr{L->V, L->r, base + w.T, L->r > 0 ? (float*)(base + w.lr_part) : nullptr, status + kLrCounterWord};
+    st = launch_okt(L->geom, x_bf16, M, ldx, 8, 0, 1, &pr, &lr, status, s);
+    if (st != BWLA_OK) return st;
+    st = launch_y_to_bf16((const float*)(base + w.Y), M, L->K, base + w.yhat, (float*)(base + w.ysum), s);
+    if (st != BWLA_OK) return st;
+    return launch_gemm_a16(base + w.yhat, (const float*)(base + w.ysum), M, L->K, L->N, L->packed, L->alpha, L->mu, L->U, L->r,
+                           L->r > 0 ? base + w.T : nullptr, out_bf16, ldo, status, s);
+}
+
 static bool valid_group(const bwla_layer* const* layers, int count) {
     if (!layers || count < 1 || count > kOktMaxProblems) return false;
     for (int i = 0; i < count; ++i) {

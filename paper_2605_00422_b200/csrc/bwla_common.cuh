@@ -213,6 +213,14 @@ struct GemmArgs {
 };
 enum { kDepChain = 0, kDepHead = 1, kDepSibling = 2 };
 
+// W1A16, the weight-only operating point (gemm_a16.cu): Y (fp32) -> bf16 + per-token sums; the bf16 contraction against
+// the packed signs with the fused epilogue.  Thl as for the int8 contractions (NULL when r == 0).
+bool a16_supports(int64_t M, int64_t K, int64_t N, int r);
+int launch_y_to_bf16(const float* Y, int64_t M, int64_t K, void* yhat, float* ysum, cudaStream_t stream);
+int launch_gemm_a16(const void* yhat, const float* ysum, int64_t M, int64_t K, int64_t N, const uint32_t* packed, const float* alpha,
+                    const float* mu, const void* U, int r, const void* Thl, void* out, int64_t ldo, uint32_t* status,
+                    cudaStream_t stream);
+
 // Final binarisation of weight rows in the rotated coordinates (binarize.cu).
 size_t binarize_workspace_bytes(int64_t K);
 int launch_binarize(const void* w, int dtype, int64_t N, int64_t K, int64_t ldw, const float* P1, int n1, const float* P2, int n2,
