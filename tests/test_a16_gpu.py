@@ -60,3 +60,24 @@ def test_qwen32b_shapes(bwla, idx, M):
 def test_prefill_sized_batch_on_sampled_tokens(bwla):
     M = 2048
     _case(bwla, 2, gen.CONFIG_SHAPES[2][0], M, sample=H.token_sample(M))
+
+
+@pytest.mark.parametrize("K,N,n1,n2,r,M", [
+    (192, 200, 12, 16, 0, 5),         # three k-blocks (an odd number: the last accumulator holds one), ragged rows, no low-rank branch
+    (1024, 129, 32, 32, 13, 130),     # one row beyond a tile, a rank that is not a multiple of 8, a ragged second token tile
+    (64, 8, 8, 8, 4, 1),              # a single k-block, one token
+    (2048, 384, 32, 64, 64, 17),      # the full rank of 64
+])
+def test_small_and_ragged_shapes(bwla, K, N, n1, n2, r, M):
+    sh = gen.small_shape(K, N, n1, n2, r, shape_id=K + N)
+    lay = gen.make_layer(0, sh, 8, with_mu=(r == 13))
+    xb = gen.make_activations(0, sh, M)
+    dl = H.DeviceLayer(lay, bwla)
+    layer = bwla.Layer(dl.P1, dl.P2, 8, dl.packed, dl.alpha, dl.U, dl.V, mu=dl.mu)
+    ws = torch.zeros(bwla.bwla_w1a16_workspace_bytes(layer, M), dtype=torch.uint8, device="cuda")
+    out = torch.full((M, N + 3), 7.0, dtype=torch.bfloat16, device="cuda")       # a row stride that is not a multiple of 8
+    bwla.bwla_layer_w1a16_linear(layer, H.bf16_to_dev(xb), out=out[:, :N], workspace=ws)
+    assert bwla.bwla_check_status(ws) == 0
+    assert torch.all(out[:, N:] == 7.0)                                           # nothing written beyond the rows
+    ref = oracle.linear_a16(xb, lay.P1, lay.P2, dl.packed_host, lay.alpha, lay.U, lay.V, mu=lay.mu)
+    H.check_output(H.bf16_to_host(out[:, :N].contiguous()), ref["y"])
