@@ -481,6 +481,39 @@ def run_ours(args):
     sampler = ClockSampler(uuid)
 
     # ------------------------------ decode ------------------------------
+    # the weight-only operating point (Table 1, upper half): W1A16, rotated activations kept in bf16
+    def measure_w1a16():
+        def a16_step(xs_, outs_, ws_, layers_):
+            for row in stack[:layers_]:
+                for lin in row:
+                    bwla.bwla_layer_w1a16_linear(lin.layer, xs_[lin.shape.K], out=outs_[lin.shape.name], workspace=ws_)
+        res = {"workload": "same stack, W1A16 (bf16 rotated activations against the packed signs, bf16 tensor-core contraction)"}
+        for Ma, La in ((args.decode_m, args.layers), (args.prefill_m, min(args.layers, 16))):
+            if Ma <= 0:
+                continue
+            xs_a, outs_a, _ = make_io(Ma)
+            ws_a = torch.zeros(max(bwla.bwla_w1a16_workspace_bytes(l.layer, Ma) for l in stack[0]), dtype=torch.uint8, device=device)
+            a16_step(xs_a, outs_a, ws_a, 1)
+            torch.cuda.synchronize()
+            g_a = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_a):
+                a16_step(xs_a, outs_a, ws_a, La)
+            ms_a = timed(g_a.replay, 3, 2) / 3 * (args.layers / La)
+            res[f"M{Ma}"] = {"ms_per_step": ms_a, "layers_timed": La,
+                             "GB/s": world * args.layers * sum(call_bytes(sh, Ma) for sh in shapes) / (ms_a * 1e-3) / 1e9,
+                             "TFLOP/s (2MKN)": world * args.layers * sum(call_ops(sh, Ma) for sh in shapes) / (ms_a * 1e-3) / 1e12,
+                             "status": bwla.bwla_check_status(ws_a)}
+            del g_a, ws_a, xs_a, outs_a
+            torch.cuda.empty_cache()
+        return res
+
+    if args.only_w1a16:
+        if rank == 0:
+            print(json.dumps({"w1a16": measure_w1a16()}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     M = args.decode_m
     xs, outs, ws = make_io(M)
     graph, launches_per_step = capture(xs, outs, ws)
@@ -576,31 +609,7 @@ def run_ours(args):
                 lin.layer = bwla.Layer(lin.P1, lin.P2, BITS, lin.packed, lin.alpha, lin.U, lin.V)
         torch.cuda.synchronize()
 
-    # the weight-only operating point (Table 1, upper half): W1A16, rotated activations kept in bf16
-    w1a16 = None
-    if not args.skip_extras:
-        def a16_step(xs_, outs_, ws_, layers_):
-            for row in stack[:layers_]:
-                for lin in row:
-                    bwla.bwla_layer_w1a16_linear(lin.layer, xs_[lin.shape.K], out=outs_[lin.shape.name], workspace=ws_)
-        w1a16 = {"workload": "same stack, W1A16 (bf16 rotated activations against the packed signs, bf16 tensor-core contraction)"}
-        for Ma, La in ((M, args.layers), (args.prefill_m, min(args.layers, 16))):
-            if Ma <= 0:
-                continue
-            xs_a, outs_a, _ = make_io(Ma)
-            ws_a = torch.zeros(max(bwla.bwla_w1a16_workspace_bytes(l.layer, Ma) for l in stack[0]), dtype=torch.uint8, device=device)
-            a16_step(xs_a, outs_a, ws_a, 1)
-            torch.cuda.synchronize()
-            g_a = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g_a):
-                a16_step(xs_a, outs_a, ws_a, La)
-            ms_a = timed(g_a.replay, 3, 2) / 3 * (args.layers / La)
-            w1a16[f"M{Ma}"] = {"ms_per_step": ms_a, "layers_timed": La,
-                               "GB/s": world * args.layers * sum(call_bytes(sh, Ma) for sh in shapes) / (ms_a * 1e-3) / 1e9,
-                               "TFLOP/s (2MKN)": world * args.layers * sum(call_ops(sh, Ma) for sh in shapes) / (ms_a * 1e-3) / 1e12,
-                               "status": bwla.bwla_check_status(ws_a)}
-            del g_a, ws_a, xs_a, outs_a
-            torch.cuda.empty_cache()
+    w1a16 = measure_w1a16() if not args.skip_extras else None
 
     # ------------------------------ prefill ------------------------------
     prefill = None
@@ -695,6 +704,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cublas", action="store_true", help="skip the cuBLAS bf16 context measurement")
     ap.add_argument("--skip-extras", action="store_true", help="skip the forced-path, W1A8 batch-4 and W1A16 steps")
+    ap.add_argument("--only-w1a16", action="store_true", help="time only the W1A16 (weight-only) stack and print its figures")
     ap.add_argument("--per-shape", action="store_true", help="time every shape of workload configs 1-3 on its own and print a table")
     ap.add_argument("--shape", default=None, help="with --per-shape: only the shape of this name (e.g. q_gate)")
     ap.add_argument("--cfg", type=int, default=0, help="with --per-shape: only this workload config (1, 2 or 3)")

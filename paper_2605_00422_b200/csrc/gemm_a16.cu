@@ -69,14 +69,13 @@ __global__ void __launch_bounds__(256) y_to_bf16_kernel(const float* __restrict_
     }
 }
 
-// Eight sign bits (bit 1 = +1) -> eight bf16 values +-1, two per word, the lower k in the low half.
-__device__ __forceinline__ uint4 expand8(uint32_t bits) {
+// Eight sign bits (bit 1 = +1), given inverted in the low byte of `nbits` -> eight bf16 values +-1, two per word, the
+// lower k in the low half.  A pair of inverted bits t = b0 + 2 b1 times (2^15 + 2^30) puts b0 at bit 15 and b1 at bit
+// 31 (and copies at bits 16 and 30, masked off): three instructions per word.
+__device__ __forceinline__ uint4 expand8(uint32_t nbits) {
     uint32_t w[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t lo = (~bits >> (2 * i)) & 1u, hi = (~bits >> (2 * i + 1)) & 1u;
-        w[i] = 0x3F803F80u | (lo << 15) | (hi << 31);
-    }
+    for (int i = 0; i < 4; ++i) w[i] = 0x3F803F80u | ((((nbits >> (2 * i)) & 3u) * 0x40008000u) & 0x80008000u);
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
@@ -199,21 +198,31 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
         const uint2* words = reinterpret_cast<const uint2*>(p.packed + (size_t)(valid ? n : 0) * (size_t)(p.K >> 5));
         bool ok = !*abort_flag;
         int s = 0; uint32_t ph = 0;
-        uint2 next = (ok && nblocks > 0) ? __ldg(words) : make_uint2(0u, 0u);
-        for (int b = 0; b < nblocks && ok; ++b) {
-            const uint2 cur = next;
-            if (b + 1 < nblocks) next = __ldg(words + b + 1);
-            if (!warp_wait(&empty[s], ph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x330); ok = false; break; }
-            uint8_t* dst = smem + s * stage_bytes + a_bytes + row * 128;
+        // The sign words come straight from global memory, 8 bytes per row and stage; eight stages' worth are kept in
+        // flight per thread (one stage ahead left the loop waiting for the memory latency at every stage).
+        constexpr int kAhead = 8;
+        uint2 ring[kAhead];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t byte = ((c < 4 ? cur.x : cur.y) >> (8 * (c & 3))) & 0xFFu;
-                *reinterpret_cast<uint4*>(dst + ((c ^ (row & 7)) << 4)) = expand8(byte);
+        for (int j = 0; j < kAhead; ++j) ring[j] = (ok && j < nblocks) ? __ldg(words + j) : make_uint2(0u, 0u);
+        for (int b0 = 0; b0 < nblocks && ok; b0 += kAhead) {
+#pragma unroll
+            for (int j = 0; j < kAhead; ++j) {
+                const int b = b0 + j;
+                if (b >= nblocks || !ok) break;
+                const uint2 cur = make_uint2(~ring[j].x, ~ring[j].y);      // inverted once: a set bit now means -1
+                if (b + kAhead < nblocks) ring[j] = __ldg(words + b + kAhead);
+                if (!warp_wait(&empty[s], ph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x330); ok = false; break; }
+                uint8_t* dst = smem + s * stage_bytes + a_bytes + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t byte = ((c < 4 ? cur.x : cur.y) >> (8 * (c & 3))) & 0xFFu;
+                    *reinterpret_cast<uint4*>(dst + ((c ^ (row & 7)) << 4)) = expand8(byte);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&b_full[s]);
+                if (++s == kStages) { s = 0; ph ^= 1u; }
             }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&b_full[s]);
-            if (++s == kStages) { s = 0; ph ^= 1u; }
         }
         if (ok && lowrank) {
             // this tile's rows of U: 128 rows x 8 chunks of 16 bytes, 128B-swizzled K-major, zero beyond N and r
