@@ -7,11 +7,12 @@
 //
 // Tile of one CTA: 128 tokens (the accumulator's lanes) x 128 weight rows (its columns) x all of K.
 //   A operand: yhat, K-major, by TMA (64 values of k = one 128-byte swizzle atom per stage);
-//   B operand: the signs of 128 rows expanded to +-1 in bf16 by four warps (one thread per row: 64 bits in, eight
-//              128-bit shared-memory stores out, in the swizzled K-major layout the MMA reads);
+//   B operand: the signs of 128 rows expanded to +-1 in bf16 by four warps (each owns one stage and takes every fourth
+//              k-block: 64 bits in, eight 128-bit shared-memory stores out per row, swizzled K-major);
 //   the tensor core adds each group of 16 products into its accumulator with truncation, so the accumulator only ever
-//   holds 128 values of k: after every 128 it is read back and added, with rounded fp32 additions, into running sums in
-//   the epilogue warps' registers while the next 128 go to the second accumulator (as in lowrank_umma.cu);
+//   holds 512 values of k (32 such additions: a bias of at most 2e-6 of the sum of magnitudes, far below the bf16
+//   output): after every 512 it is read back and added, with rounded fp32 additions, into running sums in the epilogue
+//   warps' registers while the next 512 go to the second accumulator (as in lowrank_umma.cu);
 //   the low-rank term is twelve more MMAs (three bf16 terms of T against the tile's rows of U) into a third accumulator.
 // Warp 0 copies, warp 1 allocates tensor memory and issues the MMAs, warps 2..5 expand signs and stage U, warps 6..13
 // are the epilogue (two per quarter of the lanes, 64 columns each).  Every wait is bounded (umma_wait.cuh).
@@ -27,12 +28,15 @@
 namespace bwla {
 
 namespace a16 {
-constexpr int kTok = 128, kRows = 128, kBlockK = 64, kFlushBlocks = 2, kStages = 4;
+constexpr int kTok = 128, kRows = 128, kBlockK = 64, kFlushBlocks = 8;
+// The yhat tiles come by TMA and take about a microsecond to land, the sign tiles are made on the SM: the ring of the
+// former is deep (what bounds the loop is tiles in flight over that latency), the ring of the latter short.
+constexpr int kAStages = 7, kBStages = 4;            // (an expander warp owns one sign stage: kBStages == 4 warps)
 constexpr int kExpFirst = 64, kEpiFirst = 192, kThreads = 448;
-constexpr int a_bytes = kTok * 128, b_bytes = kRows * 128, stage_bytes = a_bytes + b_bytes;
-constexpr int u_off = kStages * stage_bytes;
-constexpr int t_off = u_off + kRows * 128;
-constexpr int par_off = t_off + 3 * a_bytes;                  // alpha[128], mu[128]
+constexpr int a_bytes = kTok * 128, b_bytes = kRows * 128;
+constexpr int b_off = kAStages * a_bytes;
+constexpr int u_off = b_off + kBStages * b_bytes;
+constexpr int par_off = u_off + kRows * 128;                  // alpha[128], mu[128]
 constexpr int bars_off = par_off + 2 * kRows * 4;
 constexpr int smem_bytes = bars_off + 256 + 1024;
 constexpr int ACC_COL = 0, LR_COL = 2 * kRows, kTmemCols = 512;
@@ -85,14 +89,14 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ubuf = smem + u_off;
-    uint8_t* tbuf = smem + t_off;
     float* alpha_s = reinterpret_cast<float*>(smem + par_off);
     float* mu_s = alpha_s + kRows;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + bars_off);
-    uint64_t* a_full = bars;                  // [kStages] yhat tile landed
-    uint64_t* b_full = a_full + kStages;      // [kStages] signs expanded
-    uint64_t* empty = b_full + kStages;       // [kStages] the stage's MMAs have completed
-    uint64_t* acc_full = empty + kStages;     // [2]
+    uint64_t* a_full = bars;                  // [kAStages] yhat tile landed
+    uint64_t* a_empty = a_full + kAStages;    // [kAStages] the MMAs that read it have completed
+    uint64_t* b_full = a_empty + kAStages;    // [kBStages] signs expanded
+    uint64_t* b_empty = b_full + kBStages;    // [kBStages]
+    uint64_t* acc_full = b_empty + kBStages;  // [2]
     uint64_t* acc_free = acc_full + 2;        // [2]
     uint64_t* u_full = acc_free + 2;
     uint64_t* t_full = u_full + 1;
@@ -108,7 +112,8 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
 
     if (threadIdx.x == 0) {
         *abort_flag = (p.status && *reinterpret_cast<volatile uint32_t*>(p.status) != 0) ? 1 : 0;   // the call already failed
-        for (int i = 0; i < kStages; ++i) { mbar_init(&a_full[i], 1); mbar_init(&b_full[i], 4); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < kAStages; ++i) { mbar_init(&a_full[i], 1); mbar_init(&a_empty[i], 1); }
+        for (int i = 0; i < kBStages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_free[i], 8); }
         mbar_init(u_full, 4); mbar_init(t_full, 1); mbar_init(lr_full, 1);
         fence_barrier_init();
@@ -129,20 +134,25 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- copies: the three terms of T once, then the yhat tile stage by stage ----------------
+        // ---------------- copies: the yhat tile stage by stage, then the three terms of T into the next three slots ----------------
         if (elect_one()) {
             tma_prefetch_desc(&y_map);
-            if (lowrank && !*abort_flag) {
-                tma_prefetch_desc(&t_map);
-                mbar_expect_tx(t_full, 3 * a_bytes);
-                for (int h = 0; h < 3; ++h) tma_load_3d(tbuf + h * a_bytes, &t_map, 0, t0, h, t_full);
-            }
+            if (lowrank) tma_prefetch_desc(&t_map);
             int s = 0; uint32_t ph = 0;
-            for (int b = 0; b < nblocks && !*abort_flag; ++b) {
-                if (!wait_or_abort(&empty[s], ph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x310); break; }
+            bool ok = !*abort_flag;
+            for (int b = 0; b < nblocks && ok && !*abort_flag; ++b) {
+                if (!wait_or_abort(&a_empty[s], ph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x310); ok = false; break; }
                 mbar_expect_tx(&a_full[s], a_bytes);
-                tma_load_2d(smem + s * stage_bytes, &y_map, b * kBlockK, t0, &a_full[s]);
-                if (++s == kStages) { s = 0; ph ^= 1u; }
+                tma_load_2d(smem + s * a_bytes, &y_map, b * kBlockK, t0, &a_full[s]);
+                if (++s == kAStages) { s = 0; ph ^= 1u; }
+            }
+            if (lowrank && ok && !*abort_flag) {
+                mbar_expect_tx(t_full, 3 * a_bytes);
+                for (int h = 0; h < 3 && ok; ++h) {
+                    if (!wait_or_abort(&a_empty[s], ph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x311); ok = false; break; }
+                    tma_load_3d(smem + s * a_bytes, &t_map, 0, t0, h, t_full);
+                    if (++s == kAStages) { s = 0; ph ^= 1u; }
+                }
             }
             if (*abort_flag) for (int i = 0; i < 500; ++i) __nanosleep(100);   // let copies in flight land
         }
@@ -151,7 +161,11 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
         if (elect_one()) {
             // D = f32, A = B = bf16, both K-major, M = 128, N = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kRows >> 3) << 17) | ((128u >> 4) << 24);
-            int s = 0; uint32_t ph = 0;
+            const uint64_t desc0 = smem_desc_sw128(0u, 0u);                         // everything but the start address
+            const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)desc0 | ((smem_u32(smem) & 0x3FFFFu) >> 4);
+            const uint32_t b_lo0 = (uint32_t)desc0 | ((smem_u32(smem + b_off) & 0x3FFFFu) >> 4);
+            int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
             bool ok = !*abort_flag;
             int b = 0;
             for (int u = 0; u < units && ok; ++u) {
@@ -160,15 +174,21 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
                 tc_fence_after();
                 const uint32_t d_addr = tmem_base + ACC_COL + (uint32_t)(buf * kRows);
                 for (int i = 0; i < kFlushBlocks && b < nblocks; ++i, ++b) {
-                    if (!wait_or_abort(&a_full[s], ph, abort_flag)) { give_up(p.status, abort_flag, 0x321); ok = false; break; }
-                    if (!wait_or_abort(&b_full[s], ph, abort_flag)) { give_up(p.status, abort_flag, 0x322); ok = false; break; }
+                    if (!wait_or_abort(&a_full[sa], pha, abort_flag)) { give_up(p.status, abort_flag, 0x321); ok = false; break; }
+                    if (!wait_or_abort(&b_full[sb], phb, abort_flag)) { give_up(p.status, abort_flag, 0x322); ok = false; break; }
                     tc_fence_after();
-                    const uint32_t ya = smem_u32(smem + s * stage_bytes), sa = ya + a_bytes;
+                    // (this thread is a chain of dependent scalar instructions: descriptors are a constant high word and a
+                    // low word that only takes additions)
+                    const uint32_t a_lo = a_lo0 + (uint32_t)sa * (a_bytes >> 4), g_lo = b_lo0 + (uint32_t)sb * (b_bytes >> 4);
+                    if (i == 0) mma_f16_ss_words<false>(d_addr, a_lo, desc_hi, g_lo, desc_hi, idesc);
+                    else mma_f16_ss_words<true>(d_addr, a_lo, desc_hi, g_lo, desc_hi, idesc);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        mma_f16_ss(d_addr, smem_desc_sw128(ya, 32 * j), smem_desc_sw128(sa, 32 * j), idesc, (i | j) ? 1u : 0u);
-                    tc_commit(&empty[s]);
-                    if (++s == kStages) { s = 0; ph ^= 1u; }
+                    for (int j = 1; j < 4; ++j)
+                        mma_f16_ss_words<true>(d_addr, a_lo + 2u * j, desc_hi, g_lo + 2u * j, desc_hi, idesc);
+                    tc_commit(&a_empty[sa]);
+                    tc_commit(&b_empty[sb]);
+                    if (++sa == kAStages) { sa = 0; pha ^= 1u; }
+                    if (++sb == kBStages) { sb = 0; phb ^= 1u; }
                 }
                 if (ok) tc_commit(&acc_full[buf]);
             }
@@ -180,11 +200,13 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
                     const uint32_t u_addr = smem_u32(ubuf);
 #pragma unroll
                     for (int h = 0; h < 3; ++h) {
-                        const uint32_t t_addr = smem_u32(tbuf + h * a_bytes);
+                        // (the terms of T sit in the three slots of the yhat ring that follow the last yhat tile)
+                        const uint32_t t_addr = smem_u32(smem + sa * a_bytes);
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
                             mma_f16_ss(tmem_base + LR_COL, smem_desc_sw128(t_addr, 32 * j), smem_desc_sw128(u_addr, 32 * j), idesc,
                                        (h | j) ? 1u : 0u);
+                        if (++sa == kAStages) sa = 0;
                     }
                     tc_commit(lr_full);
                 }
@@ -192,37 +214,46 @@ a16_gemm_kernel(const __grid_constant__ CUtensorMap y_map, const __grid_constant
         }
     } else if (warp < 6) {
         // ---------------- signs of the tile's 128 rows -> +-1 in bf16, K-major, swizzled; then the rows of U ----------------
-        const int row = threadIdx.x - kExpFirst;
+        // Expander warp w takes the k-blocks w, w + 4, ... and owns sign stage w: what a warp does per block (wait for
+        // its stage, 32 stores, the fence that makes them visible to the tensor core's reads, the hand-over) is a serial
+        // chain of several hundred cycles whatever its size, so four blocks are in the making at once.  A lane expands
+        // the rows lane, lane + 32, lane + 64, lane + 96 of the tile.
+        const int w = warp - 2;
+        const int row = threadIdx.x - kExpFirst;            // (for the rows of U below)
         const int n = n0 + row;
         const bool valid = n < p.N;
-        const uint2* words = reinterpret_cast<const uint2*>(p.packed + (size_t)(valid ? n : 0) * (size_t)(p.K >> 5));
+        const uint2* words[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int ni = n0 + lane + 32 * i;
+            words[i] = reinterpret_cast<const uint2*>(p.packed + (size_t)(ni < p.N ? ni : 0) * (size_t)(p.K >> 5));
+        }
         bool ok = !*abort_flag;
-        int s = 0; uint32_t ph = 0;
-        // The sign words come straight from global memory, 8 bytes per row and stage; eight stages' worth are kept in
-        // flight per thread (one stage ahead left the loop waiting for the memory latency at every stage).
-        constexpr int kAhead = 8;
-        uint2 ring[kAhead];
+        uint2 nxt[4];
 #pragma unroll
-        for (int j = 0; j < kAhead; ++j) ring[j] = (ok && j < nblocks) ? __ldg(words + j) : make_uint2(0u, 0u);
-        for (int b0 = 0; b0 < nblocks && ok; b0 += kAhead) {
+        for (int i = 0; i < 4; ++i) nxt[i] = (ok && w < nblocks) ? __ldg(words[i] + w) : make_uint2(0u, 0u);
+        uint8_t* const stage = smem + b_off + w * b_bytes;
+        for (int b = w; b < nblocks && ok; b += kBStages) {
+            uint2 cur[4];
 #pragma unroll
-            for (int j = 0; j < kAhead; ++j) {
-                const int b = b0 + j;
-                if (b >= nblocks || !ok) break;
-                const uint2 cur = make_uint2(~ring[j].x, ~ring[j].y);      // inverted once: a set bit now means -1
-                if (b + kAhead < nblocks) ring[j] = __ldg(words + b + kAhead);
-                if (!warp_wait(&empty[s], ph ^ 1u, abort_flag)) { give_up(p.status, abort_flag, 0x330); ok = false; break; }
-                uint8_t* dst = smem + s * stage_bytes + a_bytes + row * 128;
+            for (int i = 0; i < 4; ++i) {
+                cur[i] = make_uint2(~nxt[i].x, ~nxt[i].y);            // inverted once: a set bit now means -1
+                if (b + kBStages < nblocks) nxt[i] = __ldg(words[i] + b + kBStages);
+            }
+            if (!warp_wait(&b_empty[w], (uint32_t)(((b >> 2) & 1) ^ 1), abort_flag)) { give_up(p.status, abort_flag, 0x330); ok = false; break; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = lane + 32 * i;
+                uint8_t* dst = stage + r * 128;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    const uint32_t byte = ((c < 4 ? cur.x : cur.y) >> (8 * (c & 3))) & 0xFFu;
-                    *reinterpret_cast<uint4*>(dst + ((c ^ (row & 7)) << 4)) = expand8(byte);
+                    const uint32_t byte = ((c < 4 ? cur[i].x : cur[i].y) >> (8 * (c & 3))) & 0xFFu;
+                    *reinterpret_cast<uint4*>(dst + ((c ^ (r & 7)) << 4)) = expand8(byte);
                 }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&b_full[s]);
-                if (++s == kStages) { s = 0; ph ^= 1u; }
             }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&b_full[w]);
         }
         if (ok && lowrank) {
             // this tile's rows of U: 128 rows x 8 chunks of 16 bytes, 128B-swizzled K-major, zero beyond N and r
